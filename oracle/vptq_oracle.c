@@ -1,0 +1,350 @@
+/*
+ * CPU oracle for the inference side of VPTQ (vector post-training quantization).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow definition of what the
+ * vector-quantized linear layer computes.  It is used by the tests, by the smoke
+ * check and by the benchmark's CPU-baseline leg; the product path never calls it
+ * and it shares no code, header, table or helper with the CUDA library.
+ *
+ * What is defined here and where the paper states it:
+ *   - a weight matrix W (M x N, M = output features, N = input features) is cut
+ *     into length-v vectors that run down a column (Sec. 2.2; Sec. 3.1, the
+ *     quantized column is a stack of centroids; Algorithm 1 inner loop over
+ *     m = 0, V, 2V, ...);
+ *   - inference restores the weight from the lookup table by index (Sec. 2.2
+ *     "dequantizes the original weight matrix from the lookup table by index and
+ *     centroid"; Sec. 4 last sentence);
+ *   - residual VQ decode reads one centroid from every table and sums them
+ *     (Sec. 3.2.2, last sentence);
+ *   - outlier columns use their own table with their own vector length
+ *     (Sec. 3.2.3; App. C.1 "Parameter Description"), and have no residual stage
+ *     (Algorithm 2 order; index-bit formula of App. C.2);
+ *   - the weights are restored to FP16 and then multiplied (App. D.2).
+ *   - size accounting: compression ratio / equivalent bit width (Sec. 2.2) and
+ *     the index-bit / codebook-bit formulas (App. C.2).
+ *
+ * Not stated by the paper, defined by this project (parity unpinned by the
+ * paper, consistency-checked only): the per-input-channel scale and bias and
+ * their FP32 operation order, the bit-packed index stream, and "the first
+ * n_out columns are the outlier columns".
+ *
+ * Arithmetic: lookup sum, scale and bias in FP32 with three separately rounded
+ * operations (build with -ffp-contract=off), result rounded to FP16
+ * (round-to-nearest-even), matmul in FP64 over the FP16-rounded weights with n
+ * ascending.
+ *
+ * OpenMP pragmas only split independent output rows across cores for timing;
+ * they change no result.
+ */
+#include <stdint.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------ */
+/* FP16 / BF16 <-> FP32, written at the bit level (IEEE 754 binary16)   */
+/* ------------------------------------------------------------------ */
+
+static float bits_to_float(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+static uint32_t float_to_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+float oracle_half_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) << 31;
+    uint32_t e = (h >> 10) & 0x1F;
+    uint32_t m = h & 0x3FF;
+    if (e == 0) {
+        if (m == 0) return bits_to_float(sign);
+        /* subnormal: value = m * 2^-24 */
+        float v = (float)m * (1.0f / 16777216.0f);
+        return (sign ? -v : v);
+    }
+    if (e == 31) return bits_to_float(sign | 0x7F800000u | (m << 13));
+    return bits_to_float(sign | ((e + 112) << 23) | (m << 13));
+}
+
+uint16_t oracle_float_to_half(float f)
+{
+    uint32_t u = float_to_bits(f);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000);
+    uint32_t a = u & 0x7FFFFFFFu;
+    if (a > 0x7F800000u) return (uint16_t)(sign | 0x7E00 | ((a >> 13) & 0x3FF)); /* NaN */
+    if (a >= 0x477FF000u) return (uint16_t)(sign | 0x7C00); /* >= 65520 rounds to inf */
+    int32_t e = (int32_t)(a >> 23) - 127;
+    if (e >= -14) {
+        /* normal half: keep 10 mantissa bits, round to nearest even on the 13 dropped */
+        uint32_t mant = a & 0x7FFFFF;
+        uint32_t h = ((uint32_t)(e + 15) << 10) | (mant >> 13);
+        uint32_t rem = mant & 0x1FFF;
+        if (rem > 0x1000 || (rem == 0x1000 && (h & 1))) h++;   /* carry may bump the exponent: still right */
+        return (uint16_t)(sign | h);
+    }
+    if (e < -25) return sign;   /* below half of the smallest subnormal (2^-25 itself handled below) */
+    /* subnormal half: value / 2^-24 rounded to nearest even integer */
+    uint32_t mant = (a & 0x7FFFFF) | 0x800000;      /* 24-bit significand, value = mant * 2^(e-23) */
+    int shift = (-e - 24) + 23;                     /* result = mant >> shift, with e in [-25,-15] -> shift in [14,24] */
+    uint32_t h = mant >> shift;
+    uint32_t rem = mant & ((1u << shift) - 1);
+    uint32_t half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (h & 1))) h++;
+    return (uint16_t)(sign | h);
+}
+
+float oracle_bf16_to_float(uint16_t b) { return bits_to_float((uint32_t)b << 16); }
+
+uint16_t oracle_float_to_bf16(float f)
+{
+    uint32_t u = float_to_bits(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x40);
+    uint32_t lsb = (u >> 16) & 1;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/* ------------------------------------------------------------------ */
+/* Bit-packed index stream (project-defined format)                    */
+/* ------------------------------------------------------------------ */
+/* b = max(1, ceil(log2 k)) bits per index.  Every row of the index matrix is its
+ * own little-endian bit stream: index c occupies stream bits [c*b, c*b+b), stream
+ * bit i is bit (i % 8) of byte (i / 8).  A row occupies ceil(cols*b/8) bytes rounded
+ * up to a multiple of 16; pad bits are zero. */
+
+int oracle_index_bits(int32_t k)
+{
+    int b = 0;
+    while (((int64_t)1 << b) < (int64_t)k) b++;
+    return b < 1 ? 1 : b;
+}
+
+int64_t oracle_row_bytes(int32_t cols, int32_t k)
+{
+    int64_t bits = (int64_t)cols * oracle_index_bits(k);
+    int64_t bytes = (bits + 7) / 8;
+    return (bytes + 15) / 16 * 16;
+}
+
+int64_t oracle_packed_bytes(int32_t rows, int32_t cols, int32_t k)
+{
+    return (int64_t)rows * oracle_row_bytes(cols, k);
+}
+
+/* returns 0, or -1 when some index lies outside [0, k) (nothing useful is written then) */
+int oracle_pack(const int32_t *idx, int32_t rows, int32_t cols, int32_t k, uint8_t *out)
+{
+    int b = oracle_index_bits(k);
+    int64_t stride = oracle_row_bytes(cols, k);
+    memset(out, 0, (size_t)(stride * rows));
+    for (int32_t r = 0; r < rows; r++) {
+        uint8_t *row = out + (int64_t)r * stride;
+        for (int32_t c = 0; c < cols; c++) {
+            int32_t val = idx[(int64_t)r * cols + c];
+            if (val < 0 || val >= k) return -1;
+            for (int i = 0; i < b; i++) {
+                if ((val >> i) & 1) {
+                    int64_t bit = (int64_t)c * b + i;
+                    row[bit / 8] |= (uint8_t)(1u << (bit % 8));
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+static int32_t read_index(const uint8_t *row, int64_t c, int b)
+{
+    int32_t val = 0;
+    for (int i = 0; i < b; i++) {
+        int64_t bit = c * b + i;
+        if ((row[bit / 8] >> (bit % 8)) & 1) val |= (1 << i);
+    }
+    return val;
+}
+
+void oracle_unpack(const uint8_t *packed, int32_t rows, int32_t cols, int32_t k, int32_t *idx)
+{
+    int b = oracle_index_bits(k);
+    int64_t stride = oracle_row_bytes(cols, k);
+    for (int32_t r = 0; r < rows; r++)
+        for (int32_t c = 0; c < cols; c++)
+            idx[(int64_t)r * cols + c] = read_index(packed + (int64_t)r * stride, c, b);
+}
+
+/* ------------------------------------------------------------------ */
+/* Layer description                                                   */
+/* ------------------------------------------------------------------ */
+
+typedef struct oracle_layer {
+    int32_t M, N;            /* W is [M][N]: M output features, N input features   */
+    int32_t v, k1, k2;       /* main vector length, main / residual table sizes     */
+    int32_t n_out, v0, k0;   /* leading outlier columns, their vector length/table  */
+    int32_t has_scale;       /* 1: W = t*scale[n] + bias[n]                          */
+    int32_t scale_axis;      /* 0: per input column n; 1: per output row m          */
+    const uint8_t *idx1;     /* packed [ceil(M/v)][N-n_out], b(k1) bits             */
+    const uint16_t *c1;      /* [k1][v] fp16 bits                                   */
+    const uint8_t *idx2;     /* packed, same shape, b(k2) bits (k2 > 0)             */
+    const uint16_t *c2;      /* [k2][v]                                             */
+    const uint8_t *idx0;     /* packed [ceil(M/v0)][n_out], b(k0) bits (n_out > 0)  */
+    const uint16_t *c0;      /* [k0][v0]                                            */
+    const uint16_t *scale;   /* fp16 bits, [N] (axis 0) or [M] (axis 1)             */
+    const uint16_t *bias;
+} oracle_layer;
+
+/* One restored weight, FP16 bits.  Returns 0xFFFF-coded error through *err when an
+ * index is out of range (corrupt stream): the tests treat that as a failure. */
+static uint16_t restore_weight(const oracle_layer *L, int32_t m, int32_t n, int *err)
+{
+    float t;
+    if (n < L->n_out) {
+        /* outlier column: own table, own vector length, no residual stage */
+        int64_t stride0 = oracle_row_bytes(L->n_out, L->k0);
+        int32_t r0 = m / L->v0, j0 = m % L->v0;
+        int32_t i0 = read_index(L->idx0 + (int64_t)r0 * stride0, n, oracle_index_bits(L->k0));
+        if (i0 >= L->k0) { *err = 1; return 0; }
+        t = oracle_half_to_float(L->c0[(int64_t)i0 * L->v0 + j0]);
+    } else {
+        int32_t c = n - L->n_out, Nc = L->N - L->n_out;
+        int32_t r = m / L->v, j = m % L->v;
+        int64_t stride1 = oracle_row_bytes(Nc, L->k1);
+        int32_t i1 = read_index(L->idx1 + (int64_t)r * stride1, c, oracle_index_bits(L->k1));
+        if (i1 >= L->k1) { *err = 1; return 0; }
+        t = oracle_half_to_float(L->c1[(int64_t)i1 * L->v + j]);
+        if (L->k2 > 0) {
+            int64_t stride2 = oracle_row_bytes(Nc, L->k2);
+            int32_t i2 = read_index(L->idx2 + (int64_t)r * stride2, c, oracle_index_bits(L->k2));
+            if (i2 >= L->k2) { *err = 1; return 0; }
+            float t2 = oracle_half_to_float(L->c2[(int64_t)i2 * L->v + j]);
+            t = t + t2;                     /* rounded FP32 add */
+        }
+    }
+    if (L->has_scale) {
+        int32_t a = L->scale_axis ? m : n;
+        float s = oracle_half_to_float(L->scale[a]);
+        float bb = oracle_half_to_float(L->bias[a]);
+        float p = t * s;                    /* rounded FP32 multiply */
+        t = p + bb;                         /* rounded FP32 add      */
+    }
+    return oracle_float_to_half(t);
+}
+
+/* Restore the whole matrix: W16 [M][N] FP16 bits.  Returns 0 or -1 (index out of range). */
+int oracle_dequant(const oracle_layer *L, uint16_t *W16)
+{
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(|:bad)
+    for (int32_t m = 0; m < L->M; m++) {
+        int err = 0;
+        for (int32_t n = 0; n < L->N; n++)
+            W16[(int64_t)m * L->N + n] = restore_weight(L, m, n, &err);
+        bad |= err;
+    }
+    return bad ? -1 : 0;
+}
+
+/* Restore selected rows only: rows[i] in [0,M) -> Wrows [n_rows][N]. */
+int oracle_dequant_rows(const oracle_layer *L, const int32_t *rows, int32_t n_rows, uint16_t *Wrows)
+{
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(|:bad)
+    for (int32_t i = 0; i < n_rows; i++) {
+        int err = 0;
+        for (int32_t n = 0; n < L->N; n++)
+            Wrows[(int64_t)i * L->N + n] = restore_weight(L, rows[i], n, &err);
+        bad |= err;
+    }
+    return bad ? -1 : 0;
+}
+
+static double load_x(const uint16_t *x, int64_t i, int x_is_bf16)
+{
+    return (double)(x_is_bf16 ? oracle_bf16_to_float(x[i]) : oracle_half_to_float(x[i]));
+}
+
+/* y[t][i] = sum_n x[t][n] * W16[rows[i]][n] in FP64, n ascending.
+ * rows == NULL means all M rows (n_rows must then be M).  y is [B][n_rows]. */
+int oracle_linear_rows(const oracle_layer *L, const uint16_t *x, int32_t B, int x_is_bf16,
+                       const int32_t *rows, int32_t n_rows, double *y)
+{
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 4) reduction(|:bad)
+    for (int32_t i = 0; i < n_rows; i++) {
+        int err = 0;
+        int32_t m = rows ? rows[i] : i;
+        uint16_t *w = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)L->N);
+        for (int32_t n = 0; n < L->N; n++) w[n] = restore_weight(L, m, n, &err);
+        for (int32_t t = 0; t < B; t++) {
+            double acc = 0.0;
+            for (int32_t n = 0; n < L->N; n++)
+                acc += load_x(x, (int64_t)t * L->N + n, x_is_bf16) * (double)oracle_half_to_float(w[n]);
+            y[(int64_t)t * n_rows + i] = acc;
+        }
+        free(w);
+        bad |= err;
+    }
+    return bad ? -1 : 0;
+}
+
+int oracle_linear(const oracle_layer *L, const uint16_t *x, int32_t B, int x_is_bf16, double *y)
+{
+    return oracle_linear_rows(L, x, B, x_is_bf16, NULL, L->M, y);
+}
+
+/* ------------------------------------------------------------------ */
+/* Size accounting                                                     */
+/* ------------------------------------------------------------------ */
+
+/* Codebook bits (App. C.2): (v0*k0 + v1*(k1+k2)) * 16. */
+double oracle_codebook_bits(int32_t v, int32_t k1, int32_t k2, int32_t n_out, int32_t v0, int32_t k0)
+{
+    double e = (double)v * ((double)k1 + (double)(k2 > 0 ? k2 : 0));
+    if (n_out > 0) e += (double)v0 * (double)k0;
+    return e * 16.0;
+}
+
+/* Index bits actually stored for an M x N layer, without row padding:
+ * ceil(M/v) * (N - n_out) * (b1 + b2) + ceil(M/v0) * n_out * b0  (App. C.2 with the
+ * outlier term read as log2(k0)/v0 per weight). */
+double oracle_index_bits_total(int32_t M, int32_t N, int32_t v, int32_t k1, int32_t k2,
+                               int32_t n_out, int32_t v0, int32_t k0)
+{
+    double R = (double)((M + v - 1) / v);
+    double bits = R * (double)(N - n_out) *
+                  (double)(oracle_index_bits(k1) + (k2 > 0 ? oracle_index_bits(k2) : 0));
+    if (n_out > 0) bits += (double)((M + v0 - 1) / v0) * (double)n_out * (double)oracle_index_bits(k0);
+    return bits;
+}
+
+/* Equivalent bit width (Sec. 2.2): 16 / (16*M*N / (codebook bits + index bits)). */
+double oracle_equivalent_bits(int32_t M, int32_t N, int32_t v, int32_t k1, int32_t k2,
+                              int32_t n_out, int32_t v0, int32_t k0)
+{
+    double total = oracle_codebook_bits(v, k1, k2, n_out, v0, k0) +
+                   oracle_index_bits_total(M, N, v, k1, k2, n_out, v0, k0);
+    return total / ((double)M * (double)N);
+}
+
+double oracle_compression_ratio(int32_t M, int32_t N, int32_t v, int32_t k1, int32_t k2,
+                                int32_t n_out, int32_t v0, int32_t k0)
+{
+    return 16.0 / oracle_equivalent_bits(M, N, v, k1, k2, n_out, v0, k0);
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}

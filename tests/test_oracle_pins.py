@@ -1,0 +1,342 @@
+"""Pins for the CPU oracle: each test checks it against something that is not itself —
+values the paper prints, closed forms, library routines, a separately written numpy
+statement, or brute force on tiny layers.  No GPU needed."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import mini, oracle
+from paper_2409_17066_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append(line.split())
+    return out
+
+
+# ---------------------------------------------------------------- converters
+
+def test_half_to_float_exhaustive_vs_numpy():
+    bits = np.arange(65536, dtype=np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.half_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))
+
+
+def test_float_to_half_vs_numpy():
+    rng = np.random.default_rng(1)
+    # every half value, the midpoints between neighbours, and values a hair off the midpoints
+    h = np.arange(0x7C00, dtype=np.uint16).view(np.float16).astype(np.float64)
+    mids = (h[:-1] + h[1:]) / 2
+    cand = np.concatenate([h, mids, np.nextafter(mids.astype(np.float32), np.float32(np.inf)),
+                           np.nextafter(mids.astype(np.float32), np.float32(-np.inf)),
+                           [65504.0, 65519.99, 65520.0, 65536.0, 1e9, 2.0 ** -24, 2.0 ** -25,
+                            np.nextafter(np.float32(2.0 ** -25), np.float32(1)), 2.0 ** -26, 1e-30, 0.0],
+                           rng.normal(0, 1, 20000), rng.normal(0, 1e-5, 20000),
+                           rng.uniform(-70000, 70000, 20000)]).astype(np.float32)
+    cand = np.concatenate([cand, -cand])
+    with np.errstate(over="ignore"):
+        ref = cand.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.float_to_half(float(c)) for c in cand], dtype=np.uint16)
+    assert np.array_equal(got, ref)
+
+
+def test_bf16_converters():
+    rng = np.random.default_rng(2)
+    f = np.concatenate([rng.normal(0, 1, 5000), rng.normal(0, 1e-20, 100), [0.0, 1.0, 3.0e38]]).astype(np.float32)
+    # ties: exactly halfway between two bf16 values
+    ties = ((rng.integers(0, 2 ** 15, 2000).astype(np.uint32) << 16) | 0x8000).view(np.float32)
+    ties = ties[np.isfinite(ties)]
+    f = np.concatenate([f, ties])
+    ref = synth.to_bf16_bits(f)
+    got = np.array([oracle.float_to_bf16(float(v)) for v in f], dtype=np.uint16)
+    assert np.array_equal(got, ref)
+    # a bf16 is the top half of the float: round trip is exact, and widening matches the bit shift
+    back = np.array([oracle.bf16_to_float(int(b)) for b in got], dtype=np.float32)
+    assert np.array_equal(back.view(np.uint32), got.astype(np.uint32) << 16)
+    # tie goes to the even neighbour: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert oracle.float_to_bf16(1.0 + 2.0 ** -8) == 0x3F80
+    assert oracle.float_to_bf16(1.0 + 3 * 2.0 ** -8) == 0x3F82
+
+
+# ---------------------------------------------------------------- packed stream
+
+def test_pack_hand_computed_12bit():
+    # 2 x 5 matrix at b = 12 (k = 4096).  Row stream is little-endian: index c sits in bits [12c, 12c+12).
+    idx = np.array([[0xABC, 0x123, 0xFFF, 0x000, 0x801],
+                    [0x001, 0x800, 0x00F, 0xF00, 0x0F0]], dtype=np.int32)
+    # row 0 bits: 0xABC | 0x123<<12 | 0xFFF<<24 | 0<<36 | 0x801<<48  -> bytes little-endian
+    v0 = 0xABC | (0x123 << 12) | (0xFFF << 24) | (0x000 << 36) | (0x801 << 48)
+    v1 = 0x001 | (0x800 << 12) | (0x00F << 24) | (0xF00 << 36) | (0x0F0 << 48)
+    exp = np.zeros((2, 16), dtype=np.uint8)
+    exp[0, :8] = np.frombuffer(v0.to_bytes(8, "little"), dtype=np.uint8)
+    exp[1, :8] = np.frombuffer(v1.to_bytes(8, "little"), dtype=np.uint8)
+    # spelled out for row 0: BC 3A 12 FF 0F 00 01 08
+    assert list(exp[0, :8]) == [0xBC, 0x3A, 0x12, 0xFF, 0x0F, 0x00, 0x01, 0x08]
+    got = oracle.pack(idx, 4096)
+    assert got.shape == (2, 16)
+    assert np.array_equal(got, exp)
+    assert np.array_equal(mini.pack(idx, 4096), exp)
+
+
+def test_pack_plain_widths_are_plain_arrays():
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, 256, size=(3, 32), dtype=np.int32)
+    assert np.array_equal(oracle.pack(idx, 256), idx.astype(np.uint8))
+    idx = rng.integers(0, 65536, size=(3, 16), dtype=np.int32)
+    assert np.array_equal(oracle.pack(idx, 65536).view("<u2"), idx.astype(np.uint16))
+
+
+@pytest.mark.parametrize("b", list(range(1, 17)))
+@pytest.mark.parametrize("cols", [1, 7, 41, 257, 4055])
+def test_pack_unpack_round_trip(b, cols):
+    k = 1 << b if b > 1 else 2
+    if b == 1:
+        ks = [1, 2]
+    else:
+        ks = [k, (1 << (b - 1)) + 1]          # power of two and the smallest k that needs b bits
+    rng = np.random.default_rng(100 * b + cols)
+    for kk in ks:
+        assert oracle.index_bits(kk) == b == mini.index_bits(kk)
+        for idx in (rng.integers(0, kk, size=(3, cols), dtype=np.int32),
+                    np.zeros((2, cols), np.int32), np.full((2, cols), kk - 1, np.int32)):
+            p = oracle.pack(idx, kk)
+            assert p.shape[1] % 16 == 0 and p.shape[1] == mini.row_bytes(cols, kk)
+            assert p.shape[1] - (cols * b + 7) // 8 < 16
+            assert np.array_equal(oracle.unpack(p, idx.shape[0], cols, kk), idx)
+            assert np.array_equal(p, mini.pack(idx, kk))
+            assert np.array_equal(mini.unpack(p, idx.shape[0], cols, kk), idx)
+
+
+def test_pack_rejects_out_of_range():
+    with pytest.raises(ValueError):
+        oracle.pack(np.array([[0, 5]], np.int32), 5)
+    with pytest.raises(ValueError):
+        oracle.pack(np.array([[-1, 0]], np.int32), 5)
+
+
+# ---------------------------------------------------------------- size accounting (paper's numbers)
+
+def test_worked_example_ratio_and_bits():
+    (M, N, v, k, ratio, bits), = _rows("size_worked_example.txt")
+    M, N, v, k = int(M), int(N), int(v), int(k)
+    assert round(oracle.compression_ratio(M, N, v, k), 2) == float(ratio)
+    assert round(oracle.equivalent_bits(M, N, v, k), 3) == float(bits)
+    # and the packed stream really has that many index bits: log2(k)/v per weight
+    assert oracle.packed_bytes(M // v, N, k) * 8 == M * N * np.log2(k) / v
+
+
+def _block_bits(v, k1, k2, pct, v0, k0, H=5120, F=13824):
+    layers = [(H, H)] * 4 + [(F, H), (F, H), (H, F)]
+    bits = params = 0.0
+    for (M, N) in layers:
+        n_out = synth.outlier_columns(N, pct)
+        bits += oracle.codebook_bits(v, k1, k2, n_out, v0, k0) + \
+            oracle.index_bits_total(M, N, v, k1, k2, n_out, v0, k0)
+        params += M * N
+    return bits / params
+
+
+def test_ablation_table_bit_column():
+    for row, bit, pct, v0, k0, v1, k1, k2, pin in _rows("ablation_bits.txt"):
+        got = _block_bits(int(v1), int(k1), max(int(k2), 0), float(pct), int(v0), int(k0))
+        if pin == "1":
+            assert round(got, 2) == float(bit), (row, got, bit)
+        else:
+            assert 0 <= float(bit) - got <= 0.0105, (row, got, bit)
+
+
+def test_codebook_overhead_and_outlier_bits():
+    g = dict((k, float(v)) for k, v in _rows("codebook_overhead.txt"))
+    params = 4 * 5120 * 5120 + 3 * 5120 * 13824
+    over = 7 * oracle.codebook_bits(8, 65536) / params
+    assert round(over, 2) in (g["codebook_overhead_v8_k65536"], round(g["codebook_overhead_v8_k65536"] - 0.01, 2))
+    assert oracle.index_bits(4096) / 4 == g["outlier_index_bits_v4_k4096"]
+    assert oracle.index_bits(4096) / 6 == g["main_index_bits_v6_k4096"]
+
+
+def test_measured_packed_size_matches_index_bit_formula():
+    # App. C.2: average index bits = log2(k1)/v1 + log2(k2)/v1; outlier part log2(k0)/v0.
+    for cfg in (1, 2, 3, 4):
+        for s in synth.CONFIGS[cfg]["layers"]:
+            stored = oracle.packed_bytes(s.R, s.Nc, s.k1) * 8
+            if s.k2:
+                stored += oracle.packed_bytes(s.R, s.Nc, s.k2) * 8
+            if s.n_out:
+                stored += oracle.packed_bytes(s.R0, s.n_out, s.k0) * 8
+            main = (np.log2(s.k1) + (np.log2(s.k2) if s.k2 else 0)) / s.v
+            formula = main * s.M * s.Nc
+            if s.n_out:
+                formula += np.log2(s.k0) / s.v0 * s.M * s.n_out
+            # padding only: ceil(M/v) rows and < 16 bytes per row and stream
+            pad_rows = (s.R * s.v - s.M) * s.Nc * main
+            pad_bytes = 16 * 8 * (s.R * (2 if s.k2 else 1) + s.R0)
+            assert formula <= stored <= formula + pad_rows + pad_bytes
+            assert stored / (s.M * s.N) - formula / (s.M * s.N) < 0.01
+
+
+# ---------------------------------------------------------------- lookup: closed forms and special cases
+
+def _layer(d, **kw):
+    return oracle.Layer.from_synth(d, **kw)
+
+
+def test_single_codebook_no_scale_is_pure_gather():
+    spec = synth.LayerSpec("g", 40, 33, v=8, k1=256, has_scale=False)
+    d = synth.make_layer(spec, 90, 0, 1)
+    W = _layer(d).dequant()
+    for m, n in itertools.product(range(spec.M), range(spec.N)):
+        assert W[m, n].view(np.uint16) == d["c1"][d["idx1"][m // 8, n], m % 8].view(np.uint16)
+
+
+def test_k1_closed_form():
+    # one centroid: W[m][n] = s[n]*C[0][m%v] + b[n];  y[t][m] = C[0][m%v]*sum(x s) + sum(x b) up to the FP16 rounding of W
+    spec = synth.LayerSpec("k1", 21, 64, v=4, k1=1)
+    d = synth.make_layer(spec, 91, 0, 3)
+    L = _layer(d)
+    W = L.dequant()
+    c = d["c1"][0].astype(np.float32)
+    exp = ((c[np.arange(21) % 4][:, None] * d["scale"].astype(np.float32)[None, :]).astype(np.float32)
+           + d["bias"].astype(np.float32)[None, :]).astype(np.float16)
+    assert np.array_equal(W.view(np.uint16), exp.view(np.uint16))
+    assert oracle.packed_bytes(spec.R, spec.N, 1) == spec.R * 16   # one (wasted) bit per index
+    y = L.linear(d["x"])
+    x = d["x"].astype(np.float64)
+    closed = (x @ d["scale"].astype(np.float64))[:, None] * c.astype(np.float64)[np.arange(21) % 4][None, :] \
+        + (x @ d["bias"].astype(np.float64))[:, None]
+    assert np.max(np.abs(y - closed)) <= 2.0 ** -11 * np.sum(np.abs(x), axis=1).max() * 0.05
+
+
+def test_identity_codebook_is_a_histogram():
+    # C = I_8: restored W[r*8+j][n] = 1 if I[r][n] == j else 0, so y is a sum of x over matching columns
+    v = 8
+    spec = synth.LayerSpec("id", 48, 100, v=v, k1=8, has_scale=False)
+    d = synth.make_layer(spec, 92, 0, 2)
+    d["c1"] = np.eye(8, dtype=np.float16)
+    y = _layer(d).linear(d["x"])
+    x = d["x"].astype(np.float64)
+    exp = np.zeros((2, 48))
+    for r in range(6):
+        for n in range(100):
+            exp[:, r * 8 + d["idx1"][r, n]] += x[:, n]
+    assert np.allclose(y, exp, rtol=0, atol=1e-12)
+
+
+def test_v1_integer_matmul_is_exact():
+    spec = synth.LayerSpec("v1", 17, 23, v=1, k1=256, has_scale=False)
+    d = synth.make_layer(spec, 93, 0, 2)
+    d["c1"] = (np.arange(256, dtype=np.float32) / 256).astype(np.float16).reshape(256, 1)
+    d["x"] = np.random.default_rng(5).integers(-8, 9, size=(2, 23)).astype(np.float16)
+    L = _layer(d)
+    assert np.array_equal(L.dequant().astype(np.float64) * 256, d["idx1"].astype(np.float64))
+    y = L.linear(d["x"])
+    exp = d["x"].astype(np.int64) @ d["idx1"].astype(np.int64).T
+    assert np.array_equal(y * 256, exp.astype(np.float64))
+
+
+def test_residual_special_cases():
+    spec = synth.LayerSpec("r", 32, 40, v=8, k1=256, k2=256)
+    d = synth.make_layer(spec, 94, 0, 1)
+    single = dict(d, spec=synth.LayerSpec("r1", 32, 40, v=8, k1=256), c2=None, idx2=None)
+    # C2 = 0 : same as one codebook
+    z = dict(d, c2=np.zeros_like(d["c2"]))
+    assert np.array_equal(_layer(z).dequant().view(np.uint16), _layer(single).dequant().view(np.uint16))
+    # C2 = -C1, I2 = I1 : the lookup sum cancels, W = bias exactly
+    neg = dict(d, c2=(-d["c1"]), idx2=d["idx1"].copy())
+    W = _layer(neg).dequant()
+    assert np.array_equal(W.view(np.uint16), np.broadcast_to(d["bias"][None, :], W.shape).view(np.uint16))
+    # a residual stage really adds: differs from the single-codebook result somewhere
+    assert not np.array_equal(_layer(d).dequant().view(np.uint16), _layer(single).dequant().view(np.uint16))
+
+
+def test_outlier_special_cases():
+    base = synth.LayerSpec("o", 24, 30, v=8, k1=256, n_out=30, v0=4, k0=16)
+    d = synth.make_layer(base, 95, 0, 1)
+    # all columns outliers: equals a plain layer quantized with (v0, k0)
+    plain = dict(d, spec=synth.LayerSpec("p", 24, 30, v=4, k1=16), c1=d["c0"], idx1=d["idx0"],
+                 c0=None, idx0=None)
+    d_all = dict(d, idx1=np.zeros((3, 0), np.int32))
+    assert np.array_equal(_layer(d_all).dequant().view(np.uint16), _layer(plain).dequant().view(np.uint16))
+    # mixed: outlier columns come from C0 only (no residual added there), the others from C1 + C2
+    spec = synth.LayerSpec("m", 24, 30, v=8, k1=256, k2=16, n_out=5, v0=4, k0=16, has_scale=False)
+    d = synth.make_layer(spec, 96, 0, 1)
+    W = _layer(d).dequant()
+    for m in range(24):
+        for n in range(5):
+            assert W[m, n].view(np.uint16) == d["c0"][d["idx0"][m // 4, n], m % 4].view(np.uint16)
+        for n in range(5, 30):
+            t = np.float32(d["c1"][d["idx1"][m // 8, n - 5], m % 8]) + np.float32(d["c2"][d["idx2"][m // 8, n - 5], m % 8])
+            assert W[m, n].view(np.uint16) == np.float16(t).view(np.uint16)
+
+
+def test_scale_axis_flag():
+    spec = synth.LayerSpec("a", 16, 16, v=8, k1=256)
+    d = synth.make_layer(spec, 97, 0, 1)
+    W0 = _layer(d, scale_axis=0).dequant()
+    W1 = _layer(d, scale_axis=1).dequant()
+    assert np.array_equal(W0.view(np.uint16), mini.dequant_from_synth(d, 0).view(np.uint16))
+    assert np.array_equal(W1.view(np.uint16), mini.dequant_from_synth(d, 1).view(np.uint16))
+    assert not np.array_equal(W0.view(np.uint16), W1.view(np.uint16))
+
+
+# ---------------------------------------------------------------- brute force and library routines
+
+def test_all_index_combinations_tiny():
+    # every index matrix of a 4 x 2 layer with v = 2, k = 3 (3^4 = 81 cases), against the numpy statement
+    c1 = np.array([[0.5, -1.25], [2.0, 0.125], [-3.0, 7.0]], dtype=np.float16)
+    scale = np.array([1.5, 0.75], np.float16)
+    bias = np.array([0.01, -0.02], np.float16)
+    x = np.array([[1.0, -2.0]], np.float16)
+    for combo in itertools.product(range(3), repeat=4):
+        idx = np.array(combo, np.int32).reshape(2, 2)
+        L = oracle.Layer(4, 2, 2, 3, c1, oracle.pack(idx, 3), scale=scale, bias=bias)
+        W = L.dequant()
+        ref = mini.dequant(4, 2, 2, c1, idx, scale=scale, bias=bias)
+        assert np.array_equal(W.view(np.uint16), ref.view(np.uint16))
+        assert np.allclose(L.linear(x), mini.linear(ref, x.astype(np.float64)), rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("spec", synth.small_specs(), ids=lambda s: s.name)
+def test_small_layers_vs_numpy_statement(spec):
+    for seed_layer in range(3):
+        d = synth.make_layer(spec, 80, seed_layer, 3)
+        L = _layer(d)
+        W = L.dequant()
+        ref = mini.dequant_from_synth(d)
+        assert np.array_equal(W.view(np.uint16), ref.view(np.uint16))
+        rows = np.array([0, spec.M - 1, spec.M // 2], np.int32)
+        assert np.array_equal(L.dequant_rows(rows).view(np.uint16), ref[rows].view(np.uint16))
+        # matmul step reduces to a library routine on the FP16 weights
+        y = L.linear(d["x"])
+        yr = mini.linear(ref, d["x"].astype(np.float64))
+        assert np.max(np.abs(y - yr)) <= 1e-12 * max(1.0, np.max(np.abs(yr)))
+        assert np.array_equal(L.linear(d["x"], rows), y[:, rows])
+
+
+def test_bf16_activations():
+    spec = synth.LayerSpec("b", 16, 40, v=8, k1=256, x_dtype="bf16")
+    d = synth.make_layer(spec, 81, 0, 2)
+    L = _layer(d)
+    y = L.linear(d["x"])
+    xr = synth.bf16_bits_to_f32(d["x"]).astype(np.float64)
+    assert np.allclose(y, mini.linear(L.dequant(), xr), rtol=0, atol=1e-12)
+
+
+def test_config0_and_ragged_v6_bits():
+    # config 0 itself: 1.000 index bit per weight, 1.25 with its codebook
+    s = synth.CONFIGS[0]["layers"][0]
+    assert oracle.packed_bytes(s.R, s.N, s.k1) * 8 / (s.M * s.N) == 1.0
+    assert oracle.equivalent_bits(s.M, s.N, s.v, s.k1) == 1.25
+    # the outlier column counts used for the 1 % setting
+    assert synth.outlier_columns(4096, 1.0) == 41 and synth.outlier_columns(11008, 1.0) == 110
