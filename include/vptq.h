@@ -1,0 +1,178 @@
+/*
+ * vptq.h — C ABI of libvptq: the inference hot path of VPTQ (vector post-training
+ * quantization) on NVIDIA B200 (sm_100a).
+ *
+ * The quantized weight format is the paper's (Sec. 2.2, Sec. 3.1, Sec. 3.2.2-3, App. C.1):
+ *   - the weight W_hat is [M][N], M output features, N input features;
+ *   - it is cut into length-v vectors that run down a column: vector row r of column n
+ *     covers output rows r*v .. r*v+v-1 (Sec. 3.1: a quantized column is a stack of
+ *     centroids; Algorithm 1 steps m = 0, V, 2V, ...);
+ *   - every vector is stored as an index into a codebook of k1 centroids of length v
+ *     (Sec. 2.2); with residual VQ a second index into a codebook of k2 centroids is
+ *     stored and decoding sums the two centroids (Sec. 3.2.2);
+ *   - n_outlier leading input columns are quantized separately with their own vector
+ *     length v0 and codebook of k0 centroids, and have no residual stage (Sec. 3.2.3,
+ *     App. C.1, Algorithm 2).
+ * Not stated by the paper and fixed by this library: the per-channel scale and bias
+ * (W_hat = t*scale + bias, FP32, three separately rounded operations add, multiply, add),
+ * the bit-packed index stream below, and "outlier columns come first".
+ *
+ * Packed index stream.  An index matrix I[rows][cols] with values in [0,k) uses
+ * b = max(1, ceil(log2 k)) bits per index.  Each row is its own little-endian bit
+ * stream: index c occupies stream bits [c*b, c*b+b); stream bit i is bit (i%8) of
+ * byte (i/8).  A row occupies ceil(cols*b/8) bytes rounded up to a multiple of 16; pad
+ * bits are zero.  b = 8 is a plain uint8 array, b = 16 a plain little-endian uint16 array.
+ *
+ * Conventions, unless an entry point says otherwise:
+ *   - every data pointer is a DEVICE pointer owned by the caller and must be 16-byte
+ *     aligned; the library allocates nothing and keeps no state between calls;
+ *   - `stream` is a cudaStream_t passed as void*; calls are asynchronous on it;
+ *   - the return value is 0 (VPTQ_OK) or a negative VPTQ_E_* code; nothing throws,
+ *     aborts or traps.  vptq_status_string() names a code; vptq_last_cuda_error()
+ *     gives the CUDA runtime's text for the last VPTQ_E_CUDA on this thread.
+ */
+#ifndef VPTQ_H_
+#define VPTQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VPTQ_OK              0
+#define VPTQ_E_NULL         -1   /* a required pointer is null                              */
+#define VPTQ_E_SHAPE        -2   /* M,N,v,k <= 0, k > 65536, v > 32, n_outlier > N, B <= 0  */
+#define VPTQ_E_ALIGN        -3   /* a data pointer is not 16-byte aligned                   */
+#define VPTQ_E_UNSUPPORTED  -4   /* dtype / flag combination without a kernel               */
+#define VPTQ_E_WORKSPACE    -5   /* workspace missing or smaller than the query says        */
+#define VPTQ_E_INDEX_RANGE  -6   /* vptq_pack found an index outside [0,k)                  */
+#define VPTQ_E_CUDA         -7   /* a CUDA runtime call failed                              */
+#define VPTQ_E_TIMEOUT      -8   /* a bounded device-side wait gave up (status word)        */
+
+#define VPTQ_DTYPE_FP16 0
+#define VPTQ_DTYPE_BF16 1
+#define VPTQ_DTYPE_FP32 2
+
+#define VPTQ_FLAG_SCALE_BIAS   1  /* scale and bias are present                                     */
+#define VPTQ_FLAG_SCALE_ROWS   2  /* scale/bias are per OUTPUT row ([M]) instead of per input column */
+#define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
+
+/* Geometry of one quantized linear layer (App. C.1 names: v1,k1,k2 / N%,v0,k0). */
+typedef struct vptq_layer_desc {
+    int32_t M, N;        /* out_features, in_features: W_hat is [M][N]                       */
+    int32_t v;           /* main vector length (1..32)                                       */
+    int32_t k1;          /* main codebook size (1..65536)                                    */
+    int32_t k2;          /* residual codebook size, 0 = no residual stage                    */
+    int32_t n_outlier;   /* columns [0,n_outlier) use the outlier codebook; 0 = none         */
+    int32_t v0, k0;      /* outlier vector length / codebook size (ignored if n_outlier = 0) */
+    int32_t x_dtype;     /* VPTQ_DTYPE_FP16 or _BF16                                         */
+    int32_t out_dtype;   /* VPTQ_DTYPE_FP16, _BF16 or _FP32                                  */
+    int32_t flags;       /* VPTQ_FLAG_*                                                      */
+} vptq_layer_desc;
+
+/* The nine format pointers of a layer, in the order of the paper's format statement.
+ *   packed_idx       packed [ceil(M/v)][N-n_outlier], b(k1) bits       (required unless n_outlier == N)
+ *   codebook         fp16 [k1][v]                                       (required unless n_outlier == N)
+ *   res_idx          packed, same shape, b(k2) bits                     (required iff k2 > 0)
+ *   res_codebook     fp16 [k2][v]                                       (required iff k2 > 0)
+ *   outlier_idx      packed [ceil(M/v0)][n_outlier], b(k0) bits         (required iff n_outlier > 0)
+ *   outlier_codebook fp16 [k0][v0]                                      (required iff n_outlier > 0)
+ *   scale, bias      fp16 [N] (or [M] with VPTQ_FLAG_SCALE_ROWS)        (required iff VPTQ_FLAG_SCALE_BIAS)
+ * A pointer that is not required may be null and is never read. */
+typedef struct vptq_layer_ptrs {
+    const uint8_t *packed_idx;
+    const void    *codebook;
+    const uint8_t *res_idx;
+    const void    *res_codebook;
+    const uint8_t *outlier_idx;
+    const void    *outlier_codebook;
+    const void    *scale;
+    const void    *bias;
+} vptq_layer_ptrs;
+
+/* ---- format arithmetic (host only, no CUDA call) ---------------------------------- */
+
+/* b = max(1, ceil(log2 k)): bits per index; the index-bit terms log2(k)/v of App. C.2
+ * are b/v.  Returns VPTQ_E_SHAPE for k outside [1,65536]. */
+int vptq_index_bits(int32_t k);
+/* Bytes of one packed row / of the whole packed matrix (16-byte row padding included).
+ * Negative (VPTQ_E_SHAPE) on bad arguments. */
+int64_t vptq_packed_row_bytes(int32_t n_cols, int32_t k);
+int64_t vptq_packed_bytes(int32_t n_rows, int32_t n_cols, int32_t k);
+/* Bytes the format of a layer occupies, each stream/table counted once: packed index
+ * streams + codebooks (App. C.2 "Codebook bits"/8) + scale and bias.  This is the
+ * numerator of "effective weight GB/s". */
+int64_t vptq_layer_weight_bytes(const vptq_layer_desc *desc);
+
+/* ---- pack / unpack (boundary steps, not on the timed path) ------------------------ */
+
+/* Pack idx[n_rows][n_cols] (int32, device) into the stream format (device, size
+ * vptq_packed_bytes).  Every byte of `packed`, padding included, is written.
+ * `bad_count` (device int32, may be null) receives the number of indices outside
+ * [0,k); when it is non-null the call synchronises the stream, reads it back and
+ * returns VPTQ_E_INDEX_RANGE if it is non-zero (such indices are stored as 0). */
+int vptq_pack(const int32_t *idx, int32_t n_rows, int32_t n_cols, int32_t k,
+              uint8_t *packed, int32_t *bad_count, void *stream);
+/* Inverse of vptq_pack: idx[n_rows][n_cols] (int32, device) from the packed stream,
+ * read with 128-bit loads.  Bit-exact inverse for every valid stream. */
+int vptq_unpack(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k,
+                int32_t *idx, void *stream);
+
+/* ---- dequantisation (Sec. 2.2 "dequantizes the weight matrix from the lookup table by
+ *      index and centroid"; Sec. 3.2.2 decode; Sec. 3.2.3; App. D.2 "restore to FP16") -- */
+
+/* W_out[M][N] fp16 (device, row-major) = the restored weight:
+ *   n <  n_outlier: t = C0[I0[m/v0][n]][m%v0]
+ *   n >= n_outlier: t = C1[I1[m/v][c]][m%v] (+ C2[I2[m/v][c]][m%v]), c = n - n_outlier
+ *   W = fp16_rne( fp32(fp32(t*scale) + bias) ) when VPTQ_FLAG_SCALE_BIAS, else fp16(t).
+ * Bit-exact by definition (no fused multiply-add, denormals kept).  Indices >= k in a
+ * corrupt stream are clamped to k-1, never read out of range. */
+int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p,
+                 void *W_out, void *stream);
+
+/* ---- the fused linear layer (App. D.2: dequantisation fused with the product so the
+ *      FP16 weight is never written to or read from global memory) ------------------ */
+
+/* Scratch bytes vptq_linear needs for this layer at batch B (0 is possible).  The
+ * caller allocates at least this much, 256-byte aligned; contents on entry are
+ * irrelevant and undefined on exit.  Negative VPTQ_E_* on a bad descriptor. */
+int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B);
+
+/* out[B][M] = x[B][N] * W_hat^T, W_hat as defined at vptq_dequant (without the final
+ * FP16 rounding of W_hat; FP32 accumulation; the result differs from the FP64 product
+ * over the FP16-rounded weights by at most ~1e-3 of max|out|).
+ *   x    [B][N] row-major, desc->x_dtype;  out [B][M] row-major, desc->out_dtype.
+ * B <= 16 runs the split-K decode kernels; larger B runs the tensor-core path
+ * (tcgen05) when the layer qualifies (v = 8, k1 > 8192, x bf16/fp16), otherwise the
+ * decode kernels over groups of 16 tokens.  Calls on one stream are ordered; calls
+ * on different streams must not share a workspace. */
+int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
+                const vptq_layer_ptrs *p, void *out,
+                void *workspace, size_t workspace_bytes, void *stream);
+
+/* Same product with HOST activations and HOST result: copies x_host -> x_dev, runs
+ * vptq_linear, copies out_dev -> out_host, all asynchronously on `stream` (the caller
+ * synchronises the stream before reading out_host).  x_host/out_host should be pinned
+ * host memory; x_dev ([B][N]) and out_dev ([B][M]) are caller-owned device staging
+ * buffers.  The weights (p) stay resident on the device. */
+int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
+                        const vptq_layer_ptrs *p, void *out_host,
+                        void *x_dev, void *out_dev,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- diagnostics ------------------------------------------------------------------ */
+
+const char *vptq_status_string(int code);
+const char *vptq_last_cuda_error(void);
+/* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_mma",
+ * "decode_l2_fma", "gemm_tcgen05".  For tests and benchmark logs. */
+const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B);
+/* Number of kernel launches (memsets included) one vptq_linear call issues. */
+int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VPTQ_H_ */

@@ -1,0 +1,255 @@
+"""Thin Python binding of libvptq's C ABI (include/vptq.h).
+
+Argument marshalling only: every function here passes device pointers of torch tensors
+(and torch's current CUDA stream) straight to the entry point of the same name.  torch is
+used for device memory and streams, nothing else; there is no CPU fallback — if the
+shared library is missing, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvptq.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2409_17066_b200.build` "
+        "(there is no CPU fallback)")
+
+lib = C.CDLL(LIB_PATH)
+
+OK = 0
+E_NULL, E_SHAPE, E_ALIGN, E_UNSUPPORTED, E_WORKSPACE, E_INDEX_RANGE, E_CUDA, E_TIMEOUT = range(-1, -9, -1)
+DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
+FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC = 1, 2, 4
+
+_DT = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, "fp32": DTYPE_FP32}
+_TORCH_DT = {DTYPE_FP16: torch.float16, DTYPE_BF16: torch.bfloat16, DTYPE_FP32: torch.float32}
+
+
+class LayerDesc(C.Structure):
+    """vptq_layer_desc"""
+    _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("v", C.c_int32), ("k1", C.c_int32),
+                ("k2", C.c_int32), ("n_outlier", C.c_int32), ("v0", C.c_int32), ("k0", C.c_int32),
+                ("x_dtype", C.c_int32), ("out_dtype", C.c_int32), ("flags", C.c_int32)]
+
+
+class LayerPtrs(C.Structure):
+    """vptq_layer_ptrs"""
+    _fields_ = [("packed_idx", C.c_void_p), ("codebook", C.c_void_p),
+                ("res_idx", C.c_void_p), ("res_codebook", C.c_void_p),
+                ("outlier_idx", C.c_void_p), ("outlier_codebook", C.c_void_p),
+                ("scale", C.c_void_p), ("bias", C.c_void_p)]
+
+
+EXPORTS = {
+    "vptq_index_bits": (C.c_int, [C.c_int32]),
+    "vptq_packed_row_bytes": (C.c_int64, [C.c_int32, C.c_int32]),
+    "vptq_packed_bytes": (C.c_int64, [C.c_int32, C.c_int32, C.c_int32]),
+    "vptq_layer_weight_bytes": (C.c_int64, [C.POINTER(LayerDesc)]),
+    "vptq_pack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
+    "vptq_linear_workspace_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32]),
+    "vptq_linear": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
+                              C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "vptq_linear_host_io": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                      C.c_void_p]),
+    "vptq_status_string": (C.c_char_p, [C.c_int]),
+    "vptq_last_cuda_error": (C.c_char_p, []),
+    "vptq_linear_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32]),
+    "vptq_linear_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32]),
+}
+for _name, (_res, _args) in EXPORTS.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class VptqError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        msg = lib.vptq_status_string(code).decode()
+        if code == E_CUDA:
+            msg += ": " + lib.vptq_last_cuda_error().decode()
+        super().__init__(f"libvptq error {code}: {msg}")
+
+
+def _check(code: int) -> None:
+    if code != OK:
+        raise VptqError(code)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_desc(M, N, v, k1, k2=0, n_outlier=0, v0=0, k0=0, x_dtype="fp16", out_dtype="fp16",
+              flags=FLAG_SCALE_BIAS) -> LayerDesc:
+    return LayerDesc(M, N, v, k1, k2, n_outlier, v0, k0, _DT[x_dtype], _DT[out_dtype], flags)
+
+
+# ---- entry points (same names as the C ABI) -------------------------------------------
+
+def vptq_index_bits(k: int) -> int:
+    return lib.vptq_index_bits(k)
+
+
+def vptq_packed_row_bytes(n_cols: int, k: int) -> int:
+    return lib.vptq_packed_row_bytes(n_cols, k)
+
+
+def vptq_packed_bytes(n_rows: int, n_cols: int, k: int) -> int:
+    return lib.vptq_packed_bytes(n_rows, n_cols, k)
+
+
+def vptq_layer_weight_bytes(desc: LayerDesc) -> int:
+    return lib.vptq_layer_weight_bytes(C.byref(desc))
+
+
+def vptq_pack(idx: torch.Tensor, k: int, check: bool = True) -> torch.Tensor:
+    """idx: int32 CUDA tensor [rows][cols] -> uint8 CUDA tensor [rows][row_bytes]."""
+    assert idx.is_cuda and idx.dtype == torch.int32 and idx.dim() == 2 and idx.is_contiguous()
+    rows, cols = idx.shape
+    row_b = lib.vptq_packed_row_bytes(cols, k)
+    if row_b < 0:
+        raise VptqError(int(row_b))
+    packed = torch.empty((rows, row_b), dtype=torch.uint8, device=idx.device)
+    bad = torch.zeros(1, dtype=torch.int32, device=idx.device) if check else None
+    _check(lib.vptq_pack(_ptr(idx), rows, cols, k, _ptr(packed), _ptr(bad), _stream()))
+    return packed
+
+
+def vptq_unpack(packed: torch.Tensor, rows: int, cols: int, k: int) -> torch.Tensor:
+    assert packed.is_cuda and packed.dtype == torch.uint8 and packed.is_contiguous()
+    assert packed.numel() == lib.vptq_packed_bytes(rows, cols, k)
+    idx = torch.empty((rows, cols), dtype=torch.int32, device=packed.device)
+    _check(lib.vptq_unpack(_ptr(packed), rows, cols, k, _ptr(idx), _stream()))
+    return idx
+
+
+def vptq_dequant(desc: LayerDesc, ptrs: LayerPtrs, W_out: torch.Tensor) -> torch.Tensor:
+    assert W_out.is_cuda and W_out.dtype == torch.float16 and W_out.is_contiguous()
+    assert tuple(W_out.shape) == (desc.M, desc.N)
+    _check(lib.vptq_dequant(C.byref(desc), C.byref(ptrs), _ptr(W_out), _stream()))
+    return W_out
+
+
+def vptq_linear_workspace_bytes(desc: LayerDesc, B: int) -> int:
+    n = lib.vptq_linear_workspace_bytes(C.byref(desc), B)
+    if n < 0:
+        raise VptqError(int(n))
+    return n
+
+
+def vptq_linear(desc: LayerDesc, x: torch.Tensor, ptrs: LayerPtrs, out: torch.Tensor,
+                workspace: Optional[torch.Tensor]) -> torch.Tensor:
+    assert x.is_cuda and x.is_contiguous() and out.is_cuda and out.is_contiguous()
+    assert x.dtype == _TORCH_DT[desc.x_dtype] and out.dtype == _TORCH_DT[desc.out_dtype]
+    B = x.shape[0]
+    assert tuple(x.shape) == (B, desc.N) and tuple(out.shape) == (B, desc.M)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vptq_linear(C.byref(desc), _ptr(x), B, C.byref(ptrs), _ptr(out),
+                           _ptr(workspace), ws_bytes, _stream()))
+    return out
+
+
+def vptq_linear_host_io(desc: LayerDesc, x_host: torch.Tensor, ptrs: LayerPtrs, out_host: torch.Tensor,
+                        x_dev: torch.Tensor, out_dev: torch.Tensor,
+                        workspace: Optional[torch.Tensor]) -> torch.Tensor:
+    assert not x_host.is_cuda and not out_host.is_cuda and x_dev.is_cuda and out_dev.is_cuda
+    B = x_host.shape[0]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vptq_linear_host_io(C.byref(desc), _ptr(x_host), B, C.byref(ptrs), _ptr(out_host),
+                                   _ptr(x_dev), _ptr(out_dev), _ptr(workspace), ws_bytes, _stream()))
+    return out_host
+
+
+def vptq_linear_path(desc: LayerDesc, B: int) -> str:
+    return lib.vptq_linear_path(C.byref(desc), B).decode()
+
+
+def vptq_linear_launches(desc: LayerDesc, B: int) -> int:
+    return lib.vptq_linear_launches(C.byref(desc), B)
+
+
+# ---- a quantized layer resident on the device ------------------------------------------
+
+class DeviceLayer:
+    """Holds the device tensors of one quantized layer and the desc/ptrs structs over them.
+
+    Built from a synth.make_layer() dict; the index matrices are packed ON THE DEVICE with
+    vptq_pack (the product's packer).
+    """
+
+    def __init__(self, d: Dict, device="cuda", flags: Optional[int] = None, scale_rows: bool = False):
+        s = d["spec"]
+        self.spec = s
+        dev = torch.device(device)
+
+        def up(a, dt=None):
+            if a is None:
+                return None
+            t = torch.from_numpy(np.ascontiguousarray(a))
+            if dt is not None:
+                t = t.view(dt)
+            return t.to(dev)
+
+        self.idx1 = vptq_pack(up(d["idx1"]), s.k1) if s.Nc > 0 else None
+        self.idx2 = vptq_pack(up(d["idx2"]), s.k2) if (s.k2 and s.Nc > 0) else None
+        self.idx0 = vptq_pack(up(d["idx0"]), s.k0) if s.n_out else None
+        self.c1, self.c2, self.c0 = up(d["c1"]), up(d["c2"]), up(d["c0"])
+        self.scale, self.bias = up(d["scale"]), up(d["bias"])
+        if flags is None:
+            flags = FLAG_SCALE_BIAS if d["scale"] is not None else 0
+            if scale_rows:
+                flags |= FLAG_SCALE_ROWS
+        self.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags)
+        self.ptrs = LayerPtrs(_ptr(self.idx1), _ptr(self.c1), _ptr(self.idx2), _ptr(self.c2),
+                              _ptr(self.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias))
+        self._ws: Dict[int, Optional[torch.Tensor]] = {}
+        self.device = dev
+
+    def with_flags(self, flags: int) -> "DeviceLayer":
+        other = object.__new__(DeviceLayer)
+        other.__dict__.update(self.__dict__)
+        s = self.spec
+        other.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags)
+        other._ws = {}
+        return other
+
+    def weight_bytes(self) -> int:
+        return vptq_layer_weight_bytes(self.desc)
+
+    def workspace(self, B: int) -> Optional[torch.Tensor]:
+        if B not in self._ws:
+            n = vptq_linear_workspace_bytes(self.desc, B)
+            self._ws[B] = torch.empty(n, dtype=torch.uint8, device=self.device) if n > 0 else None
+        return self._ws[B]
+
+    def upload_x(self, x_np: np.ndarray) -> torch.Tensor:
+        t = torch.from_numpy(np.ascontiguousarray(x_np))
+        if self.spec.x_dtype == "bf16":
+            t = t.view(torch.bfloat16)
+        return t.to(self.device)
+
+    def dequant(self) -> torch.Tensor:
+        W = torch.empty((self.spec.M, self.spec.N), dtype=torch.float16, device=self.device)
+        return vptq_dequant(self.desc, self.ptrs, W)
+
+    def linear(self, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B = x.shape[0]
+        if out is None:
+            out = torch.empty((B, self.spec.M), dtype=_TORCH_DT[self.desc.out_dtype], device=self.device)
+        return vptq_linear(self.desc, x, self.ptrs, out, self.workspace(B))

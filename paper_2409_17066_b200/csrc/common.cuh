@@ -1,0 +1,104 @@
+// Shared device/host helpers of libvptq (CUDA side only; the CPU oracle has its own).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/vptq.h"
+
+namespace vptq {
+
+// ---- host-side format arithmetic -----------------------------------------------------
+__host__ __device__ inline int index_bits(int k)
+{
+    int b = 0;
+    while ((1 << b) < k) b++;
+    return b < 1 ? 1 : b;
+}
+
+__host__ __device__ inline long long row_bytes(int cols, int k)
+{
+    long long bytes = ((long long)cols * index_bits(k) + 7) / 8;
+    return (bytes + 15) / 16 * 16;
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// One packed index stream as the kernels see it.
+struct Stream {
+    const uint8_t *ptr;    // packed rows
+    long long stride;      // bytes per row (multiple of 16)
+    int bits;              // bits per index
+    int k;                 // codebook size (indices are clamped to k-1)
+};
+
+inline Stream make_stream(const uint8_t *p, int cols, int k)
+{
+    Stream s;
+    s.ptr = p;
+    s.stride = row_bytes(cols, k);
+    s.bits = index_bits(k);
+    s.k = k;
+    return s;
+}
+
+// Kernel-side view of a layer.
+struct LayerView {
+    int M, N, v, k1, k2, n_out, v0, k0;
+    int R, R0, Nc;
+    int has_scale, scale_rows;
+    int x_bf16, out_dtype;
+    Stream s1, s2, s0;
+    const __half *c1, *c2, *c0;
+    const __half *scale, *bias;
+};
+
+#ifdef __CUDACC__
+// ---- device helpers --------------------------------------------------------------------
+
+// Index c of a packed row, any bit width 1..16.  Reads one or two aligned 32-bit words;
+// the second word is touched only when the index crosses a word boundary, in which case it
+// lies inside the row.
+__device__ __forceinline__ int load_index(const uint8_t *row, int c, int bits)
+{
+    unsigned bit = (unsigned)c * (unsigned)bits;
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(row) + (bit >> 5);
+    unsigned sh = bit & 31u;
+    uint32_t lo = __ldg(w);
+    uint32_t hi = (sh + bits > 32u) ? __ldg(w + 1) : 0u;
+    uint32_t val = __funnelshift_r(lo, hi, sh);
+    return (int)(val & ((1u << bits) - 1u));
+}
+
+__device__ __forceinline__ int clamp_index(int i, int k) { return i < k ? i : k - 1; }
+
+__device__ __forceinline__ float load_act(const void *x, long long i, int is_bf16)
+{
+    if (is_bf16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(x)[i]);
+    return __half2float(reinterpret_cast<const __half *>(x)[i]);
+}
+
+__device__ __forceinline__ void store_out(void *out, long long i, float val, int dtype)
+{
+    if (dtype == VPTQ_DTYPE_FP16) reinterpret_cast<__half *>(out)[i] = __float2half_rn(val);
+    else if (dtype == VPTQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16 *>(out)[i] = __float2bfloat16_rn(val);
+    else reinterpret_cast<float *>(out)[i] = val;
+}
+#endif
+
+// ---- launchers implemented in the kernel files -------------------------------------------
+cudaError_t launch_pack(const int32_t *idx, int rows, int cols, int k, uint8_t *packed,
+                        int32_t *bad_count, cudaStream_t st);
+cudaError_t launch_unpack(const uint8_t *packed, int rows, int cols, int k, int32_t *idx,
+                          cudaStream_t st);
+cudaError_t launch_dequant(const LayerView &L, __half *W, cudaStream_t st);
+
+// generic fallback linear (any geometry, any B): workspace = B*M floats
+long long generic_workspace_bytes(const LayerView &L, int B);
+cudaError_t launch_linear_generic(const LayerView &L, const void *x, int B, void *out,
+                                  void *ws, cudaStream_t st);
+int generic_launches(const LayerView &L, int B);
+
+}  // namespace vptq

@@ -1,0 +1,17 @@
+// Kernel-family selection for vptq_linear.
+#pragma once
+#include "common.cuh"
+
+namespace vptq {
+
+enum LinearPath { PATH_GENERIC = 0, PATH_DECODE_SMEM_MMA, PATH_DECODE_L2_FMA, PATH_GEMM_TCGEN05 };
+
+LinearPath choose_path(const LayerView &L, int B, int flags);
+const char *linear_path_name(const LayerView &L, int B, int flags);
+long long linear_workspace_bytes(const LayerView &L, int B, int flags);
+int linear_launches(const LayerView &L, int B, int flags);
+// returns VPTQ_OK / VPTQ_E_*; *cuda_err is set when the result is VPTQ_E_CUDA
+int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *out, void *ws,
+                    cudaStream_t st, cudaError_t *cuda_err);
+
+}  // namespace vptq

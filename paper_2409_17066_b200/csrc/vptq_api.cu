@@ -1,0 +1,259 @@
+// C ABI of libvptq: argument validation, dispatch, error reporting.  No kernel code here.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "paths.cuh"
+
+using namespace vptq;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e)
+{
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return VPTQ_E_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_desc(const vptq_layer_desc *d)
+{
+    if (d == nullptr) return VPTQ_E_NULL;
+    if (d->M <= 0 || d->N <= 0) return VPTQ_E_SHAPE;
+    if (d->v <= 0 || d->v > 32 || d->k1 <= 0 || d->k1 > 65536) return VPTQ_E_SHAPE;
+    if (d->k2 < 0 || d->k2 > 65536) return VPTQ_E_SHAPE;
+    if (d->n_outlier < 0 || d->n_outlier > d->N) return VPTQ_E_SHAPE;
+    if (d->n_outlier > 0 && (d->v0 <= 0 || d->v0 > 32 || d->k0 <= 0 || d->k0 > 65536)) return VPTQ_E_SHAPE;
+    if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
+    if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
+        d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC)) return VPTQ_E_UNSUPPORTED;
+    if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
+    return VPTQ_OK;
+}
+
+int check_ptrs(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
+{
+    if (p == nullptr) return VPTQ_E_NULL;
+    const bool has_main = d->n_outlier < d->N;
+    if (has_main && (p->packed_idx == nullptr || p->codebook == nullptr)) return VPTQ_E_NULL;
+    if (has_main && d->k2 > 0 && (p->res_idx == nullptr || p->res_codebook == nullptr)) return VPTQ_E_NULL;
+    if (d->n_outlier > 0 && (p->outlier_idx == nullptr || p->outlier_codebook == nullptr)) return VPTQ_E_NULL;
+    if ((d->flags & VPTQ_FLAG_SCALE_BIAS) && (p->scale == nullptr || p->bias == nullptr)) return VPTQ_E_NULL;
+    const void *all[8] = {has_main ? p->packed_idx : nullptr, has_main ? p->codebook : nullptr,
+                          (has_main && d->k2 > 0) ? p->res_idx : nullptr,
+                          (has_main && d->k2 > 0) ? p->res_codebook : nullptr,
+                          d->n_outlier > 0 ? p->outlier_idx : nullptr,
+                          d->n_outlier > 0 ? p->outlier_codebook : nullptr,
+                          (d->flags & VPTQ_FLAG_SCALE_BIAS) ? p->scale : nullptr,
+                          (d->flags & VPTQ_FLAG_SCALE_BIAS) ? p->bias : nullptr};
+    for (int i = 0; i < 8; i++)
+        if (all[i] != nullptr && !aligned16(all[i])) return VPTQ_E_ALIGN;
+    return VPTQ_OK;
+}
+
+LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
+{
+    LayerView L;
+    memset(&L, 0, sizeof(L));
+    L.M = d->M; L.N = d->N; L.v = d->v; L.k1 = d->k1;
+    L.n_out = d->n_outlier;
+    L.v0 = L.n_out ? d->v0 : 1;
+    L.k0 = L.n_out ? d->k0 : 1;
+    L.Nc = L.N - L.n_out;
+    L.k2 = L.Nc > 0 ? d->k2 : 0;
+    L.R = ceil_div(L.M, L.v);
+    L.R0 = L.n_out ? ceil_div(L.M, L.v0) : 0;
+    L.has_scale = (d->flags & VPTQ_FLAG_SCALE_BIAS) ? 1 : 0;
+    L.scale_rows = (d->flags & VPTQ_FLAG_SCALE_ROWS) ? 1 : 0;
+    L.x_bf16 = d->x_dtype == VPTQ_DTYPE_BF16;
+    L.out_dtype = d->out_dtype;
+    if (p != nullptr) {
+        L.s1 = make_stream(p->packed_idx, L.Nc, L.k1);
+        L.s2 = make_stream(L.k2 ? p->res_idx : nullptr, L.Nc, L.k2 ? L.k2 : 1);
+        L.s0 = make_stream(L.n_out ? p->outlier_idx : nullptr, L.n_out, L.k0);
+        L.c1 = reinterpret_cast<const __half *>(p->codebook);
+        L.c2 = L.k2 ? reinterpret_cast<const __half *>(p->res_codebook) : nullptr;
+        L.c0 = L.n_out ? reinterpret_cast<const __half *>(p->outlier_codebook) : nullptr;
+        L.scale = L.has_scale ? reinterpret_cast<const __half *>(p->scale) : nullptr;
+        L.bias = L.has_scale ? reinterpret_cast<const __half *>(p->bias) : nullptr;
+    }
+    return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+int vptq_index_bits(int32_t k)
+{
+    if (k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    return index_bits(k);
+}
+
+int64_t vptq_packed_row_bytes(int32_t n_cols, int32_t k)
+{
+    if (n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    return row_bytes(n_cols, k);
+}
+
+int64_t vptq_packed_bytes(int32_t n_rows, int32_t n_cols, int32_t k)
+{
+    if (n_rows < 0 || n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    return (int64_t)n_rows * row_bytes(n_cols, k);
+}
+
+int64_t vptq_layer_weight_bytes(const vptq_layer_desc *d)
+{
+    int rc = check_desc(d);
+    if (rc != VPTQ_OK) return rc;
+    LayerView L = make_view(d, nullptr);
+    int64_t bytes = 0;
+    if (L.Nc > 0) {
+        bytes += (int64_t)L.R * row_bytes(L.Nc, L.k1) + 2LL * L.k1 * L.v;
+        if (L.k2) bytes += (int64_t)L.R * row_bytes(L.Nc, L.k2) + 2LL * L.k2 * L.v;
+    }
+    if (L.n_out) bytes += (int64_t)L.R0 * row_bytes(L.n_out, L.k0) + 2LL * L.k0 * L.v0;
+    if (L.has_scale) bytes += 4LL * (L.scale_rows ? L.M : L.N);
+    return bytes;
+}
+
+int vptq_pack(const int32_t *idx, int32_t n_rows, int32_t n_cols, int32_t k,
+              uint8_t *packed, int32_t *bad_count, void *stream)
+{
+    if (n_rows < 0 || n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (n_rows == 0 || n_cols == 0) return VPTQ_OK;
+    if (idx == nullptr || packed == nullptr) return VPTQ_E_NULL;
+    if (!aligned16(packed)) return VPTQ_E_ALIGN;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (bad_count != nullptr) {
+        e = cudaMemsetAsync(bad_count, 0, sizeof(int32_t), st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    e = launch_pack(idx, n_rows, n_cols, k, packed, bad_count, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (bad_count != nullptr) {
+        int32_t host_bad = 0;
+        e = cudaMemcpyAsync(&host_bad, bad_count, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (host_bad != 0) return VPTQ_E_INDEX_RANGE;
+    }
+    return VPTQ_OK;
+}
+
+int vptq_unpack(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k,
+                int32_t *idx, void *stream)
+{
+    if (n_rows < 0 || n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (n_rows == 0 || n_cols == 0) return VPTQ_OK;
+    if (idx == nullptr || packed == nullptr) return VPTQ_E_NULL;
+    if (!aligned16(packed)) return VPTQ_E_ALIGN;
+    cudaError_t e = launch_unpack(packed, n_rows, n_cols, k, idx, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
+}
+
+int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, void *W_out, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    rc = check_ptrs(desc, p);
+    if (rc != VPTQ_OK) return rc;
+    if (W_out == nullptr) return VPTQ_E_NULL;
+    if (!aligned16(W_out)) return VPTQ_E_ALIGN;
+    LayerView L = make_view(desc, p);
+    cudaError_t e = launch_dequant(L, reinterpret_cast<__half *>(W_out), reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
+}
+
+int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (B <= 0) return VPTQ_E_SHAPE;
+    LayerView L = make_view(desc, nullptr);
+    return linear_workspace_bytes(L, B, desc->flags);
+}
+
+int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
+                const vptq_layer_ptrs *p, void *out,
+                void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (B <= 0) return VPTQ_E_SHAPE;
+    rc = check_ptrs(desc, p);
+    if (rc != VPTQ_OK) return rc;
+    if (x == nullptr || out == nullptr) return VPTQ_E_NULL;
+    if (!aligned16(x) || !aligned16(out)) return VPTQ_E_ALIGN;
+    LayerView L = make_view(desc, p);
+    long long need = linear_workspace_bytes(L, B, desc->flags);
+    if (need > 0) {
+        if (workspace == nullptr || (long long)workspace_bytes < need) return VPTQ_E_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return VPTQ_E_ALIGN;
+    }
+    cudaError_t e = cudaSuccess;
+    rc = linear_dispatch(L, desc->flags, x, B, out, workspace, reinterpret_cast<cudaStream_t>(stream), &e);
+    if (rc == VPTQ_E_CUDA) return cuda_fail(e);
+    return rc;
+}
+
+int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
+                        const vptq_layer_ptrs *p, void *out_host,
+                        void *x_dev, void *out_dev,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (B <= 0) return VPTQ_E_SHAPE;
+    if (x_host == nullptr || out_host == nullptr || x_dev == nullptr || out_dev == nullptr) return VPTQ_E_NULL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    size_t xb = (size_t)B * desc->N * 2;
+    size_t ob = (size_t)B * desc->M * (desc->out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = vptq_linear(desc, x_dev, B, p, out_dev, workspace, workspace_bytes, stream);
+    if (rc != VPTQ_OK) return rc;
+    e = cudaMemcpyAsync(out_host, out_dev, ob, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return VPTQ_OK;
+}
+
+const char *vptq_status_string(int code)
+{
+    switch (code) {
+    case VPTQ_OK: return "ok";
+    case VPTQ_E_NULL: return "a required pointer is null";
+    case VPTQ_E_SHAPE: return "bad shape or size argument";
+    case VPTQ_E_ALIGN: return "a data pointer is not sufficiently aligned";
+    case VPTQ_E_UNSUPPORTED: return "unsupported dtype or flag combination";
+    case VPTQ_E_WORKSPACE: return "workspace missing or too small";
+    case VPTQ_E_INDEX_RANGE: return "an index lies outside [0,k)";
+    case VPTQ_E_CUDA: return "a CUDA runtime call failed";
+    case VPTQ_E_TIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown status code";
+    }
+}
+
+const char *vptq_last_cuda_error(void) { return g_cuda_err; }
+
+const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B)
+{
+    if (check_desc(desc) != VPTQ_OK || B <= 0) return "invalid";
+    LayerView L = make_view(desc, nullptr);
+    return linear_path_name(L, B, desc->flags);
+}
+
+int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B)
+{
+    if (check_desc(desc) != VPTQ_OK || B <= 0) return VPTQ_E_SHAPE;
+    LayerView L = make_view(desc, nullptr);
+    return linear_launches(L, B, desc->flags);
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares;
+its host-only format arithmetic agrees with the oracle's and with the paper's formulas."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2409_17066_b200 import build as vbuild
+from paper_2409_17066_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    vbuild.build()
+    from paper_2409_17066_b200 import binding as b
+    return b
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "vptq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vptq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(binding):
+    names = _declared_functions()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(binding.lib, n), n
+    # and the binding wraps each of them under the same name
+    for n in names:
+        assert n in binding.EXPORTS, n
+
+
+def test_format_arithmetic_matches_oracle(binding):
+    for k in [1, 2, 3, 5, 16, 17, 255, 256, 257, 4096, 4097, 8192, 65535, 65536]:
+        assert binding.vptq_index_bits(k) == oracle.index_bits(k)
+        for cols in [0, 1, 7, 41, 4055, 4096, 10898]:
+            assert binding.vptq_packed_row_bytes(cols, k) == oracle.row_bytes(cols, k)
+            assert binding.vptq_packed_bytes(13, cols, k) == oracle.packed_bytes(13, cols, k)
+    assert binding.vptq_index_bits(0) == binding.E_SHAPE
+    assert binding.vptq_index_bits(65537) == binding.E_SHAPE
+    assert binding.vptq_packed_bytes(-1, 4, 16) == binding.E_SHAPE
+
+
+def test_layer_weight_bytes_follow_the_bit_formulas(binding):
+    # App. C.2: index bits log2(k)/v per weight and codebook bits (v0*k0 + v1*(k1+k2))*16
+    for cfg in range(5):
+        for s in synth.CONFIGS[cfg]["layers"]:
+            d = binding.make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype)
+            got = binding.vptq_layer_weight_bytes(d)
+            exp = oracle.packed_bytes(s.R, s.Nc, s.k1) + (oracle.packed_bytes(s.R, s.Nc, s.k2) if s.k2 else 0) \
+                + (oracle.packed_bytes(s.R0, s.n_out, s.k0) if s.n_out else 0) \
+                + oracle.codebook_bits(s.v, s.k1, s.k2, s.n_out, s.v0, s.k0) / 8 + 4 * s.N
+            assert got == exp
+    # the worked example of Sec. 2.2: 4096 x 4096, v = 8, k = 256, no scale/bias
+    d = binding.make_desc(4096, 4096, 8, 256, flags=0)
+    assert round(16.0 * 4096 * 4096 / (8 * binding.vptq_layer_weight_bytes(d)), 2) == 15.97
+
+
+def test_argument_errors_need_no_gpu(binding):
+    b = binding
+    d = b.make_desc(64, 64, 8, 256)
+    p = b.LayerPtrs()
+    assert b.lib.vptq_dequant(None, C.byref(p), None, None) == b.E_NULL
+    bad = b.make_desc(0, 64, 8, 256)
+    assert b.lib.vptq_dequant(C.byref(bad), C.byref(p), None, None) == b.E_SHAPE
+    bad = b.make_desc(64, 64, 8, 70000)
+    assert b.lib.vptq_linear_workspace_bytes(C.byref(bad), 1) == b.E_SHAPE
+    bad = b.make_desc(64, 64, 8, 256, n_outlier=65, v0=4, k0=16)
+    assert b.lib.vptq_linear_workspace_bytes(C.byref(bad), 1) == b.E_SHAPE
+    bad = b.make_desc(64, 64, 8, 256)
+    bad.x_dtype = 2
+    assert b.lib.vptq_linear_workspace_bytes(C.byref(bad), 1) == b.E_UNSUPPORTED
+    assert b.lib.vptq_linear_workspace_bytes(C.byref(d), 0) == b.E_SHAPE
+    # required pointers missing -> E_NULL before any CUDA call
+    assert b.lib.vptq_dequant(C.byref(d), C.byref(p), None, None) == b.E_NULL
+    assert b.lib.vptq_linear(C.byref(d), None, 1, C.byref(p), None, None, 0, None) == b.E_NULL
+    # misaligned pointer -> E_ALIGN (never dereferenced)
+    p2 = b.LayerPtrs(0x1008, 0x1000, None, None, None, None, 0x1000, 0x1000)
+    assert b.lib.vptq_dequant(C.byref(d), C.byref(p2), 0x1000, None) == b.E_ALIGN
+    assert b.lib.vptq_status_string(b.E_ALIGN).decode().startswith("a data pointer")
+    assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_mma", "decode_l2_fma", "gemm_tcgen05")
+    assert b.vptq_linear_launches(d, 1) >= 1

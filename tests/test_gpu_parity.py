@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer/byte work and the restored FP16 weights must match bit for bit; layer
+outputs must satisfy max|y_gpu - y_ref| / max|y_ref| <= 2e-3."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2409_17066_b200 import synth
+
+from helpers import TOL, rel_err, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2409_17066_b200 import build as vbuild
+    vbuild.build()
+    from paper_2409_17066_b200 import binding
+    return binding
+
+
+# ------------------------------------------------------------------ pack / unpack
+
+@pytest.mark.parametrize("k", [1, 2, 3, 16, 100, 256, 257, 4096, 5000, 8192, 40000, 65536])
+@pytest.mark.parametrize("shape", [(1, 1), (3, 7), (5, 41), (4, 257), (2, 4055), (9, 4096)])
+def test_pack_unpack_bit_exact(b, k, shape):
+    rng = np.random.default_rng(k * 7 + shape[1])
+    for idx in (rng.integers(0, k, size=shape, dtype=np.int32), np.full(shape, k - 1, np.int32)):
+        ref = oracle.pack(idx, k)
+        dev = torch.from_numpy(idx).cuda()
+        packed = b.vptq_pack(dev, k)
+        assert packed.shape == ref.shape
+        assert np.array_equal(packed.cpu().numpy(), ref)
+        # unpack what the ORACLE packed (independent of the GPU packer)
+        back = b.vptq_unpack(torch.from_numpy(ref).cuda(), shape[0], shape[1], k)
+        assert np.array_equal(back.cpu().numpy(), idx)
+
+
+def test_pack_reports_out_of_range(b):
+    idx = torch.tensor([[0, 1, 5, 2], [7, 0, -1, 3]], dtype=torch.int32, device="cuda")
+    with pytest.raises(b.VptqError) as e:
+        b.vptq_pack(idx, 5)
+    assert e.value.code == b.E_INDEX_RANGE
+    # without the check the call succeeds and stores 0 for the bad entries
+    packed = b.vptq_pack(idx, 5, check=False)
+    back = b.vptq_unpack(packed, 2, 4, 5).cpu().numpy()
+    assert np.array_equal(back, np.array([[0, 1, 0, 2], [0, 0, 0, 3]], np.int32))
+
+
+def test_empty_matrices(b):
+    assert b.lib.vptq_pack(None, 0, 5, 16, None, None, None) == b.OK
+    assert b.lib.vptq_unpack(None, 3, 0, 16, None, None) == b.OK
+
+
+# ------------------------------------------------------------------ dequant, small layers
+
+@pytest.mark.parametrize("spec", synth.small_specs(), ids=lambda s: s.name)
+@pytest.mark.parametrize("scale_rows", [False, True])
+def test_dequant_small_bit_exact(b, spec, scale_rows):
+    if scale_rows and not spec.has_scale:
+        pytest.skip("no scale")
+    d = synth.make_layer(spec, 70, 1, 1)
+    if scale_rows:   # per-output-row tables have length M
+        rng = np.random.default_rng(5)
+        d["scale"] = rng.uniform(0.5, 1.5, spec.M).astype(np.float16)
+        d["bias"] = rng.normal(0, 0.01, spec.M).astype(np.float16)
+    ref = oracle.Layer.from_synth(d, scale_axis=int(scale_rows)).dequant()
+    dl = b.DeviceLayer(d, scale_rows=scale_rows)
+    got = dl.dequant().cpu().numpy()
+    assert np.array_equal(got.view(np.uint16), ref.view(np.uint16))
+
+
+def test_dequant_extreme_values_bit_exact(b):
+    # FP16 subnormals, overflow to inf through the scale, signed zeros
+    spec = synth.LayerSpec("x", 32, 64, v=8, k1=256, k2=256)
+    d = synth.make_layer(spec, 71, 0, 1)
+    bits = np.random.default_rng(9).integers(0, 0x7C00, size=(256, 8)).astype(np.uint16)
+    bits[::2] |= 0x8000
+    d["c1"] = bits.view(np.float16)
+    d["c2"] = (np.random.default_rng(10).integers(0, 0x0400, size=(256, 8)).astype(np.uint16)).view(np.float16)
+    d["scale"][:8] = np.float16(1024.0)
+    ref = oracle.Layer.from_synth(d).dequant()
+    got = b.DeviceLayer(d).dequant().cpu().numpy()
+    assert np.array_equal(got.view(np.uint16), ref.view(np.uint16))
+    assert np.isinf(ref.astype(np.float32)).any() and (np.abs(ref.astype(np.float32)) < 6e-5).any()
+
+
+# ------------------------------------------------------------------ linear, small layers
+
+BATCHES = [1, 2, 3, 4, 5, 8, 9, 16, 17, 33]
+
+
+@pytest.mark.parametrize("spec", synth.small_specs(), ids=lambda s: s.name)
+@pytest.mark.parametrize("force_generic", [False, True])
+def test_linear_small(b, spec, force_generic):
+    for B in BATCHES:
+        d = synth.make_layer(spec, 72, 2, B)
+        y_ref = oracle.Layer.from_synth(d).linear(d["x"])
+        for out_dtype in ("fp32", "fp16"):
+            s2 = synth.LayerSpec(**{**spec.__dict__, "out_dtype": out_dtype})
+            dl = b.DeviceLayer(dict(d, spec=s2))
+            if force_generic:
+                dl = dl.with_flags(dl.desc.flags | b.FLAG_FORCE_GENERIC)
+            y = dl.linear(dl.upload_x(d["x"])).float().cpu().numpy()
+            assert y.shape == y_ref.shape
+            assert rel_err(y, y_ref) <= TOL, (spec.name, B, out_dtype, b.vptq_linear_path(dl.desc, B))
+
+
+@pytest.mark.parametrize("spec", [s for s in synth.small_specs() if s.has_scale][:5], ids=lambda s: s.name)
+def test_linear_small_scale_rows_and_bf16(b, spec):
+    rng = np.random.default_rng(6)
+    for B in (1, 4, 16):
+        s2 = synth.LayerSpec(**{**spec.__dict__, "x_dtype": "bf16", "out_dtype": "fp32"})
+        d = synth.make_layer(s2, 73, 3, B)
+        d["scale"] = rng.uniform(0.5, 1.5, spec.M).astype(np.float16)
+        d["bias"] = rng.normal(0, 0.01, spec.M).astype(np.float16)
+        y_ref = oracle.Layer.from_synth(d, scale_axis=1).linear(d["x"])
+        dl = b.DeviceLayer(d, scale_rows=True)
+        y = dl.linear(dl.upload_x(d["x"])).cpu().numpy()
+        assert rel_err(y, y_ref) <= TOL, (spec.name, B)
+        # bf16 output: equals the fp32 result rounded to bf16, up to one unit in the last place
+        s3 = synth.LayerSpec(**{**s2.__dict__, "out_dtype": "bf16"})
+        dl3 = b.DeviceLayer(dict(d, spec=s3), scale_rows=True)
+        y3 = dl3.linear(dl3.upload_x(d["x"])).float().cpu().numpy()
+        assert np.all(np.abs(y3 - y) <= np.abs(y) * 2.0 ** -7 + 1e-30)
+
+
+def test_linear_is_repeatable_and_leaves_inputs_alone(b):
+    spec = synth.small_specs()[3]
+    d = synth.make_layer(spec, 74, 0, 4)
+    dl = b.DeviceLayer(d)
+    x = dl.upload_x(d["x"])
+    x0 = x.clone()
+    y1 = dl.linear(x).clone()
+    y2 = dl.linear(x).clone()
+    assert torch.equal(x, x0)
+    assert rel_err(y2.float().cpu().numpy(), y1.double().cpu().numpy()) <= 1e-3
+
+
+def test_linear_argument_errors(b):
+    spec = synth.small_specs()[0]
+    d = synth.make_layer(spec, 75, 0, 1)
+    dl = b.DeviceLayer(d)
+    x = dl.upload_x(d["x"])
+    out = torch.empty((1, spec.M), dtype=torch.float16, device="cuda")
+    lib = b.lib
+    assert lib.vptq_linear(C.byref(dl.desc), x.data_ptr(), 0, C.byref(dl.ptrs), out.data_ptr(), None, 0, None) == b.E_SHAPE
+    assert lib.vptq_linear(C.byref(dl.desc), x.data_ptr() + 2, 1, C.byref(dl.ptrs), out.data_ptr(), None, 0, None) == b.E_ALIGN
+    need = b.vptq_linear_workspace_bytes(dl.desc, 1)
+    if need > 0:
+        assert lib.vptq_linear(C.byref(dl.desc), x.data_ptr(), 1, C.byref(dl.ptrs), out.data_ptr(), None, 0, None) == b.E_WORKSPACE
+    # a corrupt stream (index >= k) is clamped, never read out of range: k = 5 needs 3 bits, store 7 everywhere
+    spec5 = synth.LayerSpec("c", 16, 32, v=8, k1=5)
+    d5 = synth.make_layer(spec5, 75, 1, 1)
+    dl5 = b.DeviceLayer(d5)
+    dl5.idx1.fill_(0xFF)
+    W = dl5.dequant().cpu().numpy()
+    d5c = dict(d5, idx1=np.full_like(d5["idx1"], 4))
+    assert np.array_equal(W.view(np.uint16), oracle.Layer.from_synth(d5c).dequant().view(np.uint16))
+    y = dl5.linear(dl5.upload_x(d5["x"])).float().cpu().numpy()
+    assert rel_err(y, oracle.Layer.from_synth(d5c).linear(d5["x"])) <= TOL
