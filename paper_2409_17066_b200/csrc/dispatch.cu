@@ -1,12 +1,13 @@
 // Which kernel family runs a given (layer, batch), and the scratch it needs.
 #include "paths.cuh"
+#include "decode.cuh"
 
 namespace vptq {
 
 LinearPath choose_path(const LayerView &L, int B, int flags)
 {
-    (void)L; (void)B;
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
+    if (B <= 16 && smem_mma_supported(L, B)) return PATH_DECODE_SMEM_MMA;
     return PATH_GENERIC;
 }
 
@@ -23,6 +24,7 @@ const char *linear_path_name(const LayerView &L, int B, int flags)
 long long linear_workspace_bytes(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_MMA: return 0;
     default: return generic_workspace_bytes(L, B);
     }
 }
@@ -30,6 +32,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
 int linear_launches(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_MMA: return 1;
     default: return generic_launches(L, B);
     }
 }
@@ -39,6 +42,7 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
 {
     cudaError_t e;
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_MMA: e = launch_decode_smem_mma(L, x, B, out, st); break;
     default: e = launch_linear_generic(L, x, B, out, ws, st); break;
     }
     *cuda_err = e;

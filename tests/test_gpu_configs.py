@@ -61,7 +61,7 @@ def test_config_layer(b, cfg, li):
         y = dl.linear(dl.upload_x(x_np))
         torch.cuda.synchronize()
         y_rows = y[:, torch.from_numpy(rows).long().cuda()].float().cpu().numpy()
-        assert np.isfinite(y.float()).all().item()
+        assert torch.isfinite(y.float()).all().item()
         assert rel_err(y_rows, y_ref) <= TOL, (cfg, spec.name, B, b.vptq_linear_path(dl.desc, B))
         # a property that holds at any size: the whole output has the scale the samples have
         assert float(y.float().abs().max()) <= 3.0 * np.max(np.abs(y_ref)) + 1e-6
