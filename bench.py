@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the fused vector-quantized linear layer (VPTQ inference hot path) on B200.
+
+One "step" is one pass of the whole hot path over one batch: the seven linear calls
+(q, k, v, o, gate, up, down) of a LLaMA-2-70B-shaped decoder layer at batch 1, each one
+index unpack -> codebook lookups (+ residual) -> scale/bias -> contraction, through the
+C ABI (vptq_linear).  The metric is effective weight GB/s: bytes of the compressed format
+(packed index streams + codebooks + scale + bias, each counted once per call) per second.
+
+  python bench.py --gpus N --steps K --warmup W          # this library
+  python bench.py --impl reference ...                   # the CPU oracle on a bounded sample
+
+Inputs are seeded and synthetic (paper_2409_17066_b200/synth.py).  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "effective_weight_GBps_batch1"
+UNIT = "GB/s"
+WORKLOAD_CFG = 3
+WORKLOAD = "config3_llama2_70b_decoder_layer_q_k_v_o_gate_up_down_v8_k65536_res256_B1"
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def read_traffic(kernel: str):
+    """Per-launch DRAM traffic from the committed ncu summary, if one exists."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f).get(kernel)
+    return None
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+# ------------------------------------------------------------------------------ reference arm
+
+def oracle_sample_rate(layers_np, rows_per_layer, B=1):
+    """Run the CPU oracle on `rows_per_layer` sampled output rows of every layer; return
+    (seconds, compressed bytes those rows stand for)."""
+    import numpy as np
+    from oracle import oracle
+    t0 = time.perf_counter()
+    nbytes = 0.0
+    for d, L, wbytes in layers_np:
+        s = d["spec"]
+        n = min(rows_per_layer, s.M)
+        rows = np.linspace(0, s.M - 1, n).astype(np.int32)
+        L.linear(d["x"][:B], rows)
+        nbytes += wbytes * n / s.M
+    return time.perf_counter() - t0, nbytes
+
+
+def build_oracle_layers(cfg):
+    from oracle import oracle
+    from paper_2409_17066_b200 import synth
+    out = []
+    for li, spec in enumerate(synth.CONFIGS[cfg]["layers"]):
+        d = synth.make_layer(spec, cfg, li, max(synth.CONFIGS[cfg]["batches"]))
+        L = oracle.Layer.from_synth(d)
+        wb = sum(a.size for k, a in L._keep.items() if a is not None and k.startswith("idx")) + \
+            2 * sum(a.size for k, a in L._keep.items() if a is not None and not k.startswith("idx"))
+        out.append((d, L, wb))
+    return out
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    from oracle import oracle
+    layers = build_oracle_layers(WORKLOAD_CFG)
+    # size the per-step sample so that steps + warmup take about two minutes in all
+    oracle_sample_rate(layers, 4)                      # first call pays thread start-up
+    t_probe, _ = oracle_sample_rate(layers, 16)
+    per_row = t_probe / 16
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rows = max(4, min(8192, int(budget / max(per_row, 1e-6))))
+    for _ in range(args.warmup):
+        oracle_sample_rate(layers, rows)
+    t_total, b_total = 0.0, 0.0
+    for _ in range(args.steps):
+        t, nb = oracle_sample_rate(layers, rows)
+        t_total += t
+        b_total += nb
+    value = b_total / t_total / 1e9
+    sample = f"{rows} evenly spaced output rows of each of the 7 layers per step, batch 1"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ this library
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2409_17066_b200 import build as vbuild
+    from paper_2409_17066_b200 import synth
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    vbuild.build()
+    from paper_2409_17066_b200 import binding as vb
+
+    peaks = read_peaks()
+    cfg = synth.CONFIGS[WORKLOAD_CFG]
+    B = 1
+    # every rank is an independent replica with its own seeded weights (layer ordinal offset by rank)
+    copies = 2     # two copies of the index streams, walked alternately: 2 x 329 MB >> 126 MB of L2
+    layers, xs_np = [], []
+    for li, spec in enumerate(cfg["layers"]):
+        d = synth.make_layer(spec, WORKLOAD_CFG, li + 100 * rank, B)
+        dl = vb.DeviceLayer(d)
+        layers.append([dl] + [dl.clone_streams() for _ in range(copies - 1)])
+        xs_np.append(d["x"])
+        del d
+    xs = [layers[i][0].upload_x(xs_np[i]) for i in range(len(layers))]
+    outs = [torch.empty((B, l[0].spec.M), dtype=torch.float16, device="cuda") for l in layers]
+    step_bytes = sum(l[0].weight_bytes() for l in layers)
+    launches_per_step = sum(vb.vptq_linear_launches(l[0].desc, B) for l in layers)
+    paths = sorted({vb.vptq_linear_path(l[0].desc, B) for l in layers})
+
+    def step(i, events=None):
+        c = i % copies
+        for li, l in enumerate(layers):
+            if events is not None:
+                events[li][0].record()
+            l[c].linear(xs[li], outs[li])
+            if events is not None:
+                events[li][1].record()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+
+    # ---- timed region: K steps, CUDA events on the launching stream ---------------------------
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    per_call = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                 for _ in layers] for _ in range(args.steps)]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        step(i, per_call[i])
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+
+    # per-launch durations of the dominant kernel (all seven calls run the same kernel family)
+    call_ms = [[a.elapsed_time(b) for (a, b) in per_call[i]] for i in range(args.steps)]
+    kern_ms_per_step = sum(statistics.mean(call_ms[i][li] for i in range(args.steps)) for li in range(len(layers)))
+    achieved = step_bytes / (kern_ms_per_step * 1e-3) / 1e9
+    per_layer = {layers[li][0].spec.name + f"_{li}": {
+        "us": 1e3 * statistics.mean(call_ms[i][li] for i in range(args.steps)),
+        "GBps": layers[li][0].weight_bytes() / (1e-3 * statistics.mean(call_ms[i][li] for i in range(args.steps))) / 1e9}
+        for li in range(len(layers))}
+
+    # ---- end to end through the C ABI with host buffers ------------------------------------------
+    xh = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in xs_np]
+    oh = [torch.empty((B, l[0].spec.M), dtype=torch.float16).pin_memory() for l in layers]
+    h2d = sum(x.numel() * 2 for x in xh)
+    d2h = sum(o.numel() * 2 for o in oh)
+
+    def step_e2e(i):
+        c = i % copies
+        for li, l in enumerate(layers):
+            vb.vptq_linear_host_io(l[c].desc, xh[li], l[c].ptrs, oh[li], xs[li], outs[li], l[c].workspace(B))
+        torch.cuda.synchronize()     # the step's result is on the host
+
+    for i in range(3):
+        step_e2e(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step_e2e(i)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * step_bytes / (e2e_ms * 1e-3) / 1e9
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "us_per_call_mean": 1e3 * ms_step / len(layers),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch": B, "calls_per_step": len(layers),
+                       "compressed_bytes_per_step": step_bytes, "kernel_paths": paths,
+                       "l2": f"inputs larger than L2: {copies} copies of the {step_bytes / 1e6:.0f} MB index streams walked alternately",
+                       "multi_gpu": "replicas only (no sharding, no collective)"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "activations and outputs cross PCIe every step; the quantized weights stay resident"},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "decode_l2_fma_kernel<1>", "achieved": achieved,
+                         "peak": peaks["hbm"], "peak_source": peaks["source"] + " (copy bandwidth)",
+                         "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                         "frac_of_nominal_8TBps": achieved / 8000.0,
+                         "traffic": read_traffic("decode_l2_fma_kernel"),
+                         "algorithmic_bytes_per_step": step_bytes,
+                         "per_layer": per_layer}}
+
+    if rank == 0:
+        if not args.no_extra:
+            line["extra"] = extra_configs(vb, synth, peaks)
+        if not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def cpu_baseline():
+    from oracle import oracle
+    layers = build_oracle_layers(WORKLOAD_CFG)
+    oracle_sample_rate(layers, 4)                      # first call pays thread start-up
+    t_probe, _ = oracle_sample_rate(layers, 16)
+    rows = max(16, min(8192, int(15.0 / max(t_probe / 16, 1e-6))))
+    t, nb = oracle_sample_rate(layers, rows)
+    return {"value": nb / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "seconds": t,
+            "sample": f"{rows} evenly spaced output rows of each of the 7 layers of the workload, batch 1"}
+
+
+def time_calls(fn, n_variants, iters=30, warm=5):
+    """Median and min milliseconds of fn(i), CUDA events, i cycling over weight copies."""
+    import torch
+    for i in range(warm):
+        fn(i % n_variants)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for i in range(iters):
+        ev[i][0].record()
+        fn(i % n_variants)
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    return statistics.median(ms), min(ms)
+
+
+def extra_configs(vb, synth, peaks):
+    """µs/call, effective weight GB/s (and TFLOP/s for the batched case) of the other workloads."""
+    import torch
+    res = {}
+    for cfg in (0, 1, 2, 4):
+        c = synth.CONFIGS[cfg]
+        seen = set()
+        for li, spec in enumerate(c["layers"]):
+            if (spec.M, spec.N) in seen:
+                continue
+            seen.add((spec.M, spec.N))
+            Bmax = max(c["batches"])
+            d = synth.make_layer(spec, cfg, li, Bmax)
+            base = vb.DeviceLayer(d)
+            wb = base.weight_bytes()
+            n_copies = max(1, min(64, int(2 * 130e6 / wb) + 1))    # walk > 2 x L2 of weights
+            variants = [base] + [base.clone_streams() for _ in range(n_copies - 1)]
+            for B in c["batches"]:
+                x = base.upload_x(d["x"][:B])
+                out = torch.empty((B, spec.M), dtype=vb._TORCH_DT[base.desc.out_dtype], device="cuda")
+                med, mn = time_calls(lambda i: variants[i].linear(x, out), n_copies)
+                key = f"cfg{cfg}_{spec.name}_{spec.M}x{spec.N}_B{B}"
+                r = {"us_median": 1e3 * med, "us_min": 1e3 * mn, "GBps": wb / (med * 1e-3) / 1e9,
+                     "frac_hbm": wb / (med * 1e-3) / 1e9 / peaks["hbm"], "path": vb.vptq_linear_path(base.desc, B),
+                     "weight_copies": n_copies}
+                if B >= 64:
+                    fl = 2.0 * B * spec.M * spec.N
+                    r["TFLOPs"] = fl / (med * 1e-3) / 1e12
+                    r["frac_bf16_peak"] = r["TFLOPs"] / peaks["bf16"]
+                    W = torch.randn(spec.M, spec.N, device="cuda", dtype=torch.float16)
+                    xh = torch.randn(B, spec.N, device="cuda", dtype=torch.float16)
+                    dm, _ = time_calls(lambda i: torch.matmul(xh, W.t()), 1)
+                    r["dense_fp16_matmul_us"] = 1e3 * dm
+                    r["dense_fp16_TFLOPs"] = fl / (dm * 1e-3) / 1e12
+                    del W, xh
+                res[key] = r
+            del variants, base, d
+            torch.cuda.empty_cache()
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -169,7 +169,7 @@ const char *vptq_last_cuda_error(void);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_mma",
  * "decode_l2_fma", "gemm_tcgen05".  For tests and benchmark logs. */
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B);
-/* Number of kernel launches (memsets included) one vptq_linear call issues. */
+/* Number of kernels one vptq_linear call launches (scratch memsets are not counted). */
 int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B);
 
 #ifdef __cplusplus

@@ -229,6 +229,18 @@ class DeviceLayer:
         other._ws = {}
         return other
 
+    def clone_streams(self) -> "DeviceLayer":
+        """A second copy of the packed index streams (codebooks, scale, bias shared): lets a
+        benchmark walk more weight bytes than L2 holds."""
+        other = object.__new__(DeviceLayer)
+        other.__dict__.update(self.__dict__)
+        other.idx1 = None if self.idx1 is None else self.idx1.clone()
+        other.idx2 = None if self.idx2 is None else self.idx2.clone()
+        other.idx0 = None if self.idx0 is None else self.idx0.clone()
+        other.ptrs = LayerPtrs(_ptr(other.idx1), _ptr(self.c1), _ptr(other.idx2), _ptr(self.c2),
+                               _ptr(other.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias))
+        return other
+
     def weight_bytes(self) -> int:
         return vptq_layer_weight_bytes(self.desc)
 

@@ -8,4 +8,10 @@ namespace vptq {
 bool smem_mma_supported(const LayerView &L, int B);
 cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
 
+// main codebook in global memory (L2), residual codebook in shared memory, FP32 FMAs
+bool l2_fma_supported(const LayerView &L, int B);
+long long l2_fma_workspace_bytes(const LayerView &L, int B);
+int l2_fma_launches(const LayerView &L, int B);
+cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
+
 }  // namespace vptq

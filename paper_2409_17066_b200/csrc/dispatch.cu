@@ -4,10 +4,17 @@
 
 namespace vptq {
 
+namespace {
+constexpr int DECODE_MAX_B = 16;
+int decode_group(int B) { return B < DECODE_MAX_B ? B : DECODE_MAX_B; }
+}
+
 LinearPath choose_path(const LayerView &L, int B, int flags)
 {
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
-    if (B <= 16 && smem_mma_supported(L, B)) return PATH_DECODE_SMEM_MMA;
+    const int Bg = decode_group(B);
+    if (smem_mma_supported(L, Bg)) return PATH_DECODE_SMEM_MMA;
+    if (l2_fma_supported(L, Bg)) return PATH_DECODE_L2_FMA;
     return PATH_GENERIC;
 }
 
@@ -25,14 +32,19 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
     case PATH_DECODE_SMEM_MMA: return 0;
+    case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
     default: return generic_workspace_bytes(L, B);
     }
 }
 
 int linear_launches(const LayerView &L, int B, int flags)
 {
+    const int groups = (B + DECODE_MAX_B - 1) / DECODE_MAX_B;
+    const int last = B - (groups - 1) * DECODE_MAX_B;
     switch (choose_path(L, B, flags)) {
-    case PATH_DECODE_SMEM_MMA: return 1;
+    case PATH_DECODE_SMEM_MMA: return groups;
+    case PATH_DECODE_L2_FMA:
+        return (groups - 1) * l2_fma_launches(L, DECODE_MAX_B) + l2_fma_launches(L, last);
     default: return generic_launches(L, B);
     }
 }
@@ -40,10 +52,20 @@ int linear_launches(const LayerView &L, int B, int flags)
 int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *out, void *ws,
                     cudaStream_t st, cudaError_t *cuda_err)
 {
-    cudaError_t e;
-    switch (choose_path(L, B, flags)) {
-    case PATH_DECODE_SMEM_MMA: e = launch_decode_smem_mma(L, x, B, out, st); break;
-    default: e = launch_linear_generic(L, x, B, out, ws, st); break;
+    cudaError_t e = cudaSuccess;
+    const LinearPath path = choose_path(L, B, flags);
+    if (path == PATH_GENERIC) {
+        e = launch_linear_generic(L, x, B, out, ws, st);
+    } else {
+        // decode kernels take up to 16 tokens per launch
+        const size_t oe = (L.out_dtype == VPTQ_DTYPE_FP32) ? 4 : 2;
+        for (int t0 = 0; t0 < B && e == cudaSuccess; t0 += DECODE_MAX_B) {
+            const int Bg = (B - t0 < DECODE_MAX_B) ? (B - t0) : DECODE_MAX_B;
+            const void *xg = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * 2;
+            void *og = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
+            if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, st);
+            else e = launch_decode_l2_fma(L, xg, Bg, og, ws, st);
+        }
     }
     *cuda_err = e;
     return e == cudaSuccess ? VPTQ_OK : VPTQ_E_CUDA;

@@ -71,10 +71,11 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     L.scale_rows = (d->flags & VPTQ_FLAG_SCALE_ROWS) ? 1 : 0;
     L.x_bf16 = d->x_dtype == VPTQ_DTYPE_BF16;
     L.out_dtype = d->out_dtype;
+    // stream geometry is part of the view even without pointers (path selection reads it)
+    L.s1 = make_stream(p ? p->packed_idx : nullptr, L.Nc, L.k1);
+    L.s2 = make_stream((p && L.k2) ? p->res_idx : nullptr, L.Nc, L.k2 ? L.k2 : 1);
+    L.s0 = make_stream((p && L.n_out) ? p->outlier_idx : nullptr, L.n_out, L.k0);
     if (p != nullptr) {
-        L.s1 = make_stream(p->packed_idx, L.Nc, L.k1);
-        L.s2 = make_stream(L.k2 ? p->res_idx : nullptr, L.Nc, L.k2 ? L.k2 : 1);
-        L.s0 = make_stream(L.n_out ? p->outlier_idx : nullptr, L.n_out, L.k0);
         L.c1 = reinterpret_cast<const __half *>(p->codebook);
         L.c2 = L.k2 ? reinterpret_cast<const __half *>(p->res_codebook) : nullptr;
         L.c0 = L.n_out ? reinterpret_cast<const __half *>(p->outlier_codebook) : nullptr;
