@@ -50,6 +50,7 @@ extern "C" {
 #define VPTQ_E_INDEX_RANGE  -6   /* vptq_pack found an index outside [0,k)                  */
 #define VPTQ_E_CUDA         -7   /* a CUDA runtime call failed                              */
 #define VPTQ_E_TIMEOUT      -8   /* a bounded device-side wait gave up (status word)        */
+#define VPTQ_E_SCRATCH_LIMIT -9  /* vptq_linear_noalloc: layer needs more than the built-in scratch */
 
 #define VPTQ_DTYPE_FP16 0
 #define VPTQ_DTYPE_BF16 1
@@ -161,6 +162,42 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
                         const vptq_layer_ptrs *p, void *out_host,
                         void *x_dev, void *out_dev,
                         void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- the same product for callers that cannot allocate device memory ---------------- */
+
+/* The paper has no counterpart to this entry point; it exists for integration reasons only.
+ *
+ * Who needs it: code that runs where a device allocation is not an option — an engine
+ * that handed all device memory to its own arena at start-up and gives plug-in operators
+ * no way to ask for more, or a latency-critical serving loop in which cudaMalloc (which
+ * may synchronise the whole device) is forbidden after initialisation.  vptq_linear
+ * asks such a caller for a workspace it cannot provide; this variant brings its own.
+ *
+ * What it does: the split-K decode kernel of vptq_linear (main codebook in global memory,
+ * i.e. v = 8, 16-bit indices, optional 8-bit residual indices, no outlier columns,
+ * per-input-column scale/bias) for 1 <= B <= 16, with the FP32 partial-sum scratch taken
+ * from an array of VPTQ_NOALLOC_SCRATCH_BYTES that is compiled into the library.  Every GPU
+ * that loads the library holds that array until the process exits.  Inputs and outputs
+ * are the caller's, exactly as for vptq_linear; the result agrees with vptq_linear's to
+ * FP32 summation order.  The call itself allocates nothing: no cudaMalloc, no cudaFree,
+ * no allocating library routine.
+ *
+ * Limits and errors: layers of another geometry return VPTQ_E_UNSUPPORTED; a layer whose
+ * scratch need (4 * min(B,4) * M bytes plus a few KB of counters) exceeds the array
+ * returns VPTQ_E_SCRATCH_LIMIT (M up to about 65000 fits at any B); nothing is launched
+ * in either case.
+ *
+ * Set-up: the first call on each device looks up the array's device address (with that
+ * device current) and remembers it; make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, and it keeps whatever the previous
+ * call left in it.  Each call clears, on `stream`, the part that must start at zero, so
+ * back-to-back calls on one stream are safe; two calls that overlap on the GPU (different
+ * streams, or different threads without ordering) race on the array and give wrong
+ * results. */
+#define VPTQ_NOALLOC_SCRATCH_BYTES (1 << 20)
+int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
+                        const vptq_layer_ptrs *p, void *out, void *stream);
 
 /* ---- diagnostics ------------------------------------------------------------------ */
 

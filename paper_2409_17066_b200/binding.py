@@ -26,6 +26,8 @@ lib = C.CDLL(LIB_PATH)
 
 OK = 0
 E_NULL, E_SHAPE, E_ALIGN, E_UNSUPPORTED, E_WORKSPACE, E_INDEX_RANGE, E_CUDA, E_TIMEOUT = range(-1, -9, -1)
+E_SCRATCH_LIMIT = -9
+NOALLOC_SCRATCH_BYTES = 1 << 20
 DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
 FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC = 1, 2, 4
 
@@ -62,6 +64,8 @@ EXPORTS = {
     "vptq_linear_host_io": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                       C.c_void_p]),
+    "vptq_linear_noalloc": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
+                                      C.c_void_p, C.c_void_p]),
     "vptq_status_string": (C.c_char_p, [C.c_int]),
     "vptq_last_cuda_error": (C.c_char_p, []),
     "vptq_linear_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32]),
@@ -174,6 +178,17 @@ def vptq_linear_host_io(desc: LayerDesc, x_host: torch.Tensor, ptrs: LayerPtrs, 
     _check(lib.vptq_linear_host_io(C.byref(desc), _ptr(x_host), B, C.byref(ptrs), _ptr(out_host),
                                    _ptr(x_dev), _ptr(out_dev), _ptr(workspace), ws_bytes, _stream()))
     return out_host
+
+
+def vptq_linear_noalloc(desc: LayerDesc, x: torch.Tensor, ptrs: LayerPtrs, out: torch.Tensor) -> torch.Tensor:
+    """vptq_linear for callers that cannot hand over a workspace: the scratch is an array built
+    into the library (see include/vptq.h for who needs this, the limits and the sharing rules)."""
+    assert x.is_cuda and x.is_contiguous() and out.is_cuda and out.is_contiguous()
+    assert x.dtype == _TORCH_DT[desc.x_dtype] and out.dtype == _TORCH_DT[desc.out_dtype]
+    B = x.shape[0]
+    assert tuple(x.shape) == (B, desc.N) and tuple(out.shape) == (B, desc.M)
+    _check(lib.vptq_linear_noalloc(C.byref(desc), _ptr(x), B, C.byref(ptrs), _ptr(out), _stream()))
+    return out
 
 
 def vptq_linear_path(desc: LayerDesc, B: int) -> str:

@@ -2,7 +2,10 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
+#include "decode.cuh"
 #include "paths.cuh"
 
 using namespace vptq;
@@ -237,6 +240,7 @@ const char *vptq_status_string(int code)
     case VPTQ_E_INDEX_RANGE: return "an index lies outside [0,k)";
     case VPTQ_E_CUDA: return "a CUDA runtime call failed";
     case VPTQ_E_TIMEOUT: return "a bounded device-side wait gave up";
+    case VPTQ_E_SCRATCH_LIMIT: return "the layer needs more scratch than the built-in array of vptq_linear_noalloc holds";
     default: return "unknown status code";
     }
 }
@@ -258,3 +262,62 @@ int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B)
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// vptq_linear_noalloc: the split-K decode kernel with its scratch in a built-in device array.
+// ---------------------------------------------------------------------------------------------
+// The array lives in this library's device image: every GPU that loads the library holds
+// VPTQ_NOALLOC_SCRATCH_BYTES of it until the process exits.  In host code the name below is
+// only a handle for the runtime, not a device address, so the address is looked up once per
+// device with cudaGetSymbolAddress and that pointer is what the kernel receives.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[VPTQ_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void *g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the CURRENT device (looked up on first use).
+int noalloc_scratch(void **ptr)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return VPTQ_E_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[dev] == nullptr) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (p == nullptr) return VPTQ_E_CUDA;
+        g_noalloc_ptr[dev] = p;
+    }
+    *ptr = g_noalloc_ptr[dev];
+    return VPTQ_OK;
+}
+
+}  // namespace
+
+extern "C" int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
+                                   const vptq_layer_ptrs *p, void *out, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (B <= 0 || B > 16) return VPTQ_E_SHAPE;
+    rc = check_ptrs(desc, p);
+    if (rc != VPTQ_OK) return rc;
+    if (x == nullptr || out == nullptr) return VPTQ_E_NULL;
+    if (!aligned16(x) || !aligned16(out)) return VPTQ_E_ALIGN;
+    if (desc->flags & VPTQ_FLAG_FORCE_GENERIC) return VPTQ_E_UNSUPPORTED;
+    LayerView L = make_view(desc, p);
+    if (!l2_fma_supported(L, B)) return VPTQ_E_UNSUPPORTED;
+    if (l2_fma_workspace_bytes(L, B) > (long long)VPTQ_NOALLOC_SCRATCH_BYTES) return VPTQ_E_SCRATCH_LIMIT;
+    void *scratch = nullptr;
+    rc = noalloc_scratch(&scratch);
+    if (rc != VPTQ_OK) return rc;
+    // the launcher clears the part of the scratch that has to start at zero, on `stream`
+    cudaError_t e = launch_decode_l2_fma(L, x, B, out, scratch, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
+}
+
