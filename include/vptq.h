@@ -203,6 +203,11 @@ int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
 
 const char *vptq_status_string(int code);
 const char *vptq_last_cuda_error(void);
+/* Only meaningful after a vptq_linear call that took the "gemm_tcgen05" path: that path keeps an
+ * int32 status word at byte 0 of its workspace.  This call synchronises `stream`, reads the word
+ * and returns VPTQ_E_TIMEOUT if a bounded device-side wait gave up during the call (the output
+ * is then invalid; the context stays usable), else VPTQ_OK.  A null workspace returns VPTQ_OK. */
+int vptq_workspace_status(const void *workspace, void *stream);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_mma",
  * "decode_l2_fma", "gemm_tcgen05".  For tests and benchmark logs. */
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B);

@@ -68,6 +68,7 @@ EXPORTS = {
                                       C.c_void_p, C.c_void_p]),
     "vptq_status_string": (C.c_char_p, [C.c_int]),
     "vptq_last_cuda_error": (C.c_char_p, []),
+    "vptq_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "vptq_linear_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32]),
 }
@@ -189,6 +190,10 @@ def vptq_linear_noalloc(desc: LayerDesc, x: torch.Tensor, ptrs: LayerPtrs, out: 
     assert tuple(x.shape) == (B, desc.N) and tuple(out.shape) == (B, desc.M)
     _check(lib.vptq_linear_noalloc(C.byref(desc), _ptr(x), B, C.byref(ptrs), _ptr(out), _stream()))
     return out
+
+
+def vptq_workspace_status(workspace: Optional[torch.Tensor]) -> int:
+    return lib.vptq_workspace_status(_ptr(workspace), _stream())
 
 
 def vptq_linear_path(desc: LayerDesc, B: int) -> str:

@@ -1,6 +1,7 @@
 // Which kernel family runs a given (layer, batch), and the scratch it needs.
 #include "paths.cuh"
 #include "decode.cuh"
+#include "gemm.cuh"
 
 namespace vptq {
 
@@ -12,6 +13,7 @@ int decode_group(int B) { return B < DECODE_MAX_B ? B : DECODE_MAX_B; }
 LinearPath choose_path(const LayerView &L, int B, int flags)
 {
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
+    if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
     const int Bg = decode_group(B);
     if (smem_mma_supported(L, Bg)) return PATH_DECODE_SMEM_MMA;
     if (l2_fma_supported(L, Bg)) return PATH_DECODE_L2_FMA;
@@ -33,6 +35,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
     switch (choose_path(L, B, flags)) {
     case PATH_DECODE_SMEM_MMA: return 0;
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
+    case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
     default: return generic_workspace_bytes(L, B);
     }
 }
@@ -43,6 +46,7 @@ int linear_launches(const LayerView &L, int B, int flags)
     const int last = B - (groups - 1) * DECODE_MAX_B;
     switch (choose_path(L, B, flags)) {
     case PATH_DECODE_SMEM_MMA: return groups;
+    case PATH_GEMM_TCGEN05: return gemm_tcgen05_launches(L, B);
     case PATH_DECODE_L2_FMA:
         return (groups - 1) * l2_fma_launches(L, DECODE_MAX_B) + l2_fma_launches(L, last);
     default: return generic_launches(L, B);
@@ -56,6 +60,8 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
     const LinearPath path = choose_path(L, B, flags);
     if (path == PATH_GENERIC) {
         e = launch_linear_generic(L, x, B, out, ws, st);
+    } else if (path == PATH_GEMM_TCGEN05) {
+        e = launch_gemm_tcgen05(L, x, B, out, ws, st);
     } else {
         // decode kernels take up to 16 tokens per launch
         const size_t oe = (L.out_dtype == VPTQ_DTYPE_FP32) ? 4 : 2;

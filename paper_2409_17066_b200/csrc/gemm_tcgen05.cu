@@ -1,0 +1,534 @@
+// Batched / prefill path: out[B][M] = x[B][N] * W_hat^T as a tensor-core GEMM whose weight
+// operand is dequantised on the fly into shared memory (the FP16 weight matrix never exists in
+// global memory; App. D.2 describes the paper's two-phase scheme that this replaces).
+//
+//   D[m][t] (TMEM, FP32, 128 lanes x 512 columns) += A[m][k] * B[t][k]
+//   A = W tile, 128 output rows x 32 input columns, written by producer warps: one 16-byte
+//       centroid (8 consecutive output rows of one input column) = C1[i1] + C2[i2] per store,
+//       in the MN-major 128-byte-swizzled layout tcgen05.mma reads;
+//   B = x*s tile (FP16, scale folded into the activations by a pre-pass), 512 tokens x 32
+//       columns, K-major, loaded by TMA with the 64-byte swizzle (no multicast);
+//   tcgen05.mma.cta_group::1.kind::f16, M = 128, N = 256 (two per token tile), K = 16.
+//
+// Warp roles (448 threads): warp 0 TMA loads of B; warp 1 TMEM allocation + MMA issue (one
+// thread); warps 2-9 dequant producers (a pair per pipeline stage: a1 unpack, a3 main lookup
+// from the L2-resident codebook, a4 residual lookup from shared memory, add, store);
+// warps 10-13 epilogue (tcgen05.ld -> + bias term -> store or red.add).
+// Persistent grid, one CTA per SM, work units (token tile, 128-row tile, K split).
+//
+// Every mbarrier wait is bounded: after about two seconds a waiter records VPTQ_E_TIMEOUT in
+// the status word of the workspace, raises a CTA-wide abort flag and every role leaves its
+// loop; TMEM is freed on all paths.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace vptq {
+
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int TILE_K = 32;
+constexpr int TILE_N = 512;
+constexpr int MMA_N = 256;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;       // 8 KB
+constexpr int B_HALF_BYTES = MMA_N * TILE_K * 2;         // 16 KB
+constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;          // 32 KB
+constexpr int PRODUCER_WARPS = 2 * STAGES;               // 8
+constexpr int EPI_WARPS = 4;
+constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 448
+constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
+constexpr int A_LBO = 1024;   // bytes between the two 64-row blocks of the A stage
+constexpr int B_SBO = 512;    // bytes between consecutive 8-token groups of the B stage (8 x 64 B)
+constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
+
+constexpr int WS_STATUS_BYTES = 256;
+
+struct GemmParams {
+    LayerView L;
+    void *out;
+    int B;
+    int Npad;            // row stride of xs in elements
+    int tiles_m, tiles_t, splits, kb_total, kb_per_split;
+    int cb2_replicated;
+    int cb2_bytes;
+    int *status;         // workspace status word
+    const float *bterm;  // [B]
+};
+
+// ---- PTX wrappers ----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred P1;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+                 "selp.b32 %0, 1, 0, P1;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the wait was abandoned (timeout here or abort raised elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, VPTQ_E_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);            // start address, 16-byte units
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;   // leading-dimension byte offset
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;   // stride-dimension byte offset
+    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+    d |= (uint64_t)layout << 61;                         // swizzle mode
+    return d;
+}
+constexpr uint32_t LAYOUT_SW128 = 2, LAYOUT_SW64 = 4;
+
+// kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128, N = 256
+constexpr uint32_t IDESC = (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
+                           ((uint32_t)(MMA_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- pre-pass: xs = fp16(x * s), bterm[t] = sum_n x[t][n] * b[n], status = 0 --------------------
+__global__ void __launch_bounds__(256)
+gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __half *__restrict__ xs,
+                    float *__restrict__ bterm, int *status)
+{
+    const int t = blockIdx.x;
+    if (t == 0 && threadIdx.x == 0) *status = 0;
+    float acc = 0.f;
+    for (int n = threadIdx.x; n < Npad; n += 256) {
+        float xv = 0.f, sc = 1.f, bi = 0.f;
+        if (n < L.N) {
+            xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
+            if (L.has_scale) {
+                sc = __half2float(__ldg(L.scale + n));
+                bi = __half2float(__ldg(L.bias + n));
+            }
+        }
+        xs[(long long)t * Npad + n] = __float2half_rn(xv * sc);
+        acc += xv * bi;
+    }
+    __shared__ float red[8];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float a = 0.f;
+        for (int w = 0; w < 8; w++) a += red[w];
+        bterm[t] = a;
+    }
+}
+
+// ---- the GEMM ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const LayerView &L = P.L;
+    // carve shared memory; swizzled operand stages need 1024-byte alignment
+    const uint32_t raw = smem_addr(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *sm = smem_raw + (base - raw);
+    const uint32_t sA = base;                                   // STAGES x 8 KB
+    const uint32_t sB = sA + STAGES * A_STAGE_BYTES;            // STAGES x 32 KB
+    uint8_t *cb2_ptr = sm + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+    uint8_t *misc = cb2_ptr + P.cb2_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(misc);        // fullA[4] fullB[4] empty[4] accum_full accum_empty
+    const uint32_t bar0 = smem_addr(bars);
+    auto bar_fullA = [&](int s) { return bar0 + 8u * s; };
+    auto bar_fullB = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
+    const uint32_t bar_accum_full = bar0 + 8u * (3 * STAGES);
+    const uint32_t bar_accum_empty = bar0 + 8u * (3 * STAGES + 1);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * (3 * STAGES + 2));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) {
+            mbar_init(bar_fullA(s), 2);       // one arrival per producer warp of the stage's pair
+            mbar_init(bar_fullB(s), 1);       // the TMA thread's expect_tx arrival
+            mbar_init(bar_empty(s), 1);       // tcgen05.commit
+        }
+        mbar_init(bar_accum_full, 1);
+        mbar_init(bar_accum_empty, EPI_WARPS);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // residual codebook -> shared memory (all threads)
+    if (L.k2) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(L.c2);
+        uint4 *dst = reinterpret_cast<uint4 *>(cb2_ptr);
+        if (P.cb2_replicated) {
+            for (int i = threadIdx.x; i < L.k2 * 8; i += GEMM_THREADS) dst[i] = __ldg(src + (i >> 3));
+        } else {
+            for (int i = threadIdx.x; i < L.k2; i += GEMM_THREADS) dst[i] = __ldg(src + i);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_units = P.tiles_t * P.tiles_m * P.splits;
+
+    if (warp == 0) {
+        // ================= TMA: B tiles =================
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                const int ks = u % P.splits, tt = u / (P.splits * P.tiles_m);
+                const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+                const int t0 = tt * TILE_N;
+                const int halves = (P.B - t0 > MMA_N) ? 2 : 1;
+                for (int kb = kb0; kb < kb1; kb++, it++) {
+                    const int s = it % STAGES;
+                    if (!(ok = mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag, P.status))) break;
+                    mbar_expect_tx(bar_fullB(s), halves * B_HALF_BYTES);
+                    for (int h = 0; h < halves; h++)
+                        tma_load_2d(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES, &tmap_xs, bar_fullB(s),
+                                    kb * TILE_K, t0 + h * MMA_N);
+                }
+            }
+            if (!ok) {
+                // abandoned: give copies still in flight a bounded time to land before the CTA exits
+                const int first = it > STAGES ? it - STAGES : 0;
+                for (int j = first; j < it; j++) {
+                    const long long t0c = clock64();
+                    while (!mbar_try(bar_fullB(j % STAGES), (j / STAGES) & 1) && clock64() - t0c < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issue =================
+        if (lane == 0) {
+            int it = 0, unit_no = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_no++) {
+                const int ks = u % P.splits, tt = u / (P.splits * P.tiles_m);
+                const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+                const int halves = (P.B - tt * TILE_N > MMA_N) ? 2 : 1;
+                // the accumulator must have been drained by the epilogue of the previous unit
+                if (!(ok = mbar_wait(bar_accum_empty, (unit_no & 1) ^ 1, abort_flag, P.status))) break;
+                tc_fence_after();
+                for (int kb = kb0; kb < kb1; kb++, it++) {
+                    const int s = it % STAGES;
+                    const uint32_t par = (it / STAGES) & 1;
+                    if (!(ok = mbar_wait(bar_fullA(s), par, abort_flag, P.status))) break;
+                    if (!(ok = mbar_wait(bar_fullB(s), par, abort_flag, P.status))) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k16 = 0; k16 < TILE_K / 16; k16++) {
+                        const uint64_t adesc = make_smem_desc(sA + s * A_STAGE_BYTES + k16 * 2 * A_SBO,
+                                                              A_LBO, A_SBO, LAYOUT_SW128);
+                        for (int h = 0; h < halves; h++) {
+                            const uint64_t bdesc = make_smem_desc(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES + k16 * 32,
+                                                                  16, B_SBO, LAYOUT_SW64);
+                            umma_f16(tmem_base + h * MMA_N, adesc, bdesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(bar_empty(s));        // stage s may be refilled once these MMAs have read it
+                }
+                if (ok) umma_commit(bar_accum_full);  // accumulator complete
+            }
+        }
+    } else if (warp < 2 + PRODUCER_WARPS) {
+        // ================= dequant producers: A tiles =================
+        const int pw = warp - 2, pair = pw >> 1, half = pw & 1;
+        const int c = lane & 7, grp = lane >> 3;             // row chunk within the 64-row block, 8-column group
+        const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
+        const uint4 *cb2 = reinterpret_cast<const uint4 *>(cb2_ptr);
+        const int rep = P.cb2_replicated ? (lane & 7) : 0, rshift = P.cb2_replicated ? 3 : 0;
+        int it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const int ks = u % P.splits, mt = (u / P.splits) % P.tiles_m;
+            const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+            const int vrow = mt * (TILE_M / 8) + 8 * half + c;
+            const bool row_ok = vrow < L.R;
+            const uint8_t *row1 = L.s1.ptr + (long long)vrow * L.s1.stride;
+            const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)vrow * L.s2.stride : nullptr;
+            for (int kb = kb0; kb < kb1; kb++, it++) {
+                if ((it % STAGES) != pair) continue;
+                const int s = pair;
+                const int col0 = kb * TILE_K + 8 * grp;
+                // a1: packed indices of 8 columns (issued before the wait: they do not touch the stage)
+                uint4 raw1 = make_uint4(0, 0, 0, 0);
+                uint2 raw2 = make_uint2(0, 0);
+                const bool live = row_ok && col0 < L.N;
+                if (live) {
+                    raw1 = __ldg(reinterpret_cast<const uint4 *>(row1 + 2LL * col0));
+                    if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2 + col0));
+                }
+                const uint32_t w1[4] = {raw1.x, raw1.y, raw1.z, raw1.w};
+                // a3: main centroids, 8 reads in flight
+                uint4 cw[8];
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    uint32_t id = (w1[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+                    id = min(id, (uint32_t)(L.k1 - 1));
+                    cw[j] = live ? __ldg(cb1 + id) : make_uint4(0, 0, 0, 0);
+                }
+                // the whole warp takes the same decision: the stores below end in a warp-wide barrier
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag, P.status));
+                if (!ok) break;
+                const uint32_t dst0 = sA + s * A_STAGE_BYTES + grp * A_SBO + half * A_LBO;
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    uint4 w = cw[j];
+                    if (L.k2 && live) {
+                        uint32_t id2 = ((j < 4 ? raw2.x : raw2.y) >> (8 * (j & 3))) & 0xFFu;
+                        id2 = min(id2, (uint32_t)(L.k2 - 1));
+                        const uint4 rv = cb2[(id2 << rshift) + rep];
+                        __half2 a0 = __hadd2(*reinterpret_cast<__half2 *>(&w.x), *reinterpret_cast<const __half2 *>(&rv.x));
+                        __half2 a1 = __hadd2(*reinterpret_cast<__half2 *>(&w.y), *reinterpret_cast<const __half2 *>(&rv.y));
+                        __half2 a2 = __hadd2(*reinterpret_cast<__half2 *>(&w.z), *reinterpret_cast<const __half2 *>(&rv.z));
+                        __half2 a3 = __hadd2(*reinterpret_cast<__half2 *>(&w.w), *reinterpret_cast<const __half2 *>(&rv.w));
+                        w.x = *reinterpret_cast<uint32_t *>(&a0); w.y = *reinterpret_cast<uint32_t *>(&a1);
+                        w.z = *reinterpret_cast<uint32_t *>(&a2); w.w = *reinterpret_cast<uint32_t *>(&a3);
+                    }
+                    if (col0 + j >= L.N) w = make_uint4(0, 0, 0, 0);
+                    const uint32_t dst = dst0 + j * 128 + ((c ^ j) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_fullA(s));
+            }
+        }
+    } else {
+        // ================= epilogue =================
+        const int q = warp & 3;                                  // TMEM lane quarter this warp may read
+        int unit_no = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_no++) {
+            const int ks = u % P.splits, mt = (u / P.splits) % P.tiles_m, tt = u / (P.splits * P.tiles_m);
+            const int t0 = tt * TILE_N;
+            const int m = mt * TILE_M + 32 * q + lane;
+            const int t_cnt = min(TILE_N, P.B - t0);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_accum_full, unit_no & 1, abort_flag, P.status));
+            if (!ok) break;
+            tc_fence_after();
+            for (int c0 = 0; c0 < t_cnt; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, r);
+#pragma unroll
+                for (int j = 0; j < 32; j++) {
+                    const int t = t0 + c0 + j;
+                    if (t < P.B && m < L.M) {
+                        float y = __uint_as_float(r[j]);
+                        if (ks == 0) y += __ldg(P.bterm + t);
+                        if (P.splits == 1) store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
+                        else atomicAdd(reinterpret_cast<float *>(P.out) + (long long)t * L.M + m, y);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_accum_empty);
+        }
+    }
+
+    // ---- teardown: everybody meets, then the allocating warp frees TMEM ------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+struct GemmPlan {
+    int Npad, tiles_m, tiles_t, kb_total, splits, kb_per_split, cb2_rep, cb2_bytes;
+    size_t smem;
+    long long ws_bytes, off_bterm, off_xs;
+};
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else return 148;
+    }
+    return n;
+}
+
+GemmPlan plan_gemm(const LayerView &L, int B)
+{
+    GemmPlan p;
+    p.Npad = (L.N + 7) / 8 * 8;
+    p.tiles_m = ceil_div(L.M, TILE_M);
+    p.tiles_t = ceil_div(B, TILE_N);
+    p.kb_total = ceil_div(L.N, TILE_K);
+    // K splits: minimise waves * (k blocks per unit + epilogue cost in k-block units)
+    const int G = sm_count();
+    const int epi = 16;
+    long long best = -1;
+    p.splits = 1;
+    const int max_split = (L.out_dtype == VPTQ_DTYPE_FP32) ? 16 : 1;   // partial sums meet in an FP32 output
+    for (int s = 1; s <= max_split && s <= p.kb_total; s++) {
+        long long units = (long long)p.tiles_m * p.tiles_t * s;
+        long long waves = (units + G - 1) / G;
+        long long cost = waves * (ceil_div(p.kb_total, s) + epi * (s > 1 ? 2 : 1));
+        if (best < 0 || cost < best) { best = cost; p.splits = s; }
+    }
+    p.kb_per_split = ceil_div(p.kb_total, p.splits);
+    p.splits = ceil_div(p.kb_total, p.kb_per_split);
+    p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
+    p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
+    p.smem = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + p.cb2_bytes + 8 * (3 * STAGES + 2) + 16;
+    p.off_bterm = WS_STATUS_BYTES;
+    p.off_xs = p.off_bterm + ((long long)B * 4 + 255) / 256 * 256;
+    p.ws_bytes = p.off_xs + ((long long)B * p.Npad * 2 + 255) / 256 * 256;
+    return p;
+}
+
+}  // namespace
+
+bool gemm_tcgen05_supported(const LayerView &L, int B)
+{
+    if (B <= 16) return false;
+    if (L.v != 8 || L.n_out != 0 || L.scale_rows) return false;
+    if (L.s1.bits != 16) return false;
+    if (L.k2 && (L.s2.bits != 8 || L.k2 > 2048)) return false;
+    return true;
+}
+
+long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B).ws_bytes; }
+
+int gemm_tcgen05_launches(const LayerView &, int) { return 2; }   // pre-pass + GEMM
+
+cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
+{
+    const GemmPlan pl = plan_gemm(L, B);
+    uint8_t *w8 = reinterpret_cast<uint8_t *>(ws);
+    int *status = reinterpret_cast<int *>(w8);
+    float *bterm = reinterpret_cast<float *>(w8 + pl.off_bterm);
+    __half *xs = reinterpret_cast<__half *>(w8 + pl.off_xs);
+
+    EncodeTiledFn encode = get_encode_fn();
+    if (encode == nullptr) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t gdim[2] = {(cuuint64_t)L.N, (cuuint64_t)B};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pl.Npad * 2};
+    const cuuint32_t box[2] = {TILE_K, MMA_N};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, xs, gdim, gstride, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+
+    cudaError_t e;
+    gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (pl.splits > 1) {
+        e = cudaMemsetAsync(out, 0, (size_t)B * L.M * 4, st);
+        if (e != cudaSuccess) return e;
+    }
+    GemmParams P;
+    P.L = L; P.out = out; P.B = B; P.Npad = pl.Npad;
+    P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.splits = pl.splits;
+    P.kb_total = pl.kb_total; P.kb_per_split = pl.kb_per_split;
+    P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
+    P.status = status; P.bterm = bterm;
+    e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    const int units = pl.tiles_m * pl.tiles_t * pl.splits;
+    const int grid = units < sm_count() ? units : sm_count();
+    gemm_tcgen05_kernel<<<grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
+    return cudaGetLastError();
+}
+
+}  // namespace vptq

@@ -247,6 +247,18 @@ const char *vptq_status_string(int code)
 
 const char *vptq_last_cuda_error(void) { return g_cuda_err; }
 
+int vptq_workspace_status(const void *workspace, void *stream)
+{
+    if (workspace == nullptr) return VPTQ_OK;
+    int32_t word = 0;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return word == VPTQ_E_TIMEOUT ? VPTQ_E_TIMEOUT : VPTQ_OK;
+}
+
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B)
 {
     if (check_desc(desc) != VPTQ_OK || B <= 0) return "invalid";

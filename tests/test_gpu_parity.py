@@ -163,3 +163,28 @@ def test_linear_argument_errors(b):
     assert np.array_equal(W.view(np.uint16), oracle.Layer.from_synth(d5c).dequant().view(np.uint16))
     y = dl5.linear(dl5.upload_x(d5["x"])).float().cpu().numpy()
     assert rel_err(y, oracle.Layer.from_synth(d5c).linear(d5["x"])) <= TOL
+
+
+# ------------------------------------------------------------------ batched tensor-core path
+
+@pytest.mark.parametrize("M,N,k2,B,out_dtype", [
+    (136, 520, 0, 17, "fp32"),       # ragged rows, ragged last k block, one token half
+    (264, 1030, 256, 300, "fp16"),   # residual codebook, both token halves, ragged everything
+    (136, 4100, 256, 40, "fp32"),    # few row tiles and many k blocks: K is split, partial sums meet by red.add
+    (1024, 512, 256, 1100, "fp32"),  # three token tiles (the last one ragged)
+])
+def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
+    spec = synth.LayerSpec("g", M, N, v=8, k1=65536, k2=k2, x_dtype="bf16", out_dtype=out_dtype)
+    d = synth.make_layer(spec, 76, B % 7, B)
+    dl = b.DeviceLayer(d)
+    assert b.vptq_linear_path(dl.desc, B) == "gemm_tcgen05"
+    y_ref = oracle.Layer.from_synth(d).linear(d["x"])
+    x = dl.upload_x(d["x"])
+    for _ in range(2):                                  # twice: the workspace is reused
+        y = dl.linear(x)
+        assert b.vptq_workspace_status(dl.workspace(B)) == b.OK
+        assert rel_err(y.float().cpu().numpy(), y_ref) <= TOL
+    # and against the plain fallback kernel (a second CUDA formulation)
+    g = dl.with_flags(dl.desc.flags | b.FLAG_FORCE_GENERIC)
+    yg = g.linear(x).float().cpu().numpy()
+    assert rel_err(y.float().cpu().numpy(), yg.astype(np.float64)) <= TOL
