@@ -41,13 +41,21 @@ def read_peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
-def read_traffic(kernel: str):
-    """Per-launch DRAM traffic from the committed ncu summary, if one exists."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            return json.load(f).get(kernel)
-    return None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of a launch, from
+# the ncu captures summarised under profiles/ (captured on one layer of the workload; traffic grows
+# in proportion to the packed index streams, so it is scaled by the bytes a launch processes).
+# An entry is removed (-> null in the output) when its kernel changes after the capture.
+NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
+}
+
+ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
+                   "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel"}
+
+
+def read_traffic(kernel: str, algorithmic_bytes_per_launch: float):
+    """Per-launch DRAM traffic scaled from the committed ncu summary, if one exists."""
+    r = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(kernel)
+    return None if r is None else r * algorithmic_bytes_per_launch
 
 
 class ClockSampler:
@@ -139,10 +147,10 @@ def run_reference(args):
     layers = build_oracle_layers(WORKLOAD_CFG)
     # size the per-step sample so that steps + warmup take about two minutes in all
     oracle_sample_rate(layers, 4)                      # first call pays thread start-up
-    t_probe, _ = oracle_sample_rate(layers, 16)
-    per_row = t_probe / 16
+    t_probe, _ = oracle_sample_rate(layers, 64)
+    per_row = t_probe / 64
     budget = 120.0 / max(1, args.steps + args.warmup)
-    rows = max(4, min(8192, int(budget / max(per_row, 1e-6))))
+    rows = max(4, min(28672, int(budget / max(per_row, 1e-6))))
     for _ in range(args.warmup):
         oracle_sample_rate(layers, rows)
     t_total, b_total = 0.0, 0.0
@@ -183,20 +191,29 @@ def run_ours(args):
     from paper_2409_17066_b200 import binding as vb
 
     peaks = read_peaks()
-    cfg = synth.CONFIGS[WORKLOAD_CFG]
-    B = 1
+    cfg_id = args.cfg
+    cfg = synth.CONFIGS[cfg_id]
+    B = args.batch if args.batch > 0 else min(cfg["batches"])
+    keep = set(args.layers.split(",")) if args.layers else None
+    default_case = cfg_id == WORKLOAD_CFG and keep is None and B == 1
     # every rank is an independent replica with its own seeded weights (layer ordinal offset by rank)
-    copies = 2     # two copies of the index streams, walked alternately: 2 x 329 MB >> 126 MB of L2
     layers, xs_np = [], []
     for li, spec in enumerate(cfg["layers"]):
-        d = synth.make_layer(spec, WORKLOAD_CFG, li + 100 * rank, B)
+        if keep is not None and spec.name not in keep:
+            continue
+        d = synth.make_layer(spec, cfg_id, li + 100 * rank, B)
         dl = vb.DeviceLayer(d)
-        layers.append([dl] + [dl.clone_streams() for _ in range(copies - 1)])
+        layers.append([dl])
         xs_np.append(d["x"])
         del d
-    xs = [layers[i][0].upload_x(xs_np[i]) for i in range(len(layers))]
-    outs = [torch.empty((B, l[0].spec.M), dtype=torch.float16, device="cuda") for l in layers]
+    # distinct copies of the index streams, walked in turn, so that every step's weights come
+    # from HBM: copies x step bytes > 2 x L2 (the headline workload: 2 x 329 MB >> 126 MB)
     step_bytes = sum(l[0].weight_bytes() for l in layers)
+    copies = max(2, min(64, int(2 * 130e6 / step_bytes) + 1))
+    for l in layers:
+        l.extend(l[0].clone_streams() for _ in range(copies - 1))
+    xs = [layers[i][0].upload_x(xs_np[i]) for i in range(len(layers))]
+    outs = [torch.empty((B, l[0].spec.M), dtype=vb._TORCH_DT[l[0].desc.out_dtype], device="cuda") for l in layers]
     launches_per_step = sum(vb.vptq_linear_launches(l[0].desc, B) for l in layers)
     paths = sorted({vb.vptq_linear_path(l[0].desc, B) for l in layers})
 
@@ -223,8 +240,10 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
+    # per-call events on every `stride`-th step only (at most ~200 steps), to keep the stream tight
+    stride = max(1, args.steps // 200)
     per_call = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                 for _ in layers] for _ in range(args.steps)]
+                 for _ in layers] if i % stride == 0 else None for i in range(args.steps)]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
@@ -244,19 +263,21 @@ def run_ours(args):
     value = world * step_bytes / (ms_step * 1e-3) / 1e9
 
     # per-launch durations of the dominant kernel (all seven calls run the same kernel family)
-    call_ms = [[a.elapsed_time(b) for (a, b) in per_call[i]] for i in range(args.steps)]
-    kern_ms_per_step = sum(statistics.mean(call_ms[i][li] for i in range(args.steps)) for li in range(len(layers)))
+    call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call if pc is not None]
+    n_ev = len(call_ms)
+    layer_ms = [statistics.mean(call_ms[i][li] for i in range(n_ev)) for li in range(len(layers))]
+    kern_ms_per_step = sum(layer_ms)
     achieved = step_bytes / (kern_ms_per_step * 1e-3) / 1e9
     per_layer = {layers[li][0].spec.name + f"_{li}": {
-        "us": 1e3 * statistics.mean(call_ms[i][li] for i in range(args.steps)),
-        "GBps": layers[li][0].weight_bytes() / (1e-3 * statistics.mean(call_ms[i][li] for i in range(args.steps))) / 1e9}
+        "us": 1e3 * layer_ms[li],
+        "GBps": layers[li][0].weight_bytes() / (1e-3 * layer_ms[li]) / 1e9}
         for li in range(len(layers))}
 
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     xh = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in xs_np]
-    oh = [torch.empty((B, l[0].spec.M), dtype=torch.float16).pin_memory() for l in layers]
-    h2d = sum(x.numel() * 2 for x in xh)
-    d2h = sum(o.numel() * 2 for o in oh)
+    oh = [torch.empty((B, l[0].spec.M), dtype=vb._TORCH_DT[l[0].desc.out_dtype]).pin_memory() for l in layers]
+    h2d = sum(x.numel() * x.element_size() for x in xh)
+    d2h = sum(o.numel() * o.element_size() for o in oh)
 
     def step_e2e(i):
         c = i % copies
@@ -285,7 +306,9 @@ def run_ours(args):
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "us_per_call_mean": 1e3 * ms_step / len(layers),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": B, "calls_per_step": len(layers),
+            "config": {"workload": WORKLOAD if default_case else
+                       f"config{cfg_id}_{'+'.join(l[0].spec.name for l in layers)}_B{B} (profiling case, not the headline workload)",
+                       "batch": B, "calls_per_step": len(layers),
                        "compressed_bytes_per_step": step_bytes, "kernel_paths": paths,
                        "l2": f"inputs larger than L2: {copies} copies of the {step_bytes / 1e6:.0f} MB index streams walked alternately",
                        "multi_gpu": "replicas only (no sharding, no collective)"},
@@ -294,18 +317,29 @@ def run_ours(args):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "activations and outputs cross PCIe every step; the quantized weights stay resident"},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_l2_fma_kernel<1>", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": ROOFLINE_KERNEL[paths[0]], "achieved": achieved,
                          "peak": peaks["hbm"], "peak_source": peaks["source"] + " (copy bandwidth)",
                          "unit": "GB/s", "frac": achieved / peaks["hbm"],
                          "frac_of_nominal_8TBps": achieved / 8000.0,
-                         "traffic": read_traffic("decode_l2_fma_kernel"),
-                         "algorithmic_bytes_per_step": step_bytes,
+                         "traffic": read_traffic(ROOFLINE_KERNEL[paths[0]], step_bytes / launches_per_step),
+                         "algorithmic_bytes_per_launch": step_bytes / launches_per_step,
+                         "launch_us_mean": 1e3 * kern_ms_per_step / launches_per_step,
+                         "launches_per_step": launches_per_step,
+                         "note": "achieved = compressed bytes of a step / sum of the per-call event durations "
+                                 "of a step = mean bytes per launch / mean launch duration",
                          "per_layer": per_layer}}
+    if paths[0] == "gemm_tcgen05":
+        flops = sum(2.0 * B * l[0].spec.M * l[0].spec.N for l in layers)
+        tf = flops / (kern_ms_per_step * 1e-3) / 1e12
+        line["roofline"].update({"bound": "tensor", "achieved": tf, "peak": peaks["bf16"], "unit": "TFLOP/s",
+                                 "frac": tf / peaks["bf16"], "peak_source": peaks["source"] + " (cuBLAS bf16 burst)",
+                                 "traffic": None})
+        line["roofline"].pop("frac_of_nominal_8TBps")
 
     if rank == 0:
-        if not args.no_extra:
+        if not args.no_extra and default_case:
             line["extra"] = extra_configs(vb, synth, peaks)
-        if not args.no_cpu:
+        if not args.no_cpu and default_case:
             line["cpu_baseline"] = cpu_baseline()
         print(json.dumps(line))
     if world > 1:
@@ -318,8 +352,8 @@ def cpu_baseline():
     from oracle import oracle
     layers = build_oracle_layers(WORKLOAD_CFG)
     oracle_sample_rate(layers, 4)                      # first call pays thread start-up
-    t_probe, _ = oracle_sample_rate(layers, 16)
-    rows = max(16, min(8192, int(15.0 / max(t_probe / 16, 1e-6))))
+    t_probe, _ = oracle_sample_rate(layers, 256)
+    rows = max(16, min(28672, int(256 * 15.0 / max(t_probe, 1e-6))))   # about 15 s of CPU work
     t, nb = oracle_sample_rate(layers, rows)
     return {"value": nb / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "seconds": t,
@@ -386,11 +420,15 @@ def extra_configs(vb, synth, peaks):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=1500)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--cfg", type=int, default=WORKLOAD_CFG,
+                    help="workload number (default: the headline workload); others are profiling cases")
+    ap.add_argument("--layers", default="", help="comma-separated layer names to keep (profiling cases)")
+    ap.add_argument("--batch", type=int, default=0, help="tokens per call (default: the workload's smallest)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
