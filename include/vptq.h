@@ -182,10 +182,12 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
  * FP32 summation order.  The call itself allocates nothing: no cudaMalloc, no cudaFree,
  * no allocating library routine.
  *
- * Limits and errors: layers of another geometry return VPTQ_E_UNSUPPORTED; a layer whose
- * scratch need (4 * min(B,4) * M bytes plus a few KB of counters) exceeds the array
- * returns VPTQ_E_SCRATCH_LIMIT (M up to about 65000 fits at any B); nothing is launched
- * in either case.
+ * Limits and errors: layers of another geometry return VPTQ_E_UNSUPPORTED.  The kernel
+ * needs scratch only when the layer's vector rows do not divide well over the SMs (it then
+ * deals the work out regardless of rows and adds partial sums up in scratch): 4 * min(B,4) * M
+ * bytes plus a few KB of counters.  A layer whose need exceeds the array returns
+ * VPTQ_E_SCRATCH_LIMIT (M up to about 65000 fits at any B); nothing is launched in either
+ * case.  vptq_linear_workspace_bytes() tells the need of a given layer and B.
  *
  * Set-up: the first call on each device looks up the array's device address (with that
  * device current) and remembers it; make that first call outside any stream capture.

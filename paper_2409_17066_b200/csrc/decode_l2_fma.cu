@@ -1,18 +1,26 @@
 // Decode path for a main codebook too large for shared memory (k1 = 65536, v = 8: 1 MiB),
 // batch 1..4 per launch.
 //
-// The codebook stays in global memory and is served by L2 (and whatever part of it the
-// per-SM L1 holds); every index costs one 16-byte random read (a3).  The kernel is therefore
-// organised around keeping many of those reads in flight: a lane takes 8 consecutive indices
-// with one 128-bit load (a1), issues the 8 centroid loads back to back, and only then
-// consumes them.  The residual codebook (a4) sits in shared memory, replicated 8 times with a
-// 16-byte skew so that the 8 lanes of a quarter warp always hit different banks.
-//
-// Work split: grid = (row blocks, K slabs).  A CTA stages the scaled activations of its slab
-// (x*s, FP32) in shared memory once and its warps walk vector rows; per (row, slab) a warp
-// reduces its 8*B partial sums with a halving butterfly.  With one slab the result is stored
-// directly; with several, partial sums meet in an FP32 scratch array through atomic adds and
-// the last CTA of a row block (a counter tells) converts and stores (a7).
+// The codebook stays in global memory and is served by L2; every index costs one 16-byte random
+// read (a3), and the rate of those reads (about one L1-missing request per clock per SM), not
+// HBM, bounds the kernel.  It is therefore organised around keeping every SM's read path busy
+// all the time:
+//   - persistent grid, one CTA per SM; the work is cut into (vector row, 256-column chunk) tasks
+//     and every warp owns an equal, contiguous range of them;
+//   - per task a lane takes 8 consecutive indices with one 128-bit load (a1; the next task's
+//     indices are already in flight), issues its 8 centroid reads back to back and only then
+//     consumes them;
+//   - the residual codebook (a4) sits in shared memory, replicated 8 times with a 16-byte skew
+//     so that the 8 lanes of a quarter warp always hit different banks;
+//   - the scaled activations x*s (a6 folded into x) are staged per CTA in shared memory as FP16;
+//     the bias becomes one scalar per token.
+// A warp accumulates in registers while its tasks stay in one vector row and reduces the 8*B
+// partial sums with a halving butterfly at a row change.  Two ways to combine the warps (a7):
+//   OWNER    a CTA owns whole vector rows: partial sums meet in shared memory, no scratch;
+//            used when the rows divide well over the SMs;
+//   balanced tasks are dealt out regardless of rows: partial sums meet in an FP32 scratch array
+//            through atomic adds, and a task counter per block of 16 vector rows tells which warp
+//            completed the block and so converts and stores it.
 #include "common.cuh"
 #include "decode.cuh"
 
@@ -20,20 +28,23 @@ namespace vptq {
 
 namespace {
 
-constexpr int L2_WARPS = 8;
-constexpr int L2_THREADS = L2_WARPS * 32;
+constexpr int RB_ROWS = 16;                 // vector rows per completion counter (balanced mode)
+constexpr int XS_BUDGET = 64 * 1024;        // bytes of staged activations per CTA
+constexpr int PART_BUDGET = 32 * 1024;      // bytes of per-row partial sums per CTA (OWNER mode)
+constexpr int WARPS_TB4 = 16;               // 4 tokens per launch need 128 registers per thread
 
 struct L2FmaParams {
     LayerView L;
     const void *x;
     void *out;
     int B;                 // tokens in this launch (<= TB)
-    int slab_cols;         // columns per K slab (multiple of 256)
+    int slab_cols;         // columns per slab (multiple of 256); one slab of x*s is staged at a time
     int n_slabs;
-    int rows_per_warp;
+    int chunks_total;      // 256-column chunks of a whole row
     int cb2_replicated;    // 1: [k2][8 replicas][16 B], 0: [k2][16 B]
-    float *yacc;           // [B][M] scratch (n_slabs > 1)
-    unsigned *counters;    // [row blocks] scratch (n_slabs > 1)
+    int part_floats;       // OWNER: floats of the per-row partial sums
+    float *yacc;           // balanced: [B][M] scratch, zero on entry
+    unsigned *counters;    // balanced: [ceil(R / RB_ROWS)] scratch, zero on entry
 };
 
 __device__ __forceinline__ float2 h2f(uint32_t w)
@@ -41,241 +52,405 @@ __device__ __forceinline__ float2 h2f(uint32_t w)
     return __half22float2(*reinterpret_cast<__half2 *>(&w));
 }
 
-template <int TB>
-__global__ void __launch_bounds__(L2_THREADS)
+// streaming 128-/64-bit loads of the packed index rows: read once, keep them out of L1
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ld_stream8(const void *p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+// 8 consecutive activations (fp16 or bf16 bits in a uint4) -> floats
+__device__ __forceinline__ void act8_to_float(uint4 q, int is_bf16, float (&f)[8])
+{
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        float2 p;
+        if (is_bf16) p = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w[i]));
+        else p = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+        f[2 * i] = p.x; f[2 * i + 1] = p.y;
+    }
+}
+
+template <int TB, bool RES, bool OWNER, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 1)
 decode_l2_fma_kernel(L2FmaParams P)
 {
+    constexpr int THREADS = WARPS * 32;
     extern __shared__ __align__(16) uint8_t smem[];
     const LayerView &L = P.L;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int slab = blockIdx.y;
-    const int c_begin = slab * P.slab_cols;
-    const int c_end = min(L.N, c_begin + P.slab_cols);
-    const int n_iter = (c_end - c_begin + 255) / 256;
 
-    float *xs = reinterpret_cast<float *>(smem);                       // [n_iter][TB][2][32][4]
-    const int xs_floats = (P.slab_cols / 256) * TB * 256;
-    float *bterm = xs + xs_floats;                                     // [TB]
-    float *red = bterm + 4;                                            // [L2_WARPS][TB]
-    uint4 *cb2 = reinterpret_cast<uint4 *>(red + L2_WARPS * 4);
-    __shared__ unsigned s_last;
+    __half *xs = reinterpret_cast<__half *>(smem);                                   // [TB][slab_cols]
+    float *bterm = reinterpret_cast<float *>(smem + (size_t)TB * P.slab_cols * 2);   // [4]
+    float *red = bterm + 4;                                                          // [WARPS][4]
+    uint4 *cb2 = reinterpret_cast<uint4 *>(red + WARPS * 4);
+    float *part = reinterpret_cast<float *>(cb2 + (RES ? (size_t)L.k2 * (P.cb2_replicated ? 8 : 1) : 0));
 
-    // ---- stage scaled activations of the slab, and the slab's share of the bias term -----------
-    {
-        float bacc[TB];
-#pragma unroll
-        for (int t = 0; t < TB; t++) bacc[t] = 0.f;
-        for (int cl = threadIdx.x; cl < n_iter * 256; cl += L2_THREADS) {
-            const int n = c_begin + cl;
-            const int i = cl >> 8, ln = (cl >> 3) & 31, s = cl & 7;
-            float sc = 1.f, bi = 0.f;
-            if (n < c_end && L.has_scale) {
-                sc = __half2float(__ldg(L.scale + n));
-                bi = __half2float(__ldg(L.bias + n));
-            }
-#pragma unroll
-            for (int t = 0; t < TB; t++) {
-                float xv = (n < c_end && t < P.B) ? load_act(P.x, (long long)t * L.N + n, L.x_bf16) : 0.f;
-                xs[((i * TB + t) * 2 + (s >> 2)) * 128 + ln * 4 + (s & 3)] = xv * sc;
-                bacc[t] += xv * bi;
-            }
-        }
-#pragma unroll
-        for (int t = 0; t < TB; t++) {
-            float a = bacc[t];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            if (lane == 0) red[warp * 4 + t] = a;
-        }
-    }
-    // ---- residual codebook -> shared memory ---------------------------------------------------------
-    if (L.k2) {
+    // rows of this CTA (OWNER) / rank among the CTAs of its slab (balanced)
+    const int r0 = OWNER ? (int)((long long)L.R * blockIdx.x / gridDim.x) : 0;
+    const int r1 = OWNER ? (int)((long long)L.R * (blockIdx.x + 1) / gridDim.x) : L.R;
+    const int my_slab = OWNER ? 0 : blockIdx.x % P.n_slabs;
+    const int grank = OWNER ? 0 : blockIdx.x / P.n_slabs;
+    const int gsize = OWNER ? 1 : (gridDim.x - my_slab + P.n_slabs - 1) / P.n_slabs;
+
+    // ---- residual codebook -> shared memory; clear the partial sums -----------------------------------
+    if (RES) {
         const uint4 *src = reinterpret_cast<const uint4 *>(L.c2);
         if (P.cb2_replicated) {
-            for (int i = threadIdx.x; i < L.k2 * 8; i += L2_THREADS) cb2[i] = __ldg(src + (i >> 3));
+            for (int i = threadIdx.x; i < L.k2 * 8; i += THREADS) cb2[i] = __ldg(src + (i >> 3));
         } else {
-            for (int i = threadIdx.x; i < L.k2; i += L2_THREADS) cb2[i] = __ldg(src + i);
+            for (int i = threadIdx.x; i < L.k2; i += THREADS) cb2[i] = __ldg(src + i);
         }
     }
-    __syncthreads();
-    if (threadIdx.x < TB) {
-        float a = 0.f;
-        for (int w = 0; w < L2_WARPS; w++) a += red[w * 4 + threadIdx.x];
-        bterm[threadIdx.x] = a;
-    }
-    __syncthreads();
+    if (OWNER)
+        for (int i = threadIdx.x; i < P.part_floats; i += THREADS) part[i] = 0.f;
+    if (threadIdx.x < 4) bterm[threadIdx.x] = 0.f;
 
     const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
-    const int rows_per_cta = L2_WARPS * P.rows_per_warp;
-    const int r0 = blockIdx.x * rows_per_cta;
     const int rep = P.cb2_replicated ? (lane & 7) : 0;
     const int rshift = P.cb2_replicated ? 3 : 0;
+    const uint32_t kmax1 = (uint32_t)(L.k1 - 1), kmax2 = RES ? (uint32_t)(L.k2 - 1) : 0u;
 
-    for (int rw = 0; rw < P.rows_per_warp; rw++) {
-        const int r = r0 + rw * L2_WARPS + warp;
-        if (r >= L.R) break;
-        const uint8_t *row1 = L.s1.ptr + (long long)r * L.s1.stride;
-        const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)r * L.s2.stride : nullptr;
+    for (int slab = my_slab; slab < (OWNER ? P.n_slabs : my_slab + 1); slab++) {
+        const int c_begin = slab * P.slab_cols;
+        const int c_end = min(L.N, c_begin + P.slab_cols);
+        const int chunks = (c_end - c_begin + 255) >> 8;
+        // bias term: over this slab (OWNER walks all slabs) or over all columns (balanced: one slab per CTA)
+        const int b_begin = OWNER ? c_begin : 0, b_end = OWNER ? c_end : L.N;
+
+        // ---- this warp's task range: tasks are (row, chunk of the slab), chunk fastest ----------------
+        const long long n_tasks = (long long)(r1 - r0) * chunks;
+        const long long n_workers = (long long)gsize * WARPS;
+        const long long wrank = (long long)grank * WARPS + warp;
+        long long q = n_tasks * wrank / n_workers;
+        const long long q_end = n_tasks * (wrank + 1) / n_workers;
+
+        int r = r0 + (int)(q / chunks), ch = (int)(q % chunks);
+        // packed indices of the first task (a lane's 8 columns: c_begin + 256*ch + 8*lane + s), issued before
+        // the staging below so that their DRAM latency overlaps it
+        uint4 raw1 = make_uint4(0, 0, 0, 0);
+        uint2 raw2 = make_uint2(0, 0);
+        if (q < q_end) {
+            const int grp = (c_begin >> 3) + ch * 32 + lane;
+            if (8 * grp < c_end) {
+                raw1 = ld_stream16(L.s1.ptr + (long long)r * L.s1.stride + 16LL * grp);
+                if (RES) raw2 = ld_stream8(L.s2.ptr + (long long)r * L.s2.stride + 8LL * grp);
+            }
+        }
+
+        // ---- stage x*s of the slab (FP16) and accumulate the bias term sum_n x*b ----------------------
+        {
+            float bacc[TB];
+#pragma unroll
+            for (int t = 0; t < TB; t++) bacc[t] = 0.f;
+            if ((L.N & 7) == 0) {
+                // 8 columns per thread and step, 128-bit loads (rows of x start 16-byte aligned)
+                for (int n = b_begin + 8 * threadIdx.x; n < b_end; n += 8 * THREADS) {
+                    float sc[8], bi[8];
+                    if (L.has_scale) {
+                        act8_to_float(__ldg(reinterpret_cast<const uint4 *>(L.scale + n)), 0, sc);
+                        act8_to_float(__ldg(reinterpret_cast<const uint4 *>(L.bias + n)), 0, bi);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; i++) { sc[i] = 1.f; bi[i] = 0.f; }
+                    }
+                    const bool mine = n >= c_begin && n < c_end;
+#pragma unroll
+                    for (int t = 0; t < TB; t++) {
+                        float xv[8];
+                        if (t < P.B) {
+                            const uint16_t *xp = reinterpret_cast<const uint16_t *>(P.x) + (long long)t * L.N + n;
+                            act8_to_float(__ldg(reinterpret_cast<const uint4 *>(xp)), L.x_bf16, xv);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; i++) xv[i] = 0.f;
+                        }
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int i = 0; i < 4; i++) {
+                            __half2 h = __floats2half2_rn(xv[2 * i] * sc[2 * i], xv[2 * i + 1] * sc[2 * i + 1]);
+                            pk[i] = *reinterpret_cast<uint32_t *>(&h);
+                            bacc[t] += xv[2 * i] * bi[2 * i] + xv[2 * i + 1] * bi[2 * i + 1];
+                        }
+                        if (mine)
+                            *reinterpret_cast<uint4 *>(xs + t * P.slab_cols + (n - c_begin)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            } else {
+                for (int n = b_begin + threadIdx.x; n < b_end; n += THREADS) {
+                    float sc = 1.f, bi = 0.f;
+                    if (L.has_scale) {
+                        sc = __half2float(__ldg(L.scale + n));
+                        bi = __half2float(__ldg(L.bias + n));
+                    }
+                    const bool mine = n >= c_begin && n < c_end;
+#pragma unroll
+                    for (int t = 0; t < TB; t++) {
+                        const float xv = t < P.B ? load_act(P.x, (long long)t * L.N + n, L.x_bf16) : 0.f;
+                        if (mine) xs[t * P.slab_cols + (n - c_begin)] = __float2half_rn(xv * sc);
+                        bacc[t] += xv * bi;
+                    }
+                }
+            }
+            // zero the ragged end of the slab (columns >= N inside the last chunk)
+            for (int cl = (c_end - c_begin) + threadIdx.x; cl < chunks * 256; cl += THREADS)
+#pragma unroll
+                for (int t = 0; t < TB; t++) xs[t * P.slab_cols + cl] = __float2half_rn(0.f);
+#pragma unroll
+            for (int t = 0; t < TB; t++) {
+                float a = bacc[t];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                if (lane == 0) red[warp * 4 + t] = a;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < TB) {
+            float a = bterm[threadIdx.x];
+            for (int w = 0; w < WARPS; w++) a += red[w * 4 + threadIdx.x];
+            bterm[threadIdx.x] = a;
+        }
+        if (!OWNER) __syncthreads();     // balanced: a finishing warp reads bterm right away
+
         float acc[TB][8];
 #pragma unroll
         for (int t = 0; t < TB; t++)
 #pragma unroll
             for (int j = 0; j < 8; j++) acc[t][j] = 0.f;
+        unsigned done_in_row = 0;
 
-        // packed indices of iteration 0 (a lane's 8 columns: c_begin + 256*i + 8*lane + s)
-        int grp = (c_begin >> 3) + lane;
-        uint4 raw1 = make_uint4(0, 0, 0, 0);
-        uint2 raw2 = make_uint2(0, 0);
-        bool live = 8 * grp < L.N;
-        if (live) {
-            raw1 = __ldg(reinterpret_cast<const uint4 *>(row1) + grp);
-            if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2) + grp);
-        }
-        for (int i = 0; i < n_iter; i++) {
+        while (q < q_end) {
             const uint32_t w1[4] = {raw1.x, raw1.y, raw1.z, raw1.w};
             const uint2 cur2 = raw2;
-            const bool cur_live = live;
-            // prefetch the next iteration's indices
-            grp += 32;
-            live = (i + 1 < n_iter) && (8 * grp < c_end);
-            if (live) {
-                raw1 = __ldg(reinterpret_cast<const uint4 *>(row1) + grp);
-                if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2) + grp);
-            }
-            if (!cur_live) continue;       // this lane's 8 columns lie beyond the row: xs there is 0 anyway
-            // a3: 8 centroid reads in flight
-            uint4 cw[8];
-#pragma unroll
-            for (int s = 0; s < 8; s++) {
-                uint32_t id = (w1[s >> 1] >> (16 * (s & 1))) & 0xFFFFu;
-                id = min(id, (uint32_t)(L.k1 - 1));
-                cw[s] = __ldg(cb1 + id);
-            }
-            const float *xp = xs + (size_t)i * TB * 256 + lane * 4;
-#pragma unroll
-            for (int s = 0; s < 8; s++) {
-                float2 c01 = h2f(cw[s].x), c23 = h2f(cw[s].y), c45 = h2f(cw[s].z), c67 = h2f(cw[s].w);
-                if (L.k2) {
-                    uint32_t id2 = ((s < 4 ? cur2.x : cur2.y) >> (8 * (s & 3))) & 0xFFu;
-                    id2 = min(id2, (uint32_t)(L.k2 - 1));
-                    const uint4 rv = cb2[(id2 << rshift) + rep];
-                    float2 r01 = h2f(rv.x), r23 = h2f(rv.y), r45 = h2f(rv.z), r67 = h2f(rv.w);
-                    c01.x += r01.x; c01.y += r01.y; c23.x += r23.x; c23.y += r23.y;
-                    c45.x += r45.x; c45.y += r45.y; c67.x += r67.x; c67.y += r67.y;
-                }
-#pragma unroll
-                for (int t = 0; t < TB; t++) {
-                    const float xv = xp[(t * 2 + (s >> 2)) * 128 + (s & 3)];
-                    acc[t][0] += xv * c01.x; acc[t][1] += xv * c01.y;
-                    acc[t][2] += xv * c23.x; acc[t][3] += xv * c23.y;
-                    acc[t][4] += xv * c45.x; acc[t][5] += xv * c45.y;
-                    acc[t][6] += xv * c67.x; acc[t][7] += xv * c67.y;
+            const int cur_r = r, cur_ch = ch;
+            const bool cur_live = 8 * ((c_begin >> 3) + cur_ch * 32 + lane) < c_end;
+            // next task, and its indices
+            q++;
+            if (++ch == chunks) { ch = 0; r++; }
+            if (q < q_end) {
+                const int grp = (c_begin >> 3) + ch * 32 + lane;
+                if (8 * grp < c_end) {
+                    raw1 = ld_stream16(L.s1.ptr + (long long)r * L.s1.stride + 16LL * grp);
+                    if (RES) raw2 = ld_stream8(L.s2.ptr + (long long)r * L.s2.stride + 8LL * grp);
                 }
             }
-        }
-
-        // ---- halving butterfly: 8*TB partial sums per lane -> one (or a few equal) totals per lane ----
-        constexpr int NV = 8 * TB;
-        float v[NV];
+            if (cur_live) {
+                // a3: 8 centroid reads in flight
+                uint4 cw[8];
 #pragma unroll
-        for (int t = 0; t < TB; t++)
+                for (int s = 0; s < 8; s++) {
+                    uint32_t id = (w1[s >> 1] >> (16 * (s & 1))) & 0xFFFFu;
+                    id = min(id, kmax1);
+                    cw[s] = __ldg(cb1 + id);
+                }
+                // this lane's 8 scaled activations per token
+                uint4 xv4[TB];
 #pragma unroll
-            for (int j = 0; j < 8; j++) v[t * 8 + j] = acc[t][j];
-        int vi = 0;            // index of the value this lane ends up holding
-        {
-            int n = NV, o = 16;
+                for (int t = 0; t < TB; t++)
+                    xv4[t] = *reinterpret_cast<const uint4 *>(xs + t * P.slab_cols + cur_ch * 256 + lane * 8);
 #pragma unroll
-            for (int step = 0; step < 5; step++) {
-                if (n > 1) {
-                    const bool up = (lane & o) != 0;
-                    const int h = n / 2;
-#pragma unroll
-                    for (int k = 0; k < NV / 2; k++) {
-                        if (k < h) {
-                            float send = up ? v[k] : v[k + h];
-                            float keep = up ? v[k + h] : v[k];
-                            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                        }
+                for (int s = 0; s < 8; s++) {
+                    uint4 w = cw[s];
+                    if (RES) {
+                        // a4: residual centroid from shared memory, summed in FP16 (one rounding of 2^-11)
+                        uint32_t id2 = ((s < 4 ? cur2.x : cur2.y) >> (8 * (s & 3))) & 0xFFu;
+                        id2 = min(id2, kmax2);
+                        const uint4 rv = cb2[(id2 << rshift) + rep];
+                        __half2 a0 = __hadd2(*reinterpret_cast<__half2 *>(&w.x), *reinterpret_cast<const __half2 *>(&rv.x));
+                        __half2 a1 = __hadd2(*reinterpret_cast<__half2 *>(&w.y), *reinterpret_cast<const __half2 *>(&rv.y));
+                        __half2 a2 = __hadd2(*reinterpret_cast<__half2 *>(&w.z), *reinterpret_cast<const __half2 *>(&rv.z));
+                        __half2 a3 = __hadd2(*reinterpret_cast<__half2 *>(&w.w), *reinterpret_cast<const __half2 *>(&rv.w));
+                        w.x = *reinterpret_cast<uint32_t *>(&a0); w.y = *reinterpret_cast<uint32_t *>(&a1);
+                        w.z = *reinterpret_cast<uint32_t *>(&a2); w.w = *reinterpret_cast<uint32_t *>(&a3);
                     }
-                    vi += up ? h : 0;
-                    n = h;
-                } else {
-                    v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+                    const float2 c01 = h2f(w.x), c23 = h2f(w.y), c45 = h2f(w.z), c67 = h2f(w.w);
+#pragma unroll
+                    for (int t = 0; t < TB; t++) {
+                        const uint32_t xw = (s >> 1) == 0 ? xv4[t].x : (s >> 1) == 1 ? xv4[t].y : (s >> 1) == 2 ? xv4[t].z : xv4[t].w;
+                        const float2 xp = h2f(xw);
+                        const float xv = (s & 1) ? xp.y : xp.x;
+                        acc[t][0] += xv * c01.x; acc[t][1] += xv * c01.y;
+                        acc[t][2] += xv * c23.x; acc[t][3] += xv * c23.y;
+                        acc[t][4] += xv * c45.x; acc[t][5] += xv * c45.y;
+                        acc[t][6] += xv * c67.x; acc[t][7] += xv * c67.y;
+                    }
                 }
-                o >>= 1;
             }
-        }
-        // lanes that hold a distinct value: for NV = 8 those with (lane & 3) == 0, NV = 16: (lane & 1) == 0
-        const int dup = 32 / NV;
-        if ((lane & (dup - 1)) == 0) {
+            done_in_row++;
+            if (q < q_end && r == cur_r) continue;
+
+            // ---- row change (or end of range): halving butterfly, 8*TB partial sums per lane -> one per lane
+            constexpr int NV = 8 * TB;
+            float v[NV];
+#pragma unroll
+            for (int t = 0; t < TB; t++)
+#pragma unroll
+                for (int j = 0; j < 8; j++) { v[t * 8 + j] = acc[t][j]; acc[t][j] = 0.f; }
+            int vi = 0;            // index of the value this lane ends up holding
+            {
+                int n = NV, o = 16;
+#pragma unroll
+                for (int step = 0; step < 5; step++) {
+                    if (n > 1) {
+                        const bool up = (lane & o) != 0;
+                        const int h = n / 2;
+#pragma unroll
+                        for (int k = 0; k < NV / 2; k++) {
+                            if (k < h) {
+                                float send = up ? v[k] : v[k + h];
+                                float keep = up ? v[k + h] : v[k];
+                                v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                            }
+                        }
+                        vi += up ? h : 0;
+                        n = h;
+                    } else {
+                        v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+                    }
+                    o >>= 1;
+                }
+            }
+            // lanes that hold a distinct value: NV = 8: (lane & 3) == 0, NV = 16: (lane & 1) == 0, NV = 32: all
+            constexpr int dup = 32 / NV;
+            const bool holder = (lane & (dup - 1)) == 0;
             const int t = vi >> 3, j = vi & 7;
-            const int m = r * 8 + j;
-            if (t < P.B && m < L.M) {
-                float y = v[0] + bterm[t];
-                if (P.n_slabs == 1) store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
-                else atomicAdd(P.yacc + (long long)t * L.M + m, y);
+            if (OWNER) {
+                if (holder) atomicAdd(part + ((cur_r - r0) * TB + t) * 8 + j, v[0]);
+            } else {
+                const int m = cur_r * 8 + j;
+                if (holder && t < P.B && m < L.M) atomicAdd(P.yacc + (long long)t * L.M + m, v[0]);
+                // completion: the warp that brings a row block's task count to its total finishes the block
+                __threadfence();
+                __syncwarp();
+                const int rb = cur_r / RB_ROWS;
+                unsigned total = 0, before = 0;
+                if (lane == 0) {
+                    const int rows_in_rb = min(RB_ROWS, L.R - rb * RB_ROWS);
+                    total = (unsigned)rows_in_rb * (unsigned)P.chunks_total;
+                    before = atomicAdd(P.counters + rb, done_in_row);
+                }
+                total = __shfl_sync(0xffffffffu, total, 0);
+                before = __shfl_sync(0xffffffffu, before, 0);
+                if (before + done_in_row == total) {
+                    __threadfence();
+                    const int m_lo = rb * RB_ROWS * 8;
+                    const int m_hi = min(L.M, m_lo + RB_ROWS * 8);
+                    const int n_m = m_hi - m_lo;
+                    for (int i = lane; i < n_m * P.B; i += 32) {
+                        const int tt = i / n_m, mm = m_lo + i % n_m;
+                        const float y = __ldcg(P.yacc + (long long)tt * L.M + mm) + bterm[tt];
+                        store_out(P.out, (long long)tt * L.M + mm, y, L.out_dtype);
+                    }
+                }
             }
+            done_in_row = 0;
         }
+        if (OWNER) __syncthreads();      // the slab's xs is dead; part[] complete after the last slab
     }
 
-    // ---- several slabs: the last CTA of this row block converts and stores -----------------------------
-    if (P.n_slabs > 1) {
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) s_last = (atomicAdd(P.counters + blockIdx.x, 1u) == (unsigned)(P.n_slabs - 1));
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            const int m_lo = r0 * 8;
-            const int m_hi = min(L.M, (r0 + rows_per_cta) * 8);
-            const int n_m = m_hi - m_lo;
-            for (int i = threadIdx.x; i < n_m * P.B; i += L2_THREADS) {
-                const int t = i / n_m, m = m_lo + i % n_m;
-                float y = __ldcg(P.yacc + (long long)t * L.M + m);
-                store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
-            }
+    // ---- OWNER: bias term, conversion, store -----------------------------------------------------------
+    if (OWNER) {
+        const int m_lo = r0 * 8;
+        const int m_hi = min(L.M, r1 * 8);
+        const int n_m = m_hi - m_lo;
+        for (int i = threadIdx.x; i < n_m * P.B; i += THREADS) {
+            const int t = i / n_m, ml = i % n_m;       // consecutive threads -> consecutive m
+            const float y = part[((ml >> 3) * TB + t) * 8 + (ml & 7)] + bterm[t];
+            store_out(P.out, (long long)t * L.M + m_lo + ml, y, L.out_dtype);
         }
     }
 }
 
 struct L2Plan {
-    int slab_cols, n_slabs, rows_per_warp, row_blocks, cb2_rep;
+    int slab_cols, n_slabs, chunks_total, cb2_rep, grid, owner, part_floats, warps;
     size_t smem;
-    long long ws_bytes;
+    long long ws_bytes, off_counters;
 };
+
+int l2_num_sms()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else return 148;
+    }
+    return n;
+}
 
 L2Plan plan_l2(const LayerView &L, int TB)
 {
     L2Plan p;
-    const long long chunks = (L.N + 255) / 256;
-    long long units = (long long)L.R * chunks;
-    long long iters = (units + 3500) / 7000;
-    if (iters < 1) iters = 1;
-    if (iters > 8) iters = 8;
-    if (iters > chunks) iters = chunks;
-    p.n_slabs = (int)((chunks + iters - 1) / iters);
-    iters = (chunks + p.n_slabs - 1) / p.n_slabs;      // balance the slabs
-    p.slab_cols = (int)iters * 256;
-    p.n_slabs = (int)((chunks + iters - 1) / iters);
-    long long wu = (long long)L.R * p.n_slabs;
-    long long rpw = wu / (L2_WARPS * 888);
-    if (rpw < 1) rpw = 1;
-    if (rpw > 8) rpw = 8;
-    p.rows_per_warp = (int)rpw;
-    p.row_blocks = ceil_div(L.R, L2_WARPS * p.rows_per_warp);
+    p.warps = TB == 4 ? WARPS_TB4 : 32;     // 64 registers per thread suffice up to 2 tokens
+    const int n_pad = (L.N + 255) / 256 * 256;
+    int slab = XS_BUDGET / (2 * TB) / 256 * 256;
+    if (slab > n_pad) slab = n_pad;
+    p.slab_cols = slab;
+    p.n_slabs = (n_pad + slab - 1) / slab;
+    p.chunks_total = n_pad / 256;
+    const int G = l2_num_sms();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
-    p.smem = (size_t)(p.slab_cols / 256) * TB * 256 * 4 + 4 * 4 + L2_WARPS * 4 * 4 +
-             (size_t)L.k2 * 16 * (p.cb2_rep ? 8 : 1);
+    // OWNER mode when whole rows divide well over the SMs (and over the warps of a CTA)
+    const int rows_cta = ceil_div(L.R, G);
+    const double eff_cta = (double)L.R / ((double)(L.R < G ? L.R : G) * rows_cta) * (L.R < G ? (double)L.R / G : 1.0);
+    const long long t_cta = (long long)rows_cta * (slab / 256);
+    const double eff_warp = (double)t_cta / ((double)p.warps * (double)((t_cta + p.warps - 1) / p.warps));
+    p.part_floats = rows_cta * TB * 8;
+    p.owner = (eff_cta * eff_warp >= 0.80 && (long long)p.part_floats * 4 <= PART_BUDGET) ? 1 : 0;
+    if (!p.owner) p.part_floats = 0;
+    p.grid = p.owner ? (L.R < G ? L.R : G) : (G < p.n_slabs ? p.n_slabs : G);
+    p.smem = (size_t)TB * slab * 2 + 4 * 4 + (size_t)p.warps * 4 * 4 + (size_t)L.k2 * 16 * (p.cb2_rep ? 8 : 1) +
+             (size_t)p.part_floats * 4;
     p.ws_bytes = 0;
-    if (p.n_slabs > 1) {
-        long long y = ((long long)TB * L.M * 4 + 255) / 256 * 256;
-        long long c = ((long long)p.row_blocks * 4 + 255) / 256 * 256;
-        p.ws_bytes = y + c;
+    p.off_counters = 0;
+    if (!p.owner) {
+        p.off_counters = ((long long)TB * L.M * 4 + 255) / 256 * 256;
+        p.ws_bytes = p.off_counters + ((long long)ceil_div(L.R, RB_ROWS) * 4 + 255) / 256 * 256;
     }
     return p;
 }
 
 int token_group(int B) { return B >= 4 ? 4 : (B >= 2 ? 2 : 1); }
+
+template <int TB, bool RES, bool OWNER, int WARPS>
+cudaError_t launch_one(const L2FmaParams &P, const L2Plan &pl, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB, RES, OWNER, WARPS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    decode_l2_fma_kernel<TB, RES, OWNER, WARPS><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
+    return cudaGetLastError();
+}
+
+template <int TB, int WARPS>
+cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, int Bg, void *out,
+                         void *ws, cudaStream_t st)
+{
+    L2FmaParams P;
+    P.L = L; P.x = x; P.out = out; P.B = Bg;
+    P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.chunks_total = pl.chunks_total;
+    P.cb2_replicated = pl.cb2_rep; P.part_floats = pl.part_floats;
+    P.yacc = nullptr; P.counters = nullptr;
+    if (!pl.owner) {
+        P.yacc = reinterpret_cast<float *>(ws);
+        P.counters = reinterpret_cast<unsigned *>(reinterpret_cast<uint8_t *>(ws) + pl.off_counters);
+        cudaError_t e = cudaMemsetAsync(ws, 0, (size_t)pl.ws_bytes, st);
+        if (e != cudaSuccess) return e;
+    }
+    const bool res = L.k2 > 0;
+    if (pl.owner) return res ? launch_one<TB, true, true, WARPS>(P, pl, st) : launch_one<TB, false, true, WARPS>(P, pl, st);
+    return res ? launch_one<TB, true, false, WARPS>(P, pl, st) : launch_one<TB, false, false, WARPS>(P, pl, st);
+}
 
 }  // namespace
 
@@ -301,30 +476,6 @@ int l2_fma_launches(const LayerView &L, int B)
     return groups;     // one kernel per token group (the scratch memset is not a kernel)
 }
 
-template <int TB>
-static cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, int Bg, void *out,
-                                void *ws, cudaStream_t st)
-{
-    L2FmaParams P;
-    P.L = L; P.x = x; P.out = out; P.B = Bg;
-    P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.rows_per_warp = pl.rows_per_warp;
-    P.cb2_replicated = pl.cb2_rep;
-    P.yacc = nullptr; P.counters = nullptr;
-    cudaError_t e;
-    if (pl.n_slabs > 1) {
-        long long y = ((long long)TB * L.M * 4 + 255) / 256 * 256;
-        P.yacc = reinterpret_cast<float *>(ws);
-        P.counters = reinterpret_cast<unsigned *>(reinterpret_cast<uint8_t *>(ws) + y);
-        e = cudaMemsetAsync(ws, 0, (size_t)pl.ws_bytes, st);
-        if (e != cudaSuccess) return e;
-    }
-    e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-    if (e != cudaSuccess) return e;
-    dim3 grid(pl.row_blocks, pl.n_slabs);
-    decode_l2_fma_kernel<TB><<<grid, L2_THREADS, pl.smem, st>>>(P);
-    return cudaGetLastError();
-}
-
 cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
 {
     const int TB = token_group(B);
@@ -335,9 +486,9 @@ cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void 
         const void *xg = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * xe;
         void *og = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
         cudaError_t e;
-        if (TB == 4) e = launch_group<4>(L, pl, xg, Bg, og, ws, st);
-        else if (TB == 2) e = launch_group<2>(L, pl, xg, Bg, og, ws, st);
-        else e = launch_group<1>(L, pl, xg, Bg, og, ws, st);
+        if (TB == 4) e = launch_group<4, WARPS_TB4>(L, pl, xg, Bg, og, ws, st);
+        else if (TB == 2) e = launch_group<2, 32>(L, pl, xg, Bg, og, ws, st);
+        else e = launch_group<1, 32>(L, pl, xg, Bg, og, ws, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
