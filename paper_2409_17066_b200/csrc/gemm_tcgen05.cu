@@ -10,11 +10,17 @@
 //       columns, K-major, loaded by TMA with the 64-byte swizzle (no multicast);
 //   tcgen05.mma.cta_group::1.kind::f16, M = 128, N = 256 (two per token tile), K = 16.
 //
-// Warp roles (448 threads): warp 0 TMA loads of B; warp 1 TMEM allocation + MMA issue (one
-// thread); warps 2-9 dequant producers (a pair per pipeline stage: a1 unpack, a3 main lookup
-// from the L2-resident codebook, a4 residual lookup from shared memory, add, store);
-// warps 10-13 epilogue (tcgen05.ld -> + bias term -> store or red.add).
-// Persistent grid, one CTA per SM, work units (token tile, 128-row tile, K split).
+// Warp roles (576 threads): warp 0 TMA loads of B; warp 1 TMEM allocation + MMA issue (one
+// thread); warps 2-9 dequant producers (a pair per k block: a1 unpack with the next visit's
+// indices already in flight, a3 main lookup from the L2-resident codebook, a4 residual lookup
+// from shared memory, add, store); warps 10-17 epilogue (tcgen05.ld -> + bias term -> store or
+// red.add), two per TMEM lane quarter.
+// A and B have rings of their own: A is deep (the producers' gathers need about a microsecond),
+// B holds 32 KB per stage and is shallow.
+// Persistent grid, one CTA per SM.  The work is the list of (tile, k block) units, tile =
+// (token tile, 128-row tile); with an FP32 output every CTA takes an equal, contiguous share of
+// the units, whatever tile they fall in (partial tiles meet in the output by red.add), so all
+// SMs stay busy; other output types are dealt out in whole tiles.
 //
 // Every mbarrier wait is bounded: after about two seconds a waiter records VPTQ_E_TIMEOUT in
 // the status word of the workspace, raises a CTA-wide abort flag and every role leaves its
@@ -32,12 +38,14 @@ constexpr int TILE_M = 128;
 constexpr int TILE_K = 32;
 constexpr int TILE_N = 512;
 constexpr int MMA_N = 256;
-constexpr int STAGES = 4;
+constexpr int A_STAGES = 8;                              // ring of dequantised weight tiles
+constexpr int B_STAGES = 3;                              // ring of activation tiles
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;       // 8 KB
 constexpr int B_HALF_BYTES = MMA_N * TILE_K * 2;         // 16 KB
 constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;          // 32 KB
-constexpr int PRODUCER_WARPS = 2 * STAGES;               // 8
-constexpr int EPI_WARPS = 4;
+constexpr int PAIRS = 4;                                 // producer warp pairs; pair p fills k blocks p, p+PAIRS, ...
+constexpr int PRODUCER_WARPS = 2 * PAIRS;
+constexpr int EPI_WARPS = 8;
 constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 448
 constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
 constexpr int A_LBO = 1024;   // bytes between the two 64-row blocks of the A stage
@@ -51,7 +59,9 @@ struct GemmParams {
     void *out;
     int B;
     int Npad;            // row stride of xs in elements
-    int tiles_m, tiles_t, splits, kb_total, kb_per_split;
+    int tiles_m, tiles_t, kb_total;
+    int unit_gran;       // a CTA's share of the units is a multiple of this (1, or kb_total = whole tiles)
+    long long units;     // tiles_m * tiles_t * kb_total
     int cb2_replicated;
     int cb2_bytes;
     int *status;         // workspace status word
@@ -191,27 +201,32 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     const uint32_t raw = smem_addr(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
-    const uint32_t sA = base;                                   // STAGES x 8 KB
-    const uint32_t sB = sA + STAGES * A_STAGE_BYTES;            // STAGES x 32 KB
-    uint8_t *cb2_ptr = sm + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+    const uint32_t sA = base;                                   // A_STAGES x 8 KB
+    const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x 32 KB
+    uint8_t *cb2_ptr = sm + A_STAGES * A_STAGE_BYTES + B_STAGES * B_STAGE_BYTES;
     uint8_t *misc = cb2_ptr + P.cb2_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(misc);        // fullA[4] fullB[4] empty[4] accum_full accum_empty
+    uint64_t *bars = reinterpret_cast<uint64_t *>(misc);   // fullA[] emptyA[] fullB[] emptyB[] accum_full accum_empty
     const uint32_t bar0 = smem_addr(bars);
     auto bar_fullA = [&](int s) { return bar0 + 8u * s; };
-    auto bar_fullB = [&](int s) { return bar0 + 8u * (STAGES + s); };
-    auto bar_empty = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
-    const uint32_t bar_accum_full = bar0 + 8u * (3 * STAGES);
-    const uint32_t bar_accum_empty = bar0 + 8u * (3 * STAGES + 1);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * (3 * STAGES + 2));
+    auto bar_emptyA = [&](int s) { return bar0 + 8u * (A_STAGES + s); };
+    auto bar_fullB = [&](int s) { return bar0 + 8u * (2 * A_STAGES + s); };
+    auto bar_emptyB = [&](int s) { return bar0 + 8u * (2 * A_STAGES + B_STAGES + s); };
+    constexpr int N_RING_BARS = 2 * A_STAGES + 2 * B_STAGES;
+    const uint32_t bar_accum_full = bar0 + 8u * N_RING_BARS;
+    const uint32_t bar_accum_empty = bar0 + 8u * (N_RING_BARS + 1);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * (N_RING_BARS + 2));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; s++) {
-            mbar_init(bar_fullA(s), 2);       // one arrival per producer warp of the stage's pair
+        for (int s = 0; s < A_STAGES; s++) {
+            mbar_init(bar_fullA(s), 2);       // one arrival per producer warp of a pair
+            mbar_init(bar_emptyA(s), 1);      // tcgen05.commit
+        }
+        for (int s = 0; s < B_STAGES; s++) {
             mbar_init(bar_fullB(s), 1);       // the TMA thread's expect_tx arrival
-            mbar_init(bar_empty(s), 1);       // tcgen05.commit
+            mbar_init(bar_emptyB(s), 1);      // tcgen05.commit
         }
         mbar_init(bar_accum_full, 1);
         mbar_init(bar_accum_empty, EPI_WARPS);
@@ -237,21 +252,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_units = P.tiles_t * P.tiles_m * P.splits;
+    // this CTA's share of the (tile, k block) units: [u_begin, u_end), boundaries multiples of unit_gran
+    const long long groups = P.units / P.unit_gran;
+    const long long u_begin = groups * blockIdx.x / gridDim.x * P.unit_gran;
+    const long long u_end = groups * (blockIdx.x + 1) / gridDim.x * P.unit_gran;
+    // A segment is the part of one tile inside the share: k blocks [kb0, kb1) of tile `tile`.
+#define FOR_EACH_SEGMENT                                                                          \
+    for (long long u = u_begin; u < u_end && ok; u += kb1 - kb0)                                    \
+        if (tile = (int)(u / P.kb_total), kb0 = (int)(u % P.kb_total),                              \
+            kb1 = (int)min((long long)P.kb_total, kb0 + (u_end - u)), true)
+    int tile = 0, kb0 = 0, kb1 = 0;
+    bool ok = true;
 
     if (warp == 0) {
         // ================= TMA: B tiles =================
         if (lane == 0) {
             int it = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const int ks = u % P.splits, tt = u / (P.splits * P.tiles_m);
-                const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+            FOR_EACH_SEGMENT {
+                const int tt = tile / P.tiles_m;
                 const int t0 = tt * TILE_N;
                 const int halves = (P.B - t0 > MMA_N) ? 2 : 1;
                 for (int kb = kb0; kb < kb1; kb++, it++) {
-                    const int s = it % STAGES;
-                    if (!(ok = mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag, P.status))) break;
+                    const int s = it % B_STAGES;
+                    if (!(ok = mbar_wait(bar_emptyB(s), ((it / B_STAGES) & 1) ^ 1, abort_flag, P.status))) break;
                     mbar_expect_tx(bar_fullB(s), halves * B_HALF_BYTES);
                     for (int h = 0; h < halves; h++)
                         tma_load_2d(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES, &tmap_xs, bar_fullB(s),
@@ -260,44 +283,43 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
             }
             if (!ok) {
                 // abandoned: give copies still in flight a bounded time to land before the CTA exits
-                const int first = it > STAGES ? it - STAGES : 0;
+                const int first = it > B_STAGES ? it - B_STAGES : 0;
                 for (int j = first; j < it; j++) {
                     const long long t0c = clock64();
-                    while (!mbar_try(bar_fullB(j % STAGES), (j / STAGES) & 1) && clock64() - t0c < 20000000ll) {}
+                    while (!mbar_try(bar_fullB(j % B_STAGES), (j / B_STAGES) & 1) && clock64() - t0c < 20000000ll) {}
                 }
             }
         }
     } else if (warp == 1) {
         // ================= MMA issue =================
         if (lane == 0) {
-            int it = 0, unit_no = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_no++) {
-                const int ks = u % P.splits, tt = u / (P.splits * P.tiles_m);
-                const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+            int it = 0, seg_no = 0;
+            FOR_EACH_SEGMENT {
+                const int tt = tile / P.tiles_m;
                 const int halves = (P.B - tt * TILE_N > MMA_N) ? 2 : 1;
-                // the accumulator must have been drained by the epilogue of the previous unit
-                if (!(ok = mbar_wait(bar_accum_empty, (unit_no & 1) ^ 1, abort_flag, P.status))) break;
+                // the accumulator must have been drained by the epilogue of the previous segment
+                if (!(ok = mbar_wait(bar_accum_empty, (seg_no & 1) ^ 1, abort_flag, P.status))) break;
                 tc_fence_after();
                 for (int kb = kb0; kb < kb1; kb++, it++) {
-                    const int s = it % STAGES;
-                    const uint32_t par = (it / STAGES) & 1;
-                    if (!(ok = mbar_wait(bar_fullA(s), par, abort_flag, P.status))) break;
-                    if (!(ok = mbar_wait(bar_fullB(s), par, abort_flag, P.status))) break;
+                    const int sa = it % A_STAGES, sb = it % B_STAGES;
+                    if (!(ok = mbar_wait(bar_fullA(sa), (it / A_STAGES) & 1, abort_flag, P.status))) break;
+                    if (!(ok = mbar_wait(bar_fullB(sb), (it / B_STAGES) & 1, abort_flag, P.status))) break;
                     tc_fence_after();
 #pragma unroll
                     for (int k16 = 0; k16 < TILE_K / 16; k16++) {
-                        const uint64_t adesc = make_smem_desc(sA + s * A_STAGE_BYTES + k16 * 2 * A_SBO,
+                        const uint64_t adesc = make_smem_desc(sA + sa * A_STAGE_BYTES + k16 * 2 * A_SBO,
                                                               A_LBO, A_SBO, LAYOUT_SW128);
                         for (int h = 0; h < halves; h++) {
-                            const uint64_t bdesc = make_smem_desc(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES + k16 * 32,
+                            const uint64_t bdesc = make_smem_desc(sB + sb * B_STAGE_BYTES + h * B_HALF_BYTES + k16 * 32,
                                                                   16, B_SBO, LAYOUT_SW64);
                             umma_f16(tmem_base + h * MMA_N, adesc, bdesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
                         }
                     }
-                    umma_commit(bar_empty(s));        // stage s may be refilled once these MMAs have read it
+                    umma_commit(bar_emptyA(sa));      // the stages may be refilled once these MMAs have read them
+                    umma_commit(bar_emptyB(sb));
                 }
                 if (ok) umma_commit(bar_accum_full);  // accumulator complete
+                seg_no++;
             }
         }
     } else if (warp < 2 + PRODUCER_WARPS) {
@@ -307,46 +329,55 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
         const uint4 *cb2 = reinterpret_cast<const uint4 *>(cb2_ptr);
         const int rep = P.cb2_replicated ? (lane & 7) : 0, rshift = P.cb2_replicated ? 3 : 0;
-        int it = 0;
-        bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-            const int ks = u % P.splits, mt = (u / P.splits) % P.tiles_m;
-            const int kb0 = ks * P.kb_per_split, kb1 = min(P.kb_total, kb0 + P.kb_per_split);
+        const uint32_t kmax1 = (uint32_t)(L.k1 - 1), kmax2 = L.k2 ? (uint32_t)(L.k2 - 1) : 0u;
+        int it0 = 0;                                         // k blocks of earlier segments
+        FOR_EACH_SEGMENT {
+            const int mt = tile % P.tiles_m;
             const int vrow = mt * (TILE_M / 8) + 8 * half + c;
             const bool row_ok = vrow < L.R;
             const uint8_t *row1 = L.s1.ptr + (long long)vrow * L.s1.stride;
             const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)vrow * L.s2.stride : nullptr;
-            for (int kb = kb0; kb < kb1; kb++, it++) {
-                if ((it % STAGES) != pair) continue;
-                const int s = pair;
+            // this pair's k blocks of the segment: those whose running number is = pair (mod PAIRS)
+            int kb = kb0 + ((pair - it0 % PAIRS) + PAIRS) % PAIRS;
+            // a1: packed indices of 8 columns; the next visit's are loaded one visit ahead
+            uint4 raw1 = make_uint4(0, 0, 0, 0);
+            uint2 raw2 = make_uint2(0, 0);
+            if (kb < kb1 && row_ok && kb * TILE_K + 8 * grp < L.N) {
+                raw1 = __ldg(reinterpret_cast<const uint4 *>(row1 + 2LL * (kb * TILE_K + 8 * grp)));
+                if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2 + (kb * TILE_K + 8 * grp)));
+            }
+            for (; kb < kb1; kb += PAIRS) {
+                const int it = it0 + (kb - kb0);
+                const int s = it % A_STAGES;
                 const int col0 = kb * TILE_K + 8 * grp;
-                // a1: packed indices of 8 columns (issued before the wait: they do not touch the stage)
-                uint4 raw1 = make_uint4(0, 0, 0, 0);
-                uint2 raw2 = make_uint2(0, 0);
                 const bool live = row_ok && col0 < L.N;
-                if (live) {
-                    raw1 = __ldg(reinterpret_cast<const uint4 *>(row1 + 2LL * col0));
-                    if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2 + col0));
-                }
                 const uint32_t w1[4] = {raw1.x, raw1.y, raw1.z, raw1.w};
-                // a3: main centroids, 8 reads in flight
+                const uint2 cur2 = raw2;
+                {
+                    const int ncol = col0 + PAIRS * TILE_K;
+                    if (kb + PAIRS < kb1 && row_ok && ncol < L.N) {
+                        raw1 = __ldg(reinterpret_cast<const uint4 *>(row1 + 2LL * ncol));
+                        if (L.k2) raw2 = __ldg(reinterpret_cast<const uint2 *>(row2 + ncol));
+                    }
+                }
+                // a3: main centroids, 8 reads in flight (issued before the wait: they do not touch the stage)
                 uint4 cw[8];
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
                     uint32_t id = (w1[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
-                    id = min(id, (uint32_t)(L.k1 - 1));
+                    id = min(id, kmax1);
                     cw[j] = live ? __ldg(cb1 + id) : make_uint4(0, 0, 0, 0);
                 }
                 // the whole warp takes the same decision: the stores below end in a warp-wide barrier
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((it / STAGES) & 1) ^ 1, abort_flag, P.status));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_emptyA(s), ((it / A_STAGES) & 1) ^ 1, abort_flag, P.status));
                 if (!ok) break;
                 const uint32_t dst0 = sA + s * A_STAGE_BYTES + grp * A_SBO + half * A_LBO;
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
                     uint4 w = cw[j];
                     if (L.k2 && live) {
-                        uint32_t id2 = ((j < 4 ? raw2.x : raw2.y) >> (8 * (j & 3))) & 0xFFu;
-                        id2 = min(id2, (uint32_t)(L.k2 - 1));
+                        uint32_t id2 = ((j < 4 ? cur2.x : cur2.y) >> (8 * (j & 3))) & 0xFFu;
+                        id2 = min(id2, kmax2);
                         const uint4 rv = cb2[(id2 << rshift) + rep];
                         __half2 a0 = __hadd2(*reinterpret_cast<__half2 *>(&w.x), *reinterpret_cast<const __half2 *>(&rv.x));
                         __half2 a1 = __hadd2(*reinterpret_cast<__half2 *>(&w.y), *reinterpret_cast<const __half2 *>(&rv.y));
@@ -363,39 +394,78 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_fullA(s));
             }
+            it0 += kb1 - kb0;
         }
     } else {
-        // ================= epilogue =================
+        // ================= epilogue: two warps per TMEM lane quarter, one per 256-token half =================
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
-        int unit_no = 0;
-        bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_no++) {
-            const int ks = u % P.splits, mt = (u / P.splits) % P.tiles_m, tt = u / (P.splits * P.tiles_m);
+        const int h = (warp - (2 + PRODUCER_WARPS)) >> 2;        // token half of the tile
+        const bool fp32_out = L.out_dtype == VPTQ_DTYPE_FP32;
+        const unsigned Mu = (unsigned)L.M;
+        int seg_no = 0;
+        FOR_EACH_SEGMENT {
+            const int mt = tile % P.tiles_m, tt = tile / P.tiles_m;
             const int t0 = tt * TILE_N;
             const int m = mt * TILE_M + 32 * q + lane;
             const int t_cnt = min(TILE_N, P.B - t0);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_accum_full, unit_no & 1, abort_flag, P.status));
+            const bool partial = kb0 != 0 || kb1 != P.kb_total;
+            // bias terms of this warp's 256 tokens, loaded before the wait (a load inside the drain would
+            // cost an L2 round trip under load): lane l holds token 32*i + l of chunk i
+            float bt_chunk[MMA_N / 32];
+#pragma unroll
+            for (int i = 0; i < MMA_N / 32; i++) {
+                const int t = t0 + h * MMA_N + 32 * i + lane;
+                bt_chunk[i] = (kb0 == 0 && t < P.B) ? __ldg(P.bterm + t) : 0.f;
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_accum_full, seg_no & 1, abort_flag, P.status));
             if (!ok) break;
             tc_fence_after();
-            for (int c0 = 0; c0 < t_cnt; c0 += 32) {
+#pragma unroll
+            for (int ci = 0; ci < MMA_N / 32; ci++) {        // unrolled: bt_chunk[] stays in registers
+                const int c0 = h * MMA_N + 32 * ci;
+                if (c0 >= t_cnt) break;
+                const float bt_lane = bt_chunk[ci];
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, r);
+                if (kb0 == 0) {
 #pragma unroll
-                for (int j = 0; j < 32; j++) {
-                    const int t = t0 + c0 + j;
-                    if (t < P.B && m < L.M) {
-                        float y = __uint_as_float(r[j]);
-                        if (ks == 0) y += __ldg(P.bterm + t);
-                        if (P.splits == 1) store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
-                        else atomicAdd(reinterpret_cast<float *>(P.out) + (long long)t * L.M + m, y);
+                    for (int j = 0; j < 32; j++)
+                        r[j] = __float_as_uint(__uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bt_lane, j));
+                }
+                if (m < L.M) {
+                    const int nt = min(32, P.B - (t0 + c0));           // tokens of this chunk that exist
+                    if (fp32_out) {
+                        // one element per token row; independent addresses, no serial pointer chain
+                        float *p = reinterpret_cast<float *>(P.out) + (long long)(t0 + c0) * L.M + m;
+                        if (nt == 32 && !partial) {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) p[(unsigned)j * Mu] = __uint_as_float(r[j]);
+                        } else if (nt == 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) atomicAdd(p + (unsigned)j * Mu, __uint_as_float(r[j]));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) {
+                                if (j < nt) {
+                                    if (!partial) p[(unsigned)j * Mu] = __uint_as_float(r[j]);
+                                    else atomicAdd(p + (unsigned)j * Mu, __uint_as_float(r[j]));
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j++)
+                            if (j < nt) store_out(P.out, (long long)(t0 + c0 + j) * L.M + m, __uint_as_float(r[j]), L.out_dtype);
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_accum_empty);
+            seg_no++;
         }
     }
+#undef FOR_EACH_SEGMENT
 
     // ---- teardown: everybody meets, then the allocating warp frees TMEM ------------------------------
     tc_fence_before();
@@ -427,7 +497,8 @@ EncodeTiledFn get_encode_fn()
 }
 
 struct GemmPlan {
-    int Npad, tiles_m, tiles_t, kb_total, splits, kb_per_split, cb2_rep, cb2_bytes;
+    int Npad, tiles_m, tiles_t, kb_total, unit_gran, grid, any_partial, cb2_rep, cb2_bytes;
+    long long units;
     size_t smem;
     long long ws_bytes, off_bterm, off_xs;
 };
@@ -451,23 +522,19 @@ GemmPlan plan_gemm(const LayerView &L, int B)
     p.tiles_m = ceil_div(L.M, TILE_M);
     p.tiles_t = ceil_div(B, TILE_N);
     p.kb_total = ceil_div(L.N, TILE_K);
-    // K splits: minimise waves * (k blocks per unit + epilogue cost in k-block units)
+    p.units = (long long)p.tiles_m * p.tiles_t * p.kb_total;
+    // partial tiles meet in an FP32 output by red.add; other output types get whole tiles
+    p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32) ? 1 : p.kb_total;
+    const long long groups = p.units / p.unit_gran;
     const int G = sm_count();
-    const int epi = 16;
-    long long best = -1;
-    p.splits = 1;
-    const int max_split = (L.out_dtype == VPTQ_DTYPE_FP32) ? 16 : 1;   // partial sums meet in an FP32 output
-    for (int s = 1; s <= max_split && s <= p.kb_total; s++) {
-        long long units = (long long)p.tiles_m * p.tiles_t * s;
-        long long waves = (units + G - 1) / G;
-        long long cost = waves * (ceil_div(p.kb_total, s) + epi * (s > 1 ? 2 : 1));
-        if (best < 0 || cost < best) { best = cost; p.splits = s; }
-    }
-    p.kb_per_split = ceil_div(p.kb_total, p.splits);
-    p.splits = ceil_div(p.kb_total, p.kb_per_split);
+    p.grid = (int)(groups < G ? groups : G);
+    p.any_partial = 0;
+    for (int c = 1; c < p.grid; c++)
+        if ((groups * c / p.grid * p.unit_gran) % p.kb_total != 0) p.any_partial = 1;
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
     p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
-    p.smem = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + p.cb2_bytes + 8 * (3 * STAGES + 2) + 16;
+    p.smem = 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)B_STAGES * B_STAGE_BYTES + p.cb2_bytes +
+             8 * (2 * A_STAGES + 2 * B_STAGES + 2) + 16;
     p.off_bterm = WS_STATUS_BYTES;
     p.off_xs = p.off_bterm + ((long long)B * 4 + 255) / 256 * 256;
     p.ws_bytes = p.off_xs + ((long long)B * p.Npad * 2 + 255) / 256 * 256;
@@ -513,21 +580,19 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (pl.splits > 1) {
+    if (pl.any_partial) {
         e = cudaMemsetAsync(out, 0, (size_t)B * L.M * 4, st);
         if (e != cudaSuccess) return e;
     }
     GemmParams P;
     P.L = L; P.out = out; P.B = B; P.Npad = pl.Npad;
-    P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.splits = pl.splits;
-    P.kb_total = pl.kb_total; P.kb_per_split = pl.kb_per_split;
+    P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.kb_total = pl.kb_total;
+    P.unit_gran = pl.unit_gran; P.units = pl.units;
     P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
     P.status = status; P.bterm = bterm;
     e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    const int units = pl.tiles_m * pl.tiles_t * pl.splits;
-    const int grid = units < sm_count() ? units : sm_count();
-    gemm_tcgen05_kernel<<<grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
+    gemm_tcgen05_kernel<<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
     return cudaGetLastError();
 }
 
