@@ -4,7 +4,12 @@
 
 namespace vptq {
 
-// codebooks in shared memory, ldmatrix gathers + mma.sync
+// codebooks in shared memory, LDS gathers + FP32 FMAs, up to 8 tokens per launch, no scratch
+bool smem_fma_supported(const LayerView &L, int B);
+int smem_fma_launches(const LayerView &L, int B);
+cudaError_t launch_decode_smem_fma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
+
+// codebooks in shared memory, ldmatrix gathers + mma.sync (per-output-row scale, all-outlier layers)
 bool smem_mma_supported(const LayerView &L, int B);
 cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
 

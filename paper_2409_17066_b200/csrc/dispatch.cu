@@ -15,6 +15,7 @@ LinearPath choose_path(const LayerView &L, int B, int flags)
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
     if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
     const int Bg = decode_group(B);
+    if (smem_fma_supported(L, Bg)) return PATH_DECODE_SMEM_FMA;
     if (smem_mma_supported(L, Bg)) return PATH_DECODE_SMEM_MMA;
     if (l2_fma_supported(L, Bg)) return PATH_DECODE_L2_FMA;
     return PATH_GENERIC;
@@ -23,6 +24,7 @@ LinearPath choose_path(const LayerView &L, int B, int flags)
 const char *linear_path_name(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_FMA: return "decode_smem_fma";
     case PATH_DECODE_SMEM_MMA: return "decode_smem_mma";
     case PATH_DECODE_L2_FMA: return "decode_l2_fma";
     case PATH_GEMM_TCGEN05: return "gemm_tcgen05";
@@ -33,6 +35,7 @@ const char *linear_path_name(const LayerView &L, int B, int flags)
 long long linear_workspace_bytes(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_FMA: return 0;
     case PATH_DECODE_SMEM_MMA: return 0;
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
@@ -45,6 +48,8 @@ int linear_launches(const LayerView &L, int B, int flags)
     const int groups = (B + DECODE_MAX_B - 1) / DECODE_MAX_B;
     const int last = B - (groups - 1) * DECODE_MAX_B;
     switch (choose_path(L, B, flags)) {
+    case PATH_DECODE_SMEM_FMA:
+        return (groups - 1) * smem_fma_launches(L, DECODE_MAX_B) + smem_fma_launches(L, last);
     case PATH_DECODE_SMEM_MMA: return groups;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_launches(L, B);
     case PATH_DECODE_L2_FMA:
@@ -69,7 +74,8 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
             const int Bg = (B - t0 < DECODE_MAX_B) ? (B - t0) : DECODE_MAX_B;
             const void *xg = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * 2;
             void *og = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
-            if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, st);
+            if (path == PATH_DECODE_SMEM_FMA) e = launch_decode_smem_fma(L, xg, Bg, og, st);
+            else if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, st);
             else e = launch_decode_l2_fma(L, xg, Bg, og, ws, st);
         }
     }

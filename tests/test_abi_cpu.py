@@ -85,5 +85,5 @@ def test_argument_errors_need_no_gpu(binding):
     p2 = b.LayerPtrs(0x1008, 0x1000, None, None, None, None, 0x1000, 0x1000)
     assert b.lib.vptq_dequant(C.byref(d), C.byref(p2), 0x1000, None) == b.E_ALIGN
     assert b.lib.vptq_status_string(b.E_ALIGN).decode().startswith("a data pointer")
-    assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_mma", "decode_l2_fma", "gemm_tcgen05")
+    assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_fma", "decode_smem_mma", "decode_l2_fma", "gemm_tcgen05")
     assert b.vptq_linear_launches(d, 1) >= 1
