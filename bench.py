@@ -48,7 +48,7 @@ def read_peaks():
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
 }
 
-ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
+ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
                    "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel"}
 
 
