@@ -59,31 +59,38 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Stage a codebook [k][v] fp16 (dense) into shared memory as [k][8] fp16, zero padded.
+// One centroid [v] fp16 (dense table, entry e) as a zero-padded 16-byte row.
+__device__ __forceinline__ uint4 padded_centroid_row(const __half *__restrict__ tab, int e, int v)
+{
+    if (v == 8) return __ldg(reinterpret_cast<const uint4 *>(tab) + e);
+    uint32_t w[4] = {0, 0, 0, 0};
+    if ((v & 1) == 0) {
+        const uint32_t *p = reinterpret_cast<const uint32_t *>(tab) + (long long)e * (v >> 1);   // tables are 16-byte aligned
+#pragma unroll
+        for (int i = 0; i < 4; i++)
+            if (i < (v >> 1)) w[i] = __ldg(p + i);
+    } else {
+        const uint16_t *p = reinterpret_cast<const uint16_t *>(tab) + (long long)e * v;
+#pragma unroll
+        for (int i = 0; i < 8; i++)
+            if (i < v) w[i >> 1] |= (uint32_t)__ldg(p + i) << (16 * (i & 1));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Stage a codebook [k][v] fp16 (dense) into shared memory as [k][8] fp16, zero padded.  The loads of
+// 4 entries are issued before the first store: one L2 round trip per 4 entries, not per entry.
 __device__ void stage_codebook(const __half *__restrict__ src, int k, int v, __half *dst)
 {
-    if (v == 8) {
-        const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
-        uint4 *d4 = reinterpret_cast<uint4 *>(dst);
-        for (int i = threadIdx.x; i < k; i += THREADS) d4[i] = __ldg(s4 + i);
-        return;
-    }
-    uint4 z = make_uint4(0, 0, 0, 0);
     uint4 *d4 = reinterpret_cast<uint4 *>(dst);
-    for (int i = threadIdx.x; i < k; i += THREADS) d4[i] = z;
-    __syncthreads();
-    const int total = k * v;
-    if ((total & 1) == 0) {
-        const uint32_t *s2 = reinterpret_cast<const uint32_t *>(src);   // codebooks are 16-byte aligned
-        for (int w = threadIdx.x; w < total / 2; w += THREADS) {
-            uint32_t two = __ldg(s2 + w);
-            int e0 = 2 * w, e1 = 2 * w + 1;
-            reinterpret_cast<uint16_t *>(dst)[(e0 / v) * 8 + (e0 % v)] = (uint16_t)(two & 0xFFFFu);
-            reinterpret_cast<uint16_t *>(dst)[(e1 / v) * 8 + (e1 % v)] = (uint16_t)(two >> 16);
-        }
-    } else {
-        for (int e = threadIdx.x; e < total; e += THREADS)
-            dst[(e / v) * 8 + (e % v)] = __ldg(src + e);
+    for (int e0 = threadIdx.x; e0 < k; e0 += 4 * THREADS) {
+        uint4 row[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+            if (e0 + u * THREADS < k) row[u] = padded_centroid_row(src, e0 + u * THREADS, v);
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+            if (e0 + u * THREADS < k) d4[e0 + u * THREADS] = row[u];
     }
 }
 
@@ -236,6 +243,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
 #pragma unroll
         for (int t = 0; t < TP; t++) acc[t] = 0.f;
         if (L.has_scale) {
+#pragma unroll 4
             for (int n = threadIdx.x; n < L.N; n += THREADS) {
                 float bn = L.scale_rows ? 1.f : __half2float(__ldg(L.bias + n));
 #pragma unroll

@@ -17,6 +17,12 @@
 // red.add), two per TMEM lane quarter.
 // A and B have rings of their own: A is deep (the producers' gathers need about a microsecond),
 // B holds 32 KB per stage and is shallow.
+// CTA pairs (CG = 2): two CTAs of a cluster work on one 256-row tile with tcgen05.mma.cta_group::2:
+// each dequantises its own 128 rows and loads half of the tokens of every 256-token MMA (no TMA
+// multicast), the even CTA issues the MMAs for both, accumulators sit in each CTA's own TMEM.
+// That halves the activation traffic from L2 and the shared-memory traffic per MMA.  All
+// barriers the issuing thread waits on live in the even CTA (the odd CTA arrives remotely);
+// tcgen05.commit multicasts to both CTAs.  CG = 1 keeps everything in one CTA.
 // Persistent grid, one CTA per SM.  The work is the list of (tile, k block) units, tile =
 // (token tile, 128-row tile); with an FP32 output every CTA takes an equal, contiguous share of
 // the units, whatever tile they fall in (partial tiles meet in the output by red.add), so all
@@ -39,13 +45,17 @@ constexpr int TILE_K = 32;
 constexpr int TILE_N = 512;
 constexpr int MMA_N = 256;
 constexpr int A_STAGES = 8;                              // ring of dequantised weight tiles
-constexpr int B_STAGES = 3;                              // ring of activation tiles
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;       // 8 KB
-constexpr int B_HALF_BYTES = MMA_N * TILE_K * 2;         // 16 KB
-constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;          // 32 KB
+// ring of activation tiles: per CTA and stage 2 halves x (256 / CG tokens) x 32 columns
+template <int CG> struct BRing {
+    static constexpr int HALF_BYTES = (MMA_N / CG) * TILE_K * 2;     // 16 KB / 8 KB
+    static constexpr int STAGE_BYTES = 2 * HALF_BYTES;               // 32 KB / 16 KB
+    static constexpr int STAGES = CG == 1 ? 3 : 6;                   // 96 KB either way
+};
 constexpr int PAIRS = 4;                                 // producer warp pairs; pair p fills k blocks p, p+PAIRS, ...
 constexpr int PRODUCER_WARPS = 2 * PAIRS;
 constexpr int EPI_WARPS = 8;
+static_assert(A_STAGES >= PAIRS, "a producer pair needs a stage of its own");
 constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 448
 constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
 constexpr int A_LBO = 1024;   // bytes between the two 64-row blocks of the A stage
@@ -129,19 +139,78 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
 }
 constexpr uint32_t LAYOUT_SW128 = 2, LAYOUT_SW64 = 4;
 
-// kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128, N = 256
-constexpr uint32_t IDESC = (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
-                           ((uint32_t)(MMA_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+// kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128 * CG, N = 256
+template <int CG>
+__device__ __forceinline__ constexpr uint32_t idesc()
+{
+    return (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
+           ((uint32_t)(MMA_N >> 3) << 17) | ((uint32_t)((TILE_M * CG) >> 4) << 24);
+}
 
+template <int CG>
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate) : "memory");
+    if (CG == 1)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc<1>()), "r"(accumulate) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc<2>()), "r"(accumulate) : "memory");
 }
+// The MMAs of one 32-column k block: two k16 steps x one or two 256-token halves, issued back to back.
+// `ad`/`bd` describe the k16 = 0 slice of the stage; the second slice lies 2 * A_SBO (A) and 32 bytes (B)
+// further, the second token half b_half_bytes further (descriptor address units are 16 bytes).
+template <int CG>
+__device__ __forceinline__ void umma_kblock(uint32_t d_tmem, uint64_t ad, uint64_t bd, uint32_t accumulate,
+                                            bool two_halves, int b_half_bytes)
+{
+    const uint64_t ad1 = ad + (uint64_t)((2 * A_SBO) >> 4);
+    const uint64_t bd1 = bd + 2u;
+    const uint64_t bh = (uint64_t)(b_half_bytes >> 4);
+    umma_f16<CG>(d_tmem, ad, bd, accumulate);
+    if (two_halves) umma_f16<CG>(d_tmem + MMA_N, ad, bd + bh, accumulate);
+    umma_f16<CG>(d_tmem, ad1, bd1, 1u);
+    if (two_halves) umma_f16<CG>(d_tmem + MMA_N, ad1, bd1 + bh, 1u);
+}
+// Arrive on the barrier once all MMAs issued so far have completed; with CG = 2 the arrival goes
+// to the barrier at the same offset in both CTAs of the pair.
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CG == 1)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+// CG = 2: the copy lands in this CTA's shared memory and signals the barrier `bar` of the even CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -192,9 +261,14 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
 }
 
 // ---- the GEMM ------------------------------------------------------------------------------------
+template <int CG>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
 {
+    constexpr int B_STAGES = BRing<CG>::STAGES;
+    constexpr int B_STAGE_BYTES = BRing<CG>::STAGE_BYTES;
+    constexpr int B_HALF_BYTES = BRing<CG>::HALF_BYTES;
+    constexpr int TILE_ROWS = TILE_M * CG;                   // output rows of a tile
     extern __shared__ uint8_t smem_raw[];
     const LayerView &L = P.L;
     // carve shared memory; swizzled operand stages need 1024-byte alignment
@@ -202,7 +276,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const uint32_t sA = base;                                   // A_STAGES x 8 KB
-    const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x 32 KB
+    const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x (32 / CG) KB
     uint8_t *cb2_ptr = sm + A_STAGES * A_STAGE_BYTES + B_STAGES * B_STAGE_BYTES;
     uint8_t *misc = cb2_ptr + P.cb2_bytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(misc);   // fullA[] emptyA[] fullB[] emptyB[] accum_full accum_empty
@@ -218,24 +292,33 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // CG = 2: rank of this CTA in its pair; the even CTA (rank 0) issues the MMAs and owns the
+    // barriers the issuing thread waits on (fullA, fullB, accum_empty)
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < A_STAGES; s++) {
-            mbar_init(bar_fullA(s), 2);       // one arrival per producer warp of a pair
+            mbar_init(bar_fullA(s), 2 * CG);  // one arrival per producer warp of a pair, from every CTA
             mbar_init(bar_emptyA(s), 1);      // tcgen05.commit
         }
         for (int s = 0; s < B_STAGES; s++) {
-            mbar_init(bar_fullB(s), 1);       // the TMA thread's expect_tx arrival
+            mbar_init(bar_fullB(s), 1);       // the leader's expect_tx arrival
             mbar_init(bar_emptyB(s), 1);      // tcgen05.commit
         }
         mbar_init(bar_accum_full, 1);
-        mbar_init(bar_accum_empty, EPI_WARPS);
+        mbar_init(bar_accum_empty, EPI_WARPS * CG);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CG == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     // residual codebook -> shared memory (all threads)
     if (L.k2) {
@@ -249,13 +332,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anybody arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // this CTA's share of the (tile, k block) units: [u_begin, u_end), boundaries multiples of unit_gran
+    // the barriers of the even CTA, as this CTA addresses them
+    auto leader_bar = [&](uint32_t bar) { return CG == 2 ? map_to_cta(bar, 0) : bar; };
+
+    // this worker's share of the (tile, k block) units: [u_begin, u_end), boundaries multiples of
+    // unit_gran; a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
+    const long long n_workers = gridDim.x / CG, worker = blockIdx.x / CG;
     const long long groups = P.units / P.unit_gran;
-    const long long u_begin = groups * blockIdx.x / gridDim.x * P.unit_gran;
-    const long long u_end = groups * (blockIdx.x + 1) / gridDim.x * P.unit_gran;
+    const long long u_begin = groups * worker / n_workers * P.unit_gran;
+    const long long u_end = groups * (worker + 1) / n_workers * P.unit_gran;
     // A segment is the part of one tile inside the share: k blocks [kb0, kb1) of tile `tile`.
 #define FOR_EACH_SEGMENT                                                                          \
     for (long long u = u_begin; u < u_end && ok; u += kb1 - kb0)                                    \
@@ -265,23 +354,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     bool ok = true;
 
     if (warp == 0) {
-        // ================= TMA: B tiles =================
+        // ================= TMA: B tiles (every CTA loads its own share of the tokens) =================
         if (lane == 0) {
             int it = 0;
+            uint32_t s = 0, ps = 1;                              // ring position, parity to wait for
             FOR_EACH_SEGMENT {
                 const int tt = tile / P.tiles_m;
                 const int t0 = tt * TILE_N;
                 const int halves = (P.B - t0 > MMA_N) ? 2 : 1;
-                for (int kb = kb0; kb < kb1; kb++, it++) {
-                    const int s = it % B_STAGES;
-                    if (!(ok = mbar_wait(bar_emptyB(s), ((it / B_STAGES) & 1) ^ 1, abort_flag, P.status))) break;
-                    mbar_expect_tx(bar_fullB(s), halves * B_HALF_BYTES);
-                    for (int h = 0; h < halves; h++)
-                        tma_load_2d(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES, &tmap_xs, bar_fullB(s),
-                                    kb * TILE_K, t0 + h * MMA_N);
+                for (int kb = kb0; kb < kb1; kb++, it++, s = (s + 1 == B_STAGES ? 0 : s + 1), ps ^= (s == 0 ? 1u : 0u)) {
+                    if (!(ok = mbar_wait(bar_emptyB(s), ps, abort_flag, P.status))) break;
+                    if (leader) mbar_expect_tx(bar_fullB(s), CG * halves * B_HALF_BYTES);
+                    for (int h = 0; h < halves; h++) {
+                        const uint32_t dst = sB + s * B_STAGE_BYTES + h * B_HALF_BYTES;
+                        const int tok = t0 + h * MMA_N + (int)rank * (MMA_N / CG);
+                        if (CG == 1) tma_load_2d(dst, &tmap_xs, bar_fullB(s), kb * TILE_K, tok);
+                        else tma_load_2d_pair(dst, &tmap_xs, leader_bar(bar_fullB(s)), kb * TILE_K, tok);
+                    }
                 }
             }
-            if (!ok) {
+            if (!ok && CG == 1) {
                 // abandoned: give copies still in flight a bounded time to land before the CTA exits
                 const int first = it > B_STAGES ? it - B_STAGES : 0;
                 for (int j = first; j < it; j++) {
@@ -291,39 +383,39 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issue =================
-        if (lane == 0) {
-            int it = 0, seg_no = 0;
+        // ================= MMA issue (the even CTA issues for the pair) =================
+        if (lane == 0 && leader) {
+            // One thread runs this loop as a serial instruction chain, so it is kept short: descriptors
+            // are a constant plus a stage offset, stage numbers and parities are running counters, and the
+            // MMAs of a k block go out in one asm block.
+            const uint64_t adesc0 = make_smem_desc(sA, A_LBO, A_SBO, LAYOUT_SW128);
+            const uint64_t bdesc0 = make_smem_desc(sB, 16, B_SBO, LAYOUT_SW64);
+            uint32_t sa = 0, pa = 0, sb = 0, pb = 0;          // ring positions and their phase parities
+            int seg_no = 0;
             FOR_EACH_SEGMENT {
                 const int tt = tile / P.tiles_m;
-                const int halves = (P.B - tt * TILE_N > MMA_N) ? 2 : 1;
-                // the accumulator must have been drained by the epilogue of the previous segment
+                const bool two_halves = P.B - tt * TILE_N > MMA_N;
+                // the accumulators must have been drained by the epilogues of the previous segment
                 if (!(ok = mbar_wait(bar_accum_empty, (seg_no & 1) ^ 1, abort_flag, P.status))) break;
                 tc_fence_after();
-                for (int kb = kb0; kb < kb1; kb++, it++) {
-                    const int sa = it % A_STAGES, sb = it % B_STAGES;
-                    if (!(ok = mbar_wait(bar_fullA(sa), (it / A_STAGES) & 1, abort_flag, P.status))) break;
-                    if (!(ok = mbar_wait(bar_fullB(sb), (it / B_STAGES) & 1, abort_flag, P.status))) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k16 = 0; k16 < TILE_K / 16; k16++) {
-                        const uint64_t adesc = make_smem_desc(sA + sa * A_STAGE_BYTES + k16 * 2 * A_SBO,
-                                                              A_LBO, A_SBO, LAYOUT_SW128);
-                        for (int h = 0; h < halves; h++) {
-                            const uint64_t bdesc = make_smem_desc(sB + sb * B_STAGE_BYTES + h * B_HALF_BYTES + k16 * 32,
-                                                                  16, B_SBO, LAYOUT_SW64);
-                            umma_f16(tmem_base + h * MMA_N, adesc, bdesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
-                        }
-                    }
-                    umma_commit(bar_emptyA(sa));      // the stages may be refilled once these MMAs have read them
-                    umma_commit(bar_emptyB(sb));
+                for (int kb = kb0; kb < kb1; kb++) {
+                    if (!(ok = mbar_wait(bar_fullA(sa), pa, abort_flag, P.status))) break;
+                    if (!(ok = mbar_wait(bar_fullB(sb), pb, abort_flag, P.status))) break;
+                    // (stage offsets only touch the 14-bit address field of the descriptors: no carry)
+                    const uint64_t ad = adesc0 + (uint64_t)((sa * A_STAGE_BYTES) >> 4);
+                    const uint64_t bd = bdesc0 + (uint64_t)((sb * B_STAGE_BYTES) >> 4);
+                    umma_kblock<CG>(tmem_base, ad, bd, kb > kb0 ? 1u : 0u, two_halves, B_HALF_BYTES);
+                    umma_commit<CG>(bar_emptyA(sa));      // the stages may be refilled once these MMAs have read them
+                    umma_commit<CG>(bar_emptyB(sb));
+                    if (++sa == A_STAGES) { sa = 0; pa ^= 1u; }
+                    if (++sb == B_STAGES) { sb = 0; pb ^= 1u; }
                 }
-                if (ok) umma_commit(bar_accum_full);  // accumulator complete
+                if (ok) umma_commit<CG>(bar_accum_full);  // accumulators complete
                 seg_no++;
             }
         }
     } else if (warp < 2 + PRODUCER_WARPS) {
-        // ================= dequant producers: A tiles =================
+        // ================= dequant producers: A tiles (every CTA its own 128 rows) =================
         const int pw = warp - 2, pair = pw >> 1, half = pw & 1;
         const int c = lane & 7, grp = lane >> 3;             // row chunk within the 64-row block, 8-column group
         const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
@@ -333,7 +425,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         int it0 = 0;                                         // k blocks of earlier segments
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m;
-            const int vrow = mt * (TILE_M / 8) + 8 * half + c;
+            const int vrow = mt * (TILE_ROWS / 8) + (int)rank * (TILE_M / 8) + 8 * half + c;
             const bool row_ok = vrow < L.R;
             const uint8_t *row1 = L.s1.ptr + (long long)vrow * L.s1.stride;
             const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)vrow * L.s2.stride : nullptr;
@@ -392,7 +484,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_fullA(s));
+                if (lane == 0) {
+                    if (CG == 1) mbar_arrive(bar_fullA(s));
+                    else mbar_arrive_cluster(leader_bar(bar_fullA(s)));
+                }
             }
             it0 += kb1 - kb0;
         }
@@ -406,7 +501,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m, tt = tile / P.tiles_m;
             const int t0 = tt * TILE_N;
-            const int m = mt * TILE_M + 32 * q + lane;
+            const int m = mt * TILE_ROWS + (int)rank * TILE_M + 32 * q + lane;
             const int t_cnt = min(TILE_N, P.B - t0);
             const bool partial = kb0 != 0 || kb1 != P.kb_total;
             // bias terms of this warp's 256 tokens, loaded before the wait (a load inside the drain would
@@ -461,19 +556,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_accum_empty);
+            if (lane == 0) {
+                if (CG == 1) mbar_arrive(bar_accum_empty);
+                else mbar_arrive_cluster(leader_bar(bar_accum_empty));
+            }
             seg_no++;
         }
     }
 #undef FOR_EACH_SEGMENT
 
-    // ---- teardown: everybody meets, then the allocating warp frees TMEM ------------------------------
+    // ---- teardown: everybody (of both CTAs) meets, then the allocating warps free TMEM ---------------
     tc_fence_before();
+    __syncwarp();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();          // nobody leaves while its pair may still reach into it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
     }
 }
 
@@ -497,6 +598,7 @@ EncodeTiledFn get_encode_fn()
 }
 
 struct GemmPlan {
+    int cg;              // CTAs per tile: 2 = CTA pairs (tcgen05 cta_group::2), 1 = single CTAs
     int Npad, tiles_m, tiles_t, kb_total, unit_gran, grid, any_partial, cb2_rep, cb2_bytes;
     long long units;
     size_t smem;
@@ -515,26 +617,64 @@ int sm_count()
     return n;
 }
 
-GemmPlan plan_gemm(const LayerView &L, int B)
+template <int CG>
+size_t gemm_smem_bytes(int cb2_bytes)
+{
+    return 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)BRing<CG>::STAGES * BRing<CG>::STAGE_BYTES + cb2_bytes +
+           8 * (2 * A_STAGES + 2 * BRing<CG>::STAGES + 2) + 16;
+}
+
+// How many CTA pairs of the cta_group::2 kernel the device runs at once (0: cannot).  Asked once.
+int max_active_pairs(int cb2_bytes)
+{
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * sm_count(), 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = gemm_smem_bytes<2>(cb2_bytes > 0 ? cb2_bytes : 32768);
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(gemm_tcgen05_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)cfg.dynamicSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<2>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    cached = n;
+    return cached;
+}
+
+GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
 {
     GemmPlan p;
+    const int G = sm_count();
+    p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
+    p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
+    // CTA pairs when the device runs (nearly) all its SMs as pairs and the layer has rows for them
+    p.cg = 1;
+    int workers = G;
+    if (query_device && L.M > TILE_M) {
+        const int pairs = max_active_pairs(p.cb2_bytes);
+        if (2 * pairs >= G - 8) { p.cg = 2; workers = pairs; }
+    }
     p.Npad = (L.N + 7) / 8 * 8;
-    p.tiles_m = ceil_div(L.M, TILE_M);
+    p.tiles_m = ceil_div(L.M, TILE_M * p.cg);
     p.tiles_t = ceil_div(B, TILE_N);
     p.kb_total = ceil_div(L.N, TILE_K);
     p.units = (long long)p.tiles_m * p.tiles_t * p.kb_total;
     // partial tiles meet in an FP32 output by red.add; other output types get whole tiles
     p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32) ? 1 : p.kb_total;
     const long long groups = p.units / p.unit_gran;
-    const int G = sm_count();
-    p.grid = (int)(groups < G ? groups : G);
+    if (groups < workers) workers = (int)groups;
+    p.grid = workers * p.cg;
     p.any_partial = 0;
-    for (int c = 1; c < p.grid; c++)
-        if ((groups * c / p.grid * p.unit_gran) % p.kb_total != 0) p.any_partial = 1;
-    p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
-    p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
-    p.smem = 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)B_STAGES * B_STAGE_BYTES + p.cb2_bytes +
-             8 * (2 * A_STAGES + 2 * B_STAGES + 2) + 16;
+    for (int c = 1; c < workers; c++)
+        if ((groups * c / workers * p.unit_gran) % p.kb_total != 0) p.any_partial = 1;
+    p.smem = p.cg == 2 ? gemm_smem_bytes<2>(p.cb2_bytes) : gemm_smem_bytes<1>(p.cb2_bytes);
     p.off_bterm = WS_STATUS_BYTES;
     p.off_xs = p.off_bterm + ((long long)B * 4 + 255) / 256 * 256;
     p.ws_bytes = p.off_xs + ((long long)B * p.Npad * 2 + 255) / 256 * 256;
@@ -552,13 +692,14 @@ bool gemm_tcgen05_supported(const LayerView &L, int B)
     return true;
 }
 
-long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B).ws_bytes; }
+// (the scratch layout does not depend on the device, so this query makes no CUDA call)
+long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B, false).ws_bytes; }
 
 int gemm_tcgen05_launches(const LayerView &, int) { return 2; }   // pre-pass + GEMM
 
 cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
 {
-    const GemmPlan pl = plan_gemm(L, B);
+    const GemmPlan pl = plan_gemm(L, B, true);
     uint8_t *w8 = reinterpret_cast<uint8_t *>(ws);
     int *status = reinterpret_cast<int *>(w8);
     float *bterm = reinterpret_cast<float *>(w8 + pl.off_bterm);
@@ -569,7 +710,7 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     CUtensorMap tmap;
     const cuuint64_t gdim[2] = {(cuuint64_t)L.N, (cuuint64_t)B};
     const cuuint64_t gstride[1] = {(cuuint64_t)pl.Npad * 2};
-    const cuuint32_t box[2] = {TILE_K, MMA_N};
+    const cuuint32_t box[2] = {TILE_K, (cuuint32_t)(MMA_N / pl.cg)};    // a CTA of a pair loads half the tokens of an MMA
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, xs, gdim, gstride, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
@@ -590,10 +731,24 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     P.unit_gran = pl.unit_gran; P.units = pl.units;
     P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
     P.status = status; P.bterm = bterm;
-    e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (pl.cg == 1) {
+        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+        if (e != cudaSuccess) return e;
+        gemm_tcgen05_kernel<1><<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
+        return cudaGetLastError();
+    }
+    e = cudaFuncSetAttribute(gemm_tcgen05_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    gemm_tcgen05_kernel<<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(pl.grid, 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<2>, tmap, P);
 }
 
 }  // namespace vptq
