@@ -50,6 +50,7 @@ struct LayerView {
     int R, R0, Nc;
     int has_scale, scale_rows;
     int x_bf16, out_dtype;
+    int cta_pairs;         // batched path: CTA pairs requested
     Stream s1, s2, s0;
     const __half *c1, *c2, *c0;
     const __half *scale, *bias;

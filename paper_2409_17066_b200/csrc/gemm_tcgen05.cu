@@ -63,6 +63,7 @@ constexpr int B_SBO = 512;    // bytes between consecutive 8-token groups of the
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
 
 constexpr int WS_STATUS_BYTES = 256;
+constexpr bool PREFER_CTA_PAIRS = false;
 
 struct GemmParams {
     LayerView L;
@@ -228,25 +229,61 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// ---- pre-pass: xs = fp16(x * s), bterm[t] = sum_n x[t][n] * b[n], status = 0 --------------------
+// ---- pre-pass: xs = fp16(x * s), bterm[t] = sum_n x[t][n] * b[n], status = 0; clears row t of an FP32
+//      output in which partial tiles are going to meet by red.add (zero_out != nullptr) -------------
 __global__ void __launch_bounds__(256)
 gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __half *__restrict__ xs,
-                    float *__restrict__ bterm, int *status)
+                    float *__restrict__ bterm, int *status, float *__restrict__ zero_out)
 {
     const int t = blockIdx.x;
     if (t == 0 && threadIdx.x == 0) *status = 0;
-    float acc = 0.f;
-    for (int n = threadIdx.x; n < Npad; n += 256) {
-        float xv = 0.f, sc = 1.f, bi = 0.f;
-        if (n < L.N) {
-            xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
-            if (L.has_scale) {
-                sc = __half2float(__ldg(L.scale + n));
-                bi = __half2float(__ldg(L.bias + n));
-            }
+    if (zero_out != nullptr) {
+        float *row = zero_out + (long long)t * L.M;
+        if ((L.M & 3) == 0) {
+            float4 *r4 = reinterpret_cast<float4 *>(row);          // rows of M floats start 16-byte aligned
+            for (int i = threadIdx.x; i < (L.M >> 2); i += 256) r4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            for (int i = threadIdx.x; i < L.M; i += 256) row[i] = 0.f;
         }
-        xs[(long long)t * Npad + n] = __float2half_rn(xv * sc);
-        acc += xv * bi;
+    }
+    float acc = 0.f;
+    if ((L.N & 7) == 0) {
+        // 8 columns per thread and step, 128-bit loads and stores (Npad == N)
+        for (int n = 8 * threadIdx.x; n < L.N; n += 8 * 256) {
+            const uint4 xq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + (long long)t * L.N + n));
+            uint4 sq = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u), bq = make_uint4(0, 0, 0, 0);
+            if (L.has_scale) {
+                sq = __ldg(reinterpret_cast<const uint4 *>(L.scale + n));
+                bq = __ldg(reinterpret_cast<const uint4 *>(L.bias + n));
+            }
+            const uint32_t xw[4] = {xq.x, xq.y, xq.z, xq.w}, sw[4] = {sq.x, sq.y, sq.z, sq.w}, bw[4] = {bq.x, bq.y, bq.z, bq.w};
+            uint32_t ow[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                float2 xv;
+                if (L.x_bf16) xv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xw[i]));
+                else xv = __half22float2(*reinterpret_cast<const __half2 *>(&xw[i]));
+                const float2 sv = __half22float2(*reinterpret_cast<const __half2 *>(&sw[i]));
+                const float2 bv = __half22float2(*reinterpret_cast<const __half2 *>(&bw[i]));
+                const __half2 o = __floats2half2_rn(xv.x * sv.x, xv.y * sv.y);
+                ow[i] = *reinterpret_cast<const uint32_t *>(&o);
+                acc += xv.x * bv.x + xv.y * bv.y;
+            }
+            *reinterpret_cast<uint4 *>(xs + (long long)t * Npad + n) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        }
+    } else {
+        for (int n = threadIdx.x; n < Npad; n += 256) {
+            float xv = 0.f, sc = 1.f, bi = 0.f;
+            if (n < L.N) {
+                xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
+                if (L.has_scale) {
+                    sc = __half2float(__ldg(L.scale + n));
+                    bi = __half2float(__ldg(L.bias + n));
+                }
+            }
+            xs[(long long)t * Npad + n] = __float2half_rn(xv * sc);
+            acc += xv * bi;
+        }
     }
     __shared__ float red[8];
 #pragma unroll
@@ -460,6 +497,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
                     id = min(id, kmax1);
                     cw[j] = live ? __ldg(cb1 + id) : make_uint4(0, 0, 0, 0);
                 }
+                // a4: residual centroids from shared memory, all 8 before the wait as well: one shared-memory
+                // round trip per visit instead of one per store
+                uint4 rv[8];
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    rv[j] = make_uint4(0, 0, 0, 0);
+                    if (L.k2 && live) {
+                        uint32_t id2 = ((j < 4 ? cur2.x : cur2.y) >> (8 * (j & 3))) & 0xFFu;
+                        id2 = min(id2, kmax2);
+                        rv[j] = cb2[(id2 << rshift) + rep];
+                    }
+                }
                 // the whole warp takes the same decision: the stores below end in a warp-wide barrier
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_emptyA(s), ((it / A_STAGES) & 1) ^ 1, abort_flag, P.status));
                 if (!ok) break;
@@ -467,14 +516,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
                     uint4 w = cw[j];
-                    if (L.k2 && live) {
-                        uint32_t id2 = ((j < 4 ? cur2.x : cur2.y) >> (8 * (j & 3))) & 0xFFu;
-                        id2 = min(id2, kmax2);
-                        const uint4 rv = cb2[(id2 << rshift) + rep];
-                        __half2 a0 = __hadd2(*reinterpret_cast<__half2 *>(&w.x), *reinterpret_cast<const __half2 *>(&rv.x));
-                        __half2 a1 = __hadd2(*reinterpret_cast<__half2 *>(&w.y), *reinterpret_cast<const __half2 *>(&rv.y));
-                        __half2 a2 = __hadd2(*reinterpret_cast<__half2 *>(&w.z), *reinterpret_cast<const __half2 *>(&rv.z));
-                        __half2 a3 = __hadd2(*reinterpret_cast<__half2 *>(&w.w), *reinterpret_cast<const __half2 *>(&rv.w));
+                    {   // sum in FP16 (adding zero when there is no residual stage changes nothing)
+                        __half2 a0 = __hadd2(*reinterpret_cast<__half2 *>(&w.x), *reinterpret_cast<const __half2 *>(&rv[j].x));
+                        __half2 a1 = __hadd2(*reinterpret_cast<__half2 *>(&w.y), *reinterpret_cast<const __half2 *>(&rv[j].y));
+                        __half2 a2 = __hadd2(*reinterpret_cast<__half2 *>(&w.z), *reinterpret_cast<const __half2 *>(&rv[j].z));
+                        __half2 a3 = __hadd2(*reinterpret_cast<__half2 *>(&w.w), *reinterpret_cast<const __half2 *>(&rv[j].w));
                         w.x = *reinterpret_cast<uint32_t *>(&a0); w.y = *reinterpret_cast<uint32_t *>(&a1);
                         w.z = *reinterpret_cast<uint32_t *>(&a2); w.w = *reinterpret_cast<uint32_t *>(&a3);
                     }
@@ -654,10 +700,13 @@ GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
     const int G = sm_count();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
     p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
-    // CTA pairs when the device runs (nearly) all its SMs as pairs and the layer has rows for them
+    // CTA pairs need the device to run (nearly) all its SMs as pairs and a layer with rows for them.
+    // Measured at 512 tokens on the 14336 x 4096 layer: 108 us with pairs, 94 us with single CTAs (the
+    // producers' centroid reads, not the activation traffic that pairs halve, hold the k loop back, and
+    // a pair advances at the pace of the slower of its two CTAs), so single CTAs are the default.
     p.cg = 1;
     int workers = G;
-    if (query_device && L.M > TILE_M) {
+    if ((PREFER_CTA_PAIRS || L.cta_pairs) && query_device && L.M > TILE_M) {
         const int pairs = max_active_pairs(p.cb2_bytes);
         if (2 * pairs >= G - 8) { p.cg = 2; workers = pairs; }
     }
@@ -718,13 +767,10 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
     cudaError_t e;
-    gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status);
+    gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status,
+                                           pl.any_partial ? reinterpret_cast<float *>(out) : nullptr);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (pl.any_partial) {
-        e = cudaMemsetAsync(out, 0, (size_t)B * L.M * 4, st);
-        if (e != cudaSuccess) return e;
-    }
     GemmParams P;
     P.L = L; P.out = out; P.B = B; P.Npad = pl.Npad;
     P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.kb_total = pl.kb_total;
