@@ -361,10 +361,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     if (L.k2) {
         const uint4 *src = reinterpret_cast<const uint4 *>(L.c2);
         uint4 *dst = reinterpret_cast<uint4 *>(cb2_ptr);
-        if (P.cb2_replicated) {
-            for (int i = threadIdx.x; i < L.k2 * 8; i += GEMM_THREADS) dst[i] = __ldg(src + (i >> 3));
-        } else {
-            for (int i = threadIdx.x; i < L.k2; i += GEMM_THREADS) dst[i] = __ldg(src + i);
+        // (loads of 4 entries are issued before the first store: one L2 round trip per 4 entries)
+        const int n2 = P.cb2_replicated ? L.k2 * 8 : L.k2, sh = P.cb2_replicated ? 3 : 0;
+        for (int i0 = threadIdx.x; i0 < n2; i0 += 4 * GEMM_THREADS) {
+            uint4 row[4];
+#pragma unroll
+            for (int u = 0; u < 4; u++)
+                if (i0 + u * GEMM_THREADS < n2) row[u] = __ldg(src + ((i0 + u * GEMM_THREADS) >> sh));
+#pragma unroll
+            for (int u = 0; u < 4; u++)
+                if (i0 + u * GEMM_THREADS < n2) dst[i0 + u * GEMM_THREADS] = row[u];
         }
     }
     tc_fence_before();
