@@ -501,7 +501,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
                 for (int j = 0; j < 8; j++) {
                     uint32_t id = (w1[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
                     id = min(id, kmax1);
-                    cw[j] = live ? __ldg(cb1 + id) : make_uint4(0, 0, 0, 0);
+                    // (no L1 allocation: the tensor core's operand reads share the L1 data path)
+                    if (live) asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                           : "=r"(cw[j].x), "=r"(cw[j].y), "=r"(cw[j].z), "=r"(cw[j].w) : "l"(cb1 + id));
+                    else cw[j] = make_uint4(0, 0, 0, 0);
                 }
                 // a4: residual centroids from shared memory, all 8 before the wait as well: one shared-memory
                 // round trip per visit instead of one per store
