@@ -44,7 +44,7 @@ constexpr int TILE_M = 128;
 constexpr int TILE_K = 32;
 constexpr int TILE_N = 512;
 constexpr int MMA_N = 256;
-constexpr int A_STAGES = 8;                              // ring of dequantised weight tiles
+constexpr int A_STAGES = 6;                              // ring of dequantised weight tiles
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;       // 8 KB
 // ring of activation tiles: per CTA and stage 2 halves x (256 / CG tokens) x 32 columns
 template <int CG> struct BRing {
@@ -55,6 +55,9 @@ template <int CG> struct BRing {
 constexpr int PAIRS = 4;                                 // producer warp pairs; pair p fills k blocks p, p+PAIRS, ...
 constexpr int PRODUCER_WARPS = 2 * PAIRS;
 constexpr int EPI_WARPS = 8;
+constexpr int EPI_BUF_BYTES = 16 * 32 * 4;                // one staged piece of the output: 16 tokens x 32 rows, FP32
+constexpr int EPI_STAGE_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;   // two buffers per epilogue warp: 32 KB
+constexpr int CB2_REPLICAS = 4;                          // copies of a small residual table (16-byte skew)
 static_assert(A_STAGES >= PAIRS, "a producer pair needs a stage of its own");
 constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 448
 constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
@@ -75,6 +78,7 @@ struct GemmParams {
     long long units;     // tiles_m * tiles_t * kb_total
     int cb2_replicated;
     int cb2_bytes;
+    int tma_out;         // FP32 output written by TMA store / reduce from shared memory (needs M % 4 == 0)
     int *status;         // workspace status word
     const float *bterm;  // [B]
 };
@@ -229,6 +233,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// TMA store / reduce-add of a [16 tokens][32 rows] FP32 box from shared memory into the output
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y, bool add)
+{
+    if (add)
+        asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+                     ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                     ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
 // ---- pre-pass: xs = fp16(x * s), bterm[t] = sum_n x[t][n] * b[n], status = 0; clears row t of an FP32
 //      output in which partial tiles are going to meet by red.add (zero_out != nullptr) -------------
 __global__ void __launch_bounds__(256)
@@ -300,7 +325,7 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
 // ---- the GEMM ------------------------------------------------------------------------------------
 template <int CG>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
 {
     constexpr int B_STAGES = BRing<CG>::STAGES;
     constexpr int B_STAGE_BYTES = BRing<CG>::STAGE_BYTES;
@@ -315,7 +340,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
     const uint32_t sA = base;                                   // A_STAGES x 8 KB
     const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x (32 / CG) KB
     uint8_t *cb2_ptr = sm + A_STAGES * A_STAGE_BYTES + B_STAGES * B_STAGE_BYTES;
-    uint8_t *misc = cb2_ptr + P.cb2_bytes;
+    const uint32_t sEpi = smem_addr(cb2_ptr + P.cb2_bytes);     // EPI_WARPS x 2 x 2 KB output staging
+    uint8_t *misc = cb2_ptr + P.cb2_bytes + EPI_STAGE_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(misc);   // fullA[] emptyA[] fullB[] emptyB[] accum_full accum_empty
     const uint32_t bar0 = smem_addr(bars);
     auto bar_fullA = [&](int s) { return bar0 + 8u * s; };
@@ -362,7 +388,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         const uint4 *src = reinterpret_cast<const uint4 *>(L.c2);
         uint4 *dst = reinterpret_cast<uint4 *>(cb2_ptr);
         // (loads of 4 entries are issued before the first store: one L2 round trip per 4 entries)
-        const int n2 = P.cb2_replicated ? L.k2 * 8 : L.k2, sh = P.cb2_replicated ? 3 : 0;
+        const int n2 = P.cb2_replicated ? L.k2 * CB2_REPLICAS : L.k2, sh = P.cb2_replicated ? 2 : 0;
         for (int i0 = threadIdx.x; i0 < n2; i0 += 4 * GEMM_THREADS) {
             uint4 row[4];
 #pragma unroll
@@ -463,7 +489,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         const int c = lane & 7, grp = lane >> 3;             // row chunk within the 64-row block, 8-column group
         const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
         const uint4 *cb2 = reinterpret_cast<const uint4 *>(cb2_ptr);
-        const int rep = P.cb2_replicated ? (lane & 7) : 0, rshift = P.cb2_replicated ? 3 : 0;
+        const int rep = P.cb2_replicated ? (lane & (CB2_REPLICAS - 1)) : 0, rshift = P.cb2_replicated ? 2 : 0;
         const uint32_t kmax1 = (uint32_t)(L.k1 - 1), kmax2 = L.k2 ? (uint32_t)(L.k2 - 1) : 0u;
         int it0 = 0;                                         // k blocks of earlier segments
         FOR_EACH_SEGMENT {
@@ -553,6 +579,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
         const bool fp32_out = L.out_dtype == VPTQ_DTYPE_FP32;
         const unsigned Mu = (unsigned)L.M;
         int seg_no = 0;
+        unsigned epi_piece = 0;                                  // staged pieces so far (buffer parity)
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m, tt = tile / P.tiles_m;
             const int t0 = tt * TILE_N;
@@ -570,6 +597,42 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
             ok = __all_sync(0xffffffffu, mbar_wait(bar_accum_full, seg_no & 1, abort_flag, P.status));
             if (!ok) break;
             tc_fence_after();
+            if (P.tma_out) {
+                // FP32 output through shared memory: per 16 tokens a warp stages its [16][32] piece (lane =
+                // output row: conflict free) and one lane hands it to TMA (store, or reduce-add for a partial
+                // tile); two staging buffers per warp, so the copy of one piece overlaps the next.
+                const uint32_t ebuf = sEpi + (uint32_t)(warp - (2 + PRODUCER_WARPS)) * (2 * EPI_BUF_BYTES);
+                const int m0 = mt * TILE_ROWS + (int)rank * TILE_M + 32 * q;
+#pragma unroll
+                for (int ci = 0; ci < MMA_N / 32; ci++) {    // unrolled: bt_chunk[] stays in registers
+                    const int c0 = h * MMA_N + 32 * ci;
+                    if (c0 >= t_cnt) break;
+                    const float bt_lane = bt_chunk[ci];
+#pragma unroll
+                    for (int hh = 0; hh < 2; hh++) {
+                        const int c1 = c0 + 16 * hh;
+                        if (c1 >= t_cnt) break;
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c1, r);
+                        if (kb0 == 0) {
+#pragma unroll
+                            for (int j = 0; j < 16; j++)
+                                r[j] = __float_as_uint(__uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bt_lane, 16 * hh + j));
+                        }
+                        // the buffer written two pieces ago must have been read by its copy
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        __syncwarp();
+                        const uint32_t buf = ebuf + (uint32_t)(epi_piece & 1) * EPI_BUF_BYTES;
+#pragma unroll
+                        for (int j = 0; j < 16; j++)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + j * 128u + lane * 4u), "r"(r[j]) : "memory");
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0 && m0 < L.M) tma_store_2d(&tmap_out, buf, m0, t0 + c1, partial);
+                        epi_piece++;
+                    }
+                }
+            } else
 #pragma unroll
             for (int ci = 0; ci < MMA_N / 32; ci++) {        // unrolled: bt_chunk[] stays in registers
                 const int c0 = h * MMA_N + 32 * ci;
@@ -617,6 +680,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, GemmParams P)
             }
             seg_no++;
         }
+        // the staging buffers must outlive the copies that read them, the copies must land before the end
+        if (P.tma_out && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 #undef FOR_EACH_SEGMENT
 
@@ -676,7 +741,7 @@ template <int CG>
 size_t gemm_smem_bytes(int cb2_bytes)
 {
     return 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)BRing<CG>::STAGES * BRing<CG>::STAGE_BYTES + cb2_bytes +
-           8 * (2 * A_STAGES + 2 * BRing<CG>::STAGES + 2) + 16;
+           EPI_STAGE_BYTES + 8 * (2 * A_STAGES + 2 * BRing<CG>::STAGES + 2) + 16;
 }
 
 // How many CTA pairs of the cta_group::2 kernel the device runs at once (0: cannot).  Asked once.
@@ -708,7 +773,7 @@ GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
     GemmPlan p;
     const int G = sm_count();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
-    p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? 8 : 1) : 0;
+    p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? CB2_REPLICAS : 1) : 0;
     // CTA pairs need the device to run (nearly) all its SMs as pairs and a layer with rows for them.
     // Measured at 512 tokens on the 14336 x 4096 layer: 108 us with pairs, 94 us with single CTAs (the
     // producers' centroid reads, not the activation traffic that pairs halve, hold the k loop back, and
@@ -775,6 +840,19 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
                         CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
+    // FP32 output with 16-byte aligned rows: the epilogue goes through shared memory and TMA
+    const int tma_out = (L.out_dtype == VPTQ_DTYPE_FP32 && (L.M & 3) == 0) ? 1 : 0;
+    CUtensorMap tmap_out = tmap;                 // placeholder when unused
+    if (tma_out) {
+        const cuuint64_t odim[2] = {(cuuint64_t)L.M, (cuuint64_t)B};
+        const cuuint64_t ostride[1] = {(cuuint64_t)L.M * 4};
+        const cuuint32_t obox[2] = {32, 16};
+        r = encode(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odim, ostride, obox, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+
     cudaError_t e;
     gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status,
                                            pl.any_partial ? reinterpret_cast<float *>(out) : nullptr);
@@ -785,11 +863,11 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.kb_total = pl.kb_total;
     P.unit_gran = pl.unit_gran; P.units = pl.units;
     P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
-    P.status = status; P.bterm = bterm;
+    P.status = status; P.bterm = bterm; P.tma_out = tma_out;
     if (pl.cg == 1) {
         e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
         if (e != cudaSuccess) return e;
-        gemm_tcgen05_kernel<1><<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, P);
+        gemm_tcgen05_kernel<1><<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, tmap_out, P);
         return cudaGetLastError();
     }
     e = cudaFuncSetAttribute(gemm_tcgen05_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
@@ -803,7 +881,7 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = st;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<2>, tmap, P);
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<2>, tmap, tmap_out, P);
 }
 
 }  // namespace vptq
