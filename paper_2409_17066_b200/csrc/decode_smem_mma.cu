@@ -310,20 +310,28 @@ decode_smem_mma_kernel(SmemMmaParams P)
             const int grp = cb / 8 + lane;         // this lane's index group within a packed row
             const uint8_t *row1 = L.s1.ptr + (long long)p0 * L.s1.stride;
             const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)p0 * L.s2.stride : nullptr;
-            uint4 raw1 = load_raw8(row1, L.s1.stride, grp, L.Nc, L.s1.bits);
-            uint4 raw2 = make_uint4(0, 0, 0, 0);
-            if (L.k2) raw2 = load_raw8(row2, L.s2.stride, grp, L.Nc, L.s2.bits);
+            // packed indices of the next PF rows are kept in flight: one row of compute is far shorter than
+            // a DRAM round trip
+            constexpr int PF = NT == 1 ? 4 : 1;          // 16 tokens leave no registers for more
+            uint4 pre1[PF], pre2[PF];
+#pragma unroll
+            for (int i = 0; i < PF; i++) {
+                pre1[i] = make_uint4(0, 0, 0, 0);
+                pre2[i] = make_uint4(0, 0, 0, 0);
+                if (i < nrows) {
+                    pre1[i] = load_raw8(row1 + (long long)i * L.s1.stride, L.s1.stride, grp, L.Nc, L.s1.bits);
+                    if (L.k2) pre2[i] = load_raw8(row2 + (long long)i * L.s2.stride, L.s2.stride, grp, L.Nc, L.s2.bits);
+                }
+            }
             for (int rl = 0; rl < nrows; rl++) {
                 uint32_t w1[4], w2[4];
-                decode8(raw1, L.s1.bits, L.k1, w1);
-                if (L.k2) decode8(raw2, L.s2.bits, L.k2, w2);
-                if (rl + 1 < nrows) {     // prefetch the next row's indices
-                    row1 += L.s1.stride;
-                    raw1 = load_raw8(row1, L.s1.stride, grp, L.Nc, L.s1.bits);
-                    if (L.k2) {
-                        row2 += L.s2.stride;
-                        raw2 = load_raw8(row2, L.s2.stride, grp, L.Nc, L.s2.bits);
-                    }
+                decode8(pre1[0], L.s1.bits, L.k1, w1);
+                if (L.k2) decode8(pre2[0], L.s2.bits, L.k2, w2);
+#pragma unroll
+                for (int i = 0; i + 1 < PF; i++) { pre1[i] = pre1[i + 1]; pre2[i] = pre2[i + 1]; }
+                if (rl + PF < nrows) {
+                    pre1[PF - 1] = load_raw8(row1 + (long long)(rl + PF) * L.s1.stride, L.s1.stride, grp, L.Nc, L.s1.bits);
+                    if (L.k2) pre2[PF - 1] = load_raw8(row2 + (long long)(rl + PF) * L.s2.stride, L.s2.stride, grp, L.Nc, L.s2.bits);
                 }
                 float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
