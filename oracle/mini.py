@@ -10,6 +10,7 @@ packed format; the packed format has its own decoder below.
 Restored weight (Sec. 2.2, Sec. 3.2.2 last sentence, Sec. 3.2.3, App. C.1):
   outlier column n < n_out :  t = C0[I0[m // v0, n], m % v0]
   other columns            :  t = C1[I1[m // v, c], m % v] (+ C2[I2[m // v, c], m % v]),  c = n - n_out
+  group-wise (Sec. 3.1)    :  C1, C2 are those of the column group g = c // ceil(Nc / group num)
   (project-defined)           W = fp16( fp32(fp32(t * scale) + bias) )
 """
 from __future__ import annotations
@@ -46,14 +47,20 @@ def unpack(packed: np.ndarray, rows: int, cols: int, k: int) -> np.ndarray:
 
 
 def dequant(M, N, v, c1, idx1, c2=None, idx2=None, n_out=0, v0=0, c0=None, idx0=None,
-            scale=None, bias=None, scale_axis=0) -> np.ndarray:
+            scale=None, bias=None, scale_axis=0, n_groups=1) -> np.ndarray:
     """float16 [M][N] from integer index matrices and float16 tables."""
     W = np.zeros((M, N), dtype=np.float32)
     m = np.arange(M)
     if n_out < N:
-        main = np.asarray(c1, np.float16)[np.asarray(idx1)[m // v], (m % v)[:, None]].astype(np.float32)
+        # one codebook pair per run of consecutive columns: entry i of group g sits at row g*k + i
+        G = max(1, int(n_groups))
+        Nc = N - n_out
+        grp = (np.arange(Nc) // (-(-Nc // G)))[None, :]
+        k1 = np.asarray(c1).shape[0] // G
+        main = np.asarray(c1, np.float16)[grp * k1 + np.asarray(idx1)[m // v], (m % v)[:, None]].astype(np.float32)
         if c2 is not None:
-            res = np.asarray(c2, np.float16)[np.asarray(idx2)[m // v], (m % v)[:, None]].astype(np.float32)
+            k2 = np.asarray(c2).shape[0] // G
+            res = np.asarray(c2, np.float16)[grp * k2 + np.asarray(idx2)[m // v], (m % v)[:, None]].astype(np.float32)
             main = (main + res).astype(np.float32)
         W[:, n_out:] = main
     if n_out > 0:
@@ -79,4 +86,4 @@ def linear(W16: np.ndarray, x_f64: np.ndarray) -> np.ndarray:
 def dequant_from_synth(d, scale_axis=0) -> np.ndarray:
     s = d["spec"]
     return dequant(s.M, s.N, s.v, d["c1"], d["idx1"], d["c2"], d["idx2"], s.n_out, s.v0,
-                   d["c0"], d["idx0"], d["scale"], d["bias"], scale_axis)
+                   d["c0"], d["idx0"], d["scale"], d["bias"], scale_axis, getattr(s, "n_groups", 1))

@@ -24,7 +24,7 @@ class _Layer(C.Structure):
     _fields_ = [("M", C.c_int32), ("N", C.c_int32),
                 ("v", C.c_int32), ("k1", C.c_int32), ("k2", C.c_int32),
                 ("n_out", C.c_int32), ("v0", C.c_int32), ("k0", C.c_int32),
-                ("has_scale", C.c_int32), ("scale_axis", C.c_int32),
+                ("has_scale", C.c_int32), ("scale_axis", C.c_int32), ("n_groups", C.c_int32),
                 ("idx1", C.c_void_p), ("c1", C.c_void_p),
                 ("idx2", C.c_void_p), ("c2", C.c_void_p),
                 ("idx0", C.c_void_p), ("c0", C.c_void_p),
@@ -59,6 +59,8 @@ _lib.oracle_linear_rows.argtypes = [C.POINTER(_Layer), C.c_void_p, C.c_int32, C.
 for _n in ("oracle_codebook_bits",):
     getattr(_lib, _n).restype = C.c_double
     getattr(_lib, _n).argtypes = [C.c_int32] * 6
+_lib.oracle_equivalent_bits_grouped.restype = C.c_double
+_lib.oracle_equivalent_bits_grouped.argtypes = [C.c_int32] * 9
 for _n in ("oracle_index_bits_total", "oracle_equivalent_bits", "oracle_compression_ratio"):
     getattr(_lib, _n).restype = C.c_double
     getattr(_lib, _n).argtypes = [C.c_int32] * 8
@@ -118,7 +120,7 @@ class Layer:
 
     def __init__(self, M, N, v, k1, c1, idx1_packed, k2=0, c2=None, idx2_packed=None,
                  n_out=0, v0=0, k0=0, c0=None, idx0_packed=None,
-                 scale=None, bias=None, scale_axis=0):
+                 scale=None, bias=None, scale_axis=0, n_groups=1):
         def u16(a):
             return None if a is None else np.ascontiguousarray(a).view(np.uint16).reshape(-1).copy()
 
@@ -127,12 +129,13 @@ class Layer:
 
         self.M, self.N, self.v, self.k1, self.k2 = M, N, v, k1, k2
         self.n_out, self.v0, self.k0 = n_out, v0, k0
+        self.n_groups = G = max(1, int(n_groups))
         self._keep = dict(idx1=u8(idx1_packed), c1=u16(c1), idx2=u8(idx2_packed), c2=u16(c2),
                           idx0=u8(idx0_packed), c0=u16(c0), scale=u16(scale), bias=u16(bias))
         R, Nc = -(-M // v), N - n_out
-        assert self._keep["idx1"].size == packed_bytes(R, Nc, k1) and self._keep["c1"].size == k1 * v
+        assert self._keep["idx1"].size == packed_bytes(R, Nc, k1) and self._keep["c1"].size == G * k1 * v
         if k2:
-            assert self._keep["idx2"].size == packed_bytes(R, Nc, k2) and self._keep["c2"].size == k2 * v
+            assert self._keep["idx2"].size == packed_bytes(R, Nc, k2) and self._keep["c2"].size == G * k2 * v
         if n_out:
             assert self._keep["idx0"].size == packed_bytes(-(-M // v0), n_out, k0)
             assert self._keep["c0"].size == k0 * v0
@@ -141,7 +144,7 @@ class Layer:
             assert self._keep["scale"].size == (M if scale_axis else N)
             assert self._keep["bias"].size == (M if scale_axis else N)
         p = lambda n: (self._keep[n].ctypes.data if self._keep[n] is not None else None)
-        self.c = _Layer(M, N, v, k1, k2, n_out, v0, k0, int(has_scale), scale_axis,
+        self.c = _Layer(M, N, v, k1, k2, n_out, v0, k0, int(has_scale), scale_axis, G,
                         p("idx1"), p("c1"), p("idx2"), p("c2"), p("idx0"), p("c0"),
                         p("scale"), p("bias"))
 
@@ -153,7 +156,8 @@ class Layer:
                    k2=s.k2, c2=d["c2"], idx2_packed=pack(d["idx2"], s.k2) if s.k2 else None,
                    n_out=s.n_out, v0=s.v0, k0=s.k0, c0=d["c0"],
                    idx0_packed=pack(d["idx0"], s.k0) if s.n_out else None,
-                   scale=d["scale"], bias=d["bias"], scale_axis=scale_axis)
+                   scale=d["scale"], bias=d["bias"], scale_axis=scale_axis,
+                   n_groups=getattr(s, "n_groups", 1))
 
     def dequant(self) -> np.ndarray:
         """W16 [M][N] as numpy float16 (bit-exact definition of the restored weight)."""
@@ -197,6 +201,10 @@ def index_bits_total(M, N, v, k1, k2=0, n_out=0, v0=0, k0=0) -> float:
 
 def equivalent_bits(M, N, v, k1, k2=0, n_out=0, v0=0, k0=0) -> float:
     return float(_lib.oracle_equivalent_bits(M, N, v, k1, k2, n_out, v0, k0))
+
+
+def equivalent_bits_grouped(M, N, v, k1, k2=0, n_out=0, v0=0, k0=0, n_groups=1) -> float:
+    return float(_lib.oracle_equivalent_bits_grouped(M, N, v, k1, k2, n_out, v0, k0, n_groups))
 
 
 def compression_ratio(M, N, v, k1, k2=0, n_out=0, v0=0, k0=0) -> float:

@@ -182,10 +182,11 @@ typedef struct oracle_layer {
     int32_t n_out, v0, k0;   /* leading outlier columns, their vector length/table  */
     int32_t has_scale;       /* 1: W = t*scale[n] + bias[n]                          */
     int32_t scale_axis;      /* 0: per input column n; 1: per output row m          */
+    int32_t n_groups;        /* column groups with codebooks of their own (Sec. 3.1); <= 1: one */
     const uint8_t *idx1;     /* packed [ceil(M/v)][N-n_out], b(k1) bits             */
-    const uint16_t *c1;      /* [k1][v] fp16 bits                                   */
+    const uint16_t *c1;      /* [n_groups][k1][v] fp16 bits                         */
     const uint8_t *idx2;     /* packed, same shape, b(k2) bits (k2 > 0)             */
-    const uint16_t *c2;      /* [k2][v]                                             */
+    const uint16_t *c2;      /* [n_groups][k2][v]                                   */
     const uint8_t *idx0;     /* packed [ceil(M/v0)][n_out], b(k0) bits (n_out > 0)  */
     const uint16_t *c0;      /* [k0][v0]                                            */
     const uint16_t *scale;   /* fp16 bits, [N] (axis 0) or [M] (axis 1)             */
@@ -207,15 +208,20 @@ static uint16_t restore_weight(const oracle_layer *L, int32_t m, int32_t n, int 
     } else {
         int32_t c = n - L->n_out, Nc = L->N - L->n_out;
         int32_t r = m / L->v, j = m % L->v;
+        /* Sec. 3.1: the (non-outlier) columns are split into `group num` equal runs of consecutive
+         * columns, each with codebooks of its own; the last run is shorter when Nc is not a multiple. */
+        int32_t G = L->n_groups > 1 ? L->n_groups : 1;
+        int32_t cols_per_group = (Nc + G - 1) / G;
+        int32_t g = c / cols_per_group;
         int64_t stride1 = oracle_row_bytes(Nc, L->k1);
         int32_t i1 = read_index(L->idx1 + (int64_t)r * stride1, c, oracle_index_bits(L->k1));
         if (i1 >= L->k1) { *err = 1; return 0; }
-        t = oracle_half_to_float(L->c1[(int64_t)i1 * L->v + j]);
+        t = oracle_half_to_float(L->c1[((int64_t)g * L->k1 + i1) * L->v + j]);
         if (L->k2 > 0) {
             int64_t stride2 = oracle_row_bytes(Nc, L->k2);
             int32_t i2 = read_index(L->idx2 + (int64_t)r * stride2, c, oracle_index_bits(L->k2));
             if (i2 >= L->k2) { *err = 1; return 0; }
-            float t2 = oracle_half_to_float(L->c2[(int64_t)i2 * L->v + j]);
+            float t2 = oracle_half_to_float(L->c2[((int64_t)g * L->k2 + i2) * L->v + j]);
             t = t + t2;                     /* rounded FP32 add */
         }
     }
@@ -329,6 +335,17 @@ double oracle_compression_ratio(int32_t M, int32_t N, int32_t v, int32_t k1, int
                                 int32_t n_out, int32_t v0, int32_t k0)
 {
     return 16.0 / oracle_equivalent_bits(M, N, v, k1, k2, n_out, v0, k0);
+}
+
+/* The same with `group num` independent main/residual codebooks (Sec. 3.1; Table of App. B with the
+ * parameters of the published 2-bit models): the codebook term grows G-fold, the index term does not. */
+double oracle_equivalent_bits_grouped(int32_t M, int32_t N, int32_t v, int32_t k1, int32_t k2,
+                                      int32_t n_out, int32_t v0, int32_t k0, int32_t n_groups)
+{
+    double G = n_groups > 1 ? (double)n_groups : 1.0;
+    double codebooks = G * (double)v * ((double)k1 + (double)(k2 > 0 ? k2 : 0)) * 16.0;
+    if (n_out > 0) codebooks += (double)v0 * (double)k0 * 16.0;
+    return (codebooks + oracle_index_bits_total(M, N, v, k1, k2, n_out, v0, k0)) / ((double)M * (double)N);
 }
 
 int oracle_num_threads(void)

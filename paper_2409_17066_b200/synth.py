@@ -39,6 +39,7 @@ class LayerSpec:
     x_dtype: str = "fp16"     # "fp16" | "bf16"
     out_dtype: str = "fp16"   # "fp16" | "bf16" | "fp32"
     has_scale: bool = True
+    n_groups: int = 1         # column groups with codebooks of their own (Sec. 3.1 / App. B table)
 
     @property
     def R(self) -> int:
@@ -132,8 +133,9 @@ def make_indices(spec: LayerSpec, config: int, layer: int, dist: str = "uniform"
 
 def make_tables(spec: LayerSpec, config: int, layer: int):
     """Codebooks (float16) and per-input-channel scale / bias (float16)."""
-    c1 = _rng(config, layer, T_C1).normal(0.0, 0.02, size=(spec.k1, spec.v)).astype(np.float16)
-    c2 = (_rng(config, layer, T_C2).normal(0.0, 0.005, size=(spec.k2, spec.v)).astype(np.float16)
+    G = max(1, spec.n_groups)       # group g's codebook: rows [g*k, (g+1)*k)
+    c1 = _rng(config, layer, T_C1).normal(0.0, 0.02, size=(G * spec.k1, spec.v)).astype(np.float16)
+    c2 = (_rng(config, layer, T_C2).normal(0.0, 0.005, size=(G * spec.k2, spec.v)).astype(np.float16)
           if spec.k2 else None)
     c0 = (_rng(config, layer, T_C0).normal(0.0, 0.02, size=(spec.k0, spec.v0)).astype(np.float16)
           if spec.n_out else None)

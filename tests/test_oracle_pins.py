@@ -340,3 +340,61 @@ def test_config0_and_ragged_v6_bits():
     assert oracle.equivalent_bits(s.M, s.N, s.v, s.k1) == 1.25
     # the outlier column counts used for the 1 % setting
     assert synth.outlier_columns(4096, 1.0) == 41 and synth.outlier_columns(11008, 1.0) == 110
+
+
+# ---------------------------------------------------------------- group-wise codebooks (Sec. 3.1)
+
+def test_group_codebook_bits_reproduce_the_published_settings():
+    """The "bit" column of the App. B table with the parameters of the published 2-bit models:
+    it only comes out when every column group carries codebooks of its own."""
+    for model, h, f, kv, bit, pct, v0, k0, v, k1, k2, G in _rows("quant_args_bits.txt"):
+        h, f, kv, v0, k0, v, k1, k2, G = map(int, (h, f, kv, v0, k0, v, k1, k2, G))
+        linears = [(h, h), (kv, h), (kv, h), (h, h), (f, h), (f, h), (h, f)]
+        bits = weights = 0.0
+        for M, N in linears:
+            n_out = synth.outlier_columns(N, float(pct))
+            bits += oracle.equivalent_bits_grouped(M, N, v, k1, k2, n_out, v0, k0, G) * M * N
+            weights += M * N
+        assert abs(bits / weights - float(bit)) <= 0.011, (model, bit, bits / weights)
+    # a single shared codebook would miss the grouped rows by far more than the rounding
+    M = N = 4096
+    one = oracle.equivalent_bits_grouped(M, N, 12, 4096, 4096, 41, 4, 8192, 1)
+    four = oracle.equivalent_bits_grouped(M, N, 12, 4096, 4096, 41, 4, 8192, 4)
+    assert four - one == pytest.approx(3 * 12 * 8192 * 16 / (M * N))
+
+
+def test_groups_with_identical_codebooks_equal_one_codebook():
+    spec1 = synth.LayerSpec("g1", 50, 90, v=6, k1=64, k2=16, n_out=5, v0=4, k0=32)
+    d1 = synth.make_layer(spec1, 91, 0, 3)
+    ref = oracle.Layer.from_synth(d1)
+    for G in (2, 3, 7, 85):
+        specG = synth.LayerSpec(**{**spec1.__dict__, "n_groups": G})
+        dG = dict(d1, spec=specG, c1=np.tile(d1["c1"], (G, 1)), c2=np.tile(d1["c2"], (G, 1)))
+        LG = oracle.Layer.from_synth(dG)
+        assert np.array_equal(LG.dequant().view(np.uint16), ref.dequant().view(np.uint16))
+        assert np.array_equal(LG.linear(d1["x"]), ref.linear(d1["x"]))
+
+
+@pytest.mark.parametrize("G", [2, 3, 4, 16])
+def test_grouped_layers_vs_numpy_statement_and_group_boundaries(G):
+    spec = synth.LayerSpec("gg", 44, 101, v=12, k1=32, k2=8, n_out=3, v0=4, k0=16, n_groups=G)
+    d = synth.make_layer(spec, 92, G, 2)
+    L = oracle.Layer.from_synth(d)
+    W = L.dequant()
+    assert np.array_equal(W.view(np.uint16), mini.dequant_from_synth(d).view(np.uint16))
+    # a column's weights come from its own group's tables: zeroing every other group's tables
+    # must leave that group's columns untouched and change nothing but the others
+    Nc = spec.N - spec.n_out
+    cpg = -(-Nc // G)
+    g = G // 2
+    d0 = dict(d, c1=d["c1"].copy(), c2=d["c2"].copy())
+    keep1 = np.zeros(G * spec.k1, bool); keep1[g * spec.k1:(g + 1) * spec.k1] = True
+    keep2 = np.zeros(G * spec.k2, bool); keep2[g * spec.k2:(g + 1) * spec.k2] = True
+    d0["c1"][~keep1] = 0
+    d0["c2"][~keep2] = 0
+    W0 = oracle.Layer.from_synth(d0).dequant()
+    cols = spec.n_out + np.arange(g * cpg, min(Nc, (g + 1) * cpg))
+    assert np.array_equal(W0[:, cols].view(np.uint16), W[:, cols].view(np.uint16))
+    others = np.setdiff1d(np.arange(spec.n_out, spec.N), cols)
+    bias = d["bias"].astype(np.float32)[others]
+    assert np.array_equal(W0[:, others].astype(np.float32), np.broadcast_to(bias.astype(np.float16).astype(np.float32), (spec.M, others.size)))
