@@ -43,7 +43,7 @@ extern "C" {
 
 #define VPTQ_OK              0
 #define VPTQ_E_NULL         -1   /* a required pointer is null                              */
-#define VPTQ_E_SHAPE        -2   /* M,N,v,k <= 0, k > 65536, v > 32, n_outlier > N, B <= 0  */
+#define VPTQ_E_SHAPE        -2   /* M,N,v,k <= 0, k > 65536, v > 32, n_outlier > N, B <= 0, n_groups < 0 or > N - n_outlier */
 #define VPTQ_E_ALIGN        -3   /* a data pointer is not 16-byte aligned                   */
 #define VPTQ_E_UNSUPPORTED  -4   /* dtype / flag combination without a kernel               */
 #define VPTQ_E_WORKSPACE    -5   /* workspace missing or smaller than the query says        */
@@ -73,13 +73,16 @@ typedef struct vptq_layer_desc {
     int32_t x_dtype;     /* VPTQ_DTYPE_FP16 or _BF16                                         */
     int32_t out_dtype;   /* VPTQ_DTYPE_FP16, _BF16 or _FP32                                  */
     int32_t flags;       /* VPTQ_FLAG_*                                                      */
+    int32_t n_groups;    /* Sec. 3.1: the non-outlier columns are split into this many equal runs of
+                            consecutive columns (ceil((N-n_outlier)/n_groups) each, the last one
+                            shorter), each with main/residual codebooks of its own; 0 or 1 = one   */
 } vptq_layer_desc;
 
 /* The nine format pointers of a layer, in the order of the paper's format statement.
  *   packed_idx       packed [ceil(M/v)][N-n_outlier], b(k1) bits       (required unless n_outlier == N)
- *   codebook         fp16 [k1][v]                                       (required unless n_outlier == N)
+ *   codebook         fp16 [n_groups][k1][v]                             (required unless n_outlier == N)
  *   res_idx          packed, same shape, b(k2) bits                     (required iff k2 > 0)
- *   res_codebook     fp16 [k2][v]                                       (required iff k2 > 0)
+ *   res_codebook     fp16 [n_groups][k2][v]                             (required iff k2 > 0)
  *   outlier_idx      packed [ceil(M/v0)][n_outlier], b(k0) bits         (required iff n_outlier > 0)
  *   outlier_codebook fp16 [k0][v0]                                      (required iff n_outlier > 0)
  *   scale, bias      fp16 [N] (or [M] with VPTQ_FLAG_SCALE_ROWS)        (required iff VPTQ_FLAG_SCALE_BIAS)
@@ -128,7 +131,8 @@ int vptq_unpack(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k
 
 /* W_out[M][N] fp16 (device, row-major) = the restored weight:
  *   n <  n_outlier: t = C0[I0[m/v0][n]][m%v0]
- *   n >= n_outlier: t = C1[I1[m/v][c]][m%v] (+ C2[I2[m/v][c]][m%v]), c = n - n_outlier
+ *   n >= n_outlier: t = C1[I1[m/v][c]][m%v] (+ C2[I2[m/v][c]][m%v]), c = n - n_outlier,
+ *                   C1/C2 = the tables of column group c / ceil((N-n_outlier)/n_groups)
  *   W = fp16_rne( fp32(fp32(t*scale) + bias) ) when VPTQ_FLAG_SCALE_BIAS, else fp16(t).
  * Bit-exact by definition (no fused multiply-add, denormals kept).  Indices >= k in a
  * corrupt stream are clamped to k-1, never read out of range. */

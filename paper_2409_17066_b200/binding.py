@@ -39,7 +39,8 @@ class LayerDesc(C.Structure):
     """vptq_layer_desc"""
     _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("v", C.c_int32), ("k1", C.c_int32),
                 ("k2", C.c_int32), ("n_outlier", C.c_int32), ("v0", C.c_int32), ("k0", C.c_int32),
-                ("x_dtype", C.c_int32), ("out_dtype", C.c_int32), ("flags", C.c_int32)]
+                ("x_dtype", C.c_int32), ("out_dtype", C.c_int32), ("flags", C.c_int32),
+                ("n_groups", C.c_int32)]
 
 
 class LayerPtrs(C.Structure):
@@ -101,8 +102,8 @@ def _stream() -> int:
 
 
 def make_desc(M, N, v, k1, k2=0, n_outlier=0, v0=0, k0=0, x_dtype="fp16", out_dtype="fp16",
-              flags=FLAG_SCALE_BIAS) -> LayerDesc:
-    return LayerDesc(M, N, v, k1, k2, n_outlier, v0, k0, _DT[x_dtype], _DT[out_dtype], flags)
+              flags=FLAG_SCALE_BIAS, n_groups=1) -> LayerDesc:
+    return LayerDesc(M, N, v, k1, k2, n_outlier, v0, k0, _DT[x_dtype], _DT[out_dtype], flags, n_groups)
 
 
 # ---- entry points (same names as the C ABI) -------------------------------------------
@@ -235,7 +236,8 @@ class DeviceLayer:
             flags = FLAG_SCALE_BIAS if d["scale"] is not None else 0
             if scale_rows:
                 flags |= FLAG_SCALE_ROWS
-        self.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags)
+        self.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags,
+                              getattr(s, "n_groups", 1))
         self.ptrs = LayerPtrs(_ptr(self.idx1), _ptr(self.c1), _ptr(self.idx2), _ptr(self.c2),
                               _ptr(self.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias))
         self._ws: Dict[int, Optional[torch.Tensor]] = {}
@@ -245,7 +247,8 @@ class DeviceLayer:
         other = object.__new__(DeviceLayer)
         other.__dict__.update(self.__dict__)
         s = self.spec
-        other.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags)
+        other.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags,
+                               getattr(s, "n_groups", 1))
         other._ws = {}
         return other
 

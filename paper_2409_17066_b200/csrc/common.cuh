@@ -48,6 +48,7 @@ inline Stream make_stream(const uint8_t *p, int cols, int k)
 struct LayerView {
     int M, N, v, k1, k2, n_out, v0, k0;
     int R, R0, Nc;
+    int G, cpg;            // column groups with codebooks of their own, columns per group (Sec. 3.1)
     int has_scale, scale_rows;
     int x_bf16, out_dtype;
     int cta_pairs;         // batched path: CTA pairs requested

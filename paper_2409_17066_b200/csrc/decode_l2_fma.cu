@@ -456,6 +456,7 @@ cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, in
 
 bool l2_fma_supported(const LayerView &L, int B)
 {
+    if (L.G > 1) return false;          // one codebook pair per layer here
     if (B < 1 || B > 16) return false;
     if (L.v != 8 || L.n_out != 0 || L.scale_rows) return false;
     if (L.s1.bits != 16) return false;

@@ -473,6 +473,7 @@ cudaError_t launch_vv(const SmemFmaParams &P, const SmemFmaPlan &pl, int v, bool
 
 bool smem_fma_supported(const LayerView &L, int B)
 {
+    if (L.G > 1) return false;          // one codebook pair per layer here
     if (B < 1 || B > SMEM_FMA_MAX_B) return false;     // beyond that the mma.sync kernel is faster
     if (L.Nc <= 0 || L.scale_rows) return false;
     if (L.v > 8 || (L.n_out > 0 && L.v0 > 8)) return false;

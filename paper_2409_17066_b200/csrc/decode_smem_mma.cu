@@ -454,6 +454,7 @@ int pad16(int x) { return (x + 15) / 16 * 16; }
 
 bool smem_mma_supported(const LayerView &L, int B)
 {
+    if (L.G > 1) return false;          // one codebook pair per layer here
     if (B < 1 || B > 16) return false;
     if (L.v > 8 || (L.n_out > 0 && L.v0 > 8)) return false;
     if (L.Nc > 0 && (long long)L.k1 * 16 > 128 * 1024) return false;

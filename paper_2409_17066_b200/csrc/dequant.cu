@@ -36,10 +36,11 @@ dequant_kernel(LayerView L, __half *__restrict__ W)
         e1 = L.c0 + (long long)i0 * vlen;
     } else {
         int i1 = clamp_index(load_index(L.s1.ptr + (long long)r * L.s1.stride, c, L.s1.bits), L.k1);
-        e1 = L.c1 + (long long)i1 * vlen;
+        const int g = c / L.cpg;                       // Sec. 3.1: this column's group has its own tables
+        e1 = L.c1 + ((long long)g * L.k1 + i1) * vlen;
         if (L.k2 > 0) {
             int i2 = clamp_index(load_index(L.s2.ptr + (long long)r * L.s2.stride, c, L.s2.bits), L.k2);
-            e2 = L.c2 + (long long)i2 * vlen;
+            e2 = L.c2 + ((long long)g * L.k2 + i2) * vlen;
         }
     }
     float s = 1.f, b = 0.f;

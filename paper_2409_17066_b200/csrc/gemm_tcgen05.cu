@@ -808,6 +808,7 @@ GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
 
 bool gemm_tcgen05_supported(const LayerView &L, int B)
 {
+    if (L.G > 1) return false;          // one codebook pair per layer here
     if (B <= 16) return false;
     if (L.v != 8 || L.n_out != 0 || L.scale_rows) return false;
     if (L.s1.bits != 16) return false;

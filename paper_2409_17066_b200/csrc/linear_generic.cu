@@ -39,10 +39,11 @@ linear_generic_kernel(LayerView L, const void *__restrict__ x, int B, void *__re
             } else {
                 int c = n - L.n_out;
                 int i1 = clamp_index(load_index(row1, c, L.s1.bits), L.k1);
-                w = __half2float(__ldg(L.c1 + (long long)i1 * L.v + j));
+                const int g = c / L.cpg;          // Sec. 3.1: this column's group has its own tables
+                w = __half2float(__ldg(L.c1 + ((long long)g * L.k1 + i1) * L.v + j));
                 if (L.k2) {
                     int i2 = clamp_index(load_index(row2, c, L.s2.bits), L.k2);
-                    w += __half2float(__ldg(L.c2 + (long long)i2 * L.v + j));
+                    w += __half2float(__ldg(L.c2 + ((long long)g * L.k2 + i2) * L.v + j));
                 }
             }
             if (L.has_scale) {

@@ -29,6 +29,7 @@ int check_desc(const vptq_layer_desc *d)
     if (d->v <= 0 || d->v > 32 || d->k1 <= 0 || d->k1 > 65536) return VPTQ_E_SHAPE;
     if (d->k2 < 0 || d->k2 > 65536) return VPTQ_E_SHAPE;
     if (d->n_outlier < 0 || d->n_outlier > d->N) return VPTQ_E_SHAPE;
+    if (d->n_groups < 0 || (d->n_groups > 1 && d->n_groups > d->N - d->n_outlier)) return VPTQ_E_SHAPE;
     if (d->n_outlier > 0 && (d->v0 <= 0 || d->v0 > 32 || d->k0 <= 0 || d->k0 > 65536)) return VPTQ_E_SHAPE;
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
@@ -68,6 +69,8 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     L.k0 = L.n_out ? d->k0 : 1;
     L.Nc = L.N - L.n_out;
     L.k2 = L.Nc > 0 ? d->k2 : 0;
+    L.G = (d->n_groups > 1 && L.Nc > 0) ? d->n_groups : 1;
+    L.cpg = L.Nc > 0 ? ceil_div(L.Nc, L.G) : 1;
     L.R = ceil_div(L.M, L.v);
     L.R0 = L.n_out ? ceil_div(L.M, L.v0) : 0;
     L.has_scale = (d->flags & VPTQ_FLAG_SCALE_BIAS) ? 1 : 0;
@@ -118,8 +121,8 @@ int64_t vptq_layer_weight_bytes(const vptq_layer_desc *d)
     LayerView L = make_view(d, nullptr);
     int64_t bytes = 0;
     if (L.Nc > 0) {
-        bytes += (int64_t)L.R * row_bytes(L.Nc, L.k1) + 2LL * L.k1 * L.v;
-        if (L.k2) bytes += (int64_t)L.R * row_bytes(L.Nc, L.k2) + 2LL * L.k2 * L.v;
+        bytes += (int64_t)L.R * row_bytes(L.Nc, L.k1) + 2LL * L.G * L.k1 * L.v;
+        if (L.k2) bytes += (int64_t)L.R * row_bytes(L.Nc, L.k2) + 2LL * L.G * L.k2 * L.v;
     }
     if (L.n_out) bytes += (int64_t)L.R0 * row_bytes(L.n_out, L.k0) + 2LL * L.k0 * L.v0;
     if (L.has_scale) bytes += 4LL * (L.scale_rows ? L.M : L.N);

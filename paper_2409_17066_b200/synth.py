@@ -176,4 +176,8 @@ def small_specs() -> List[LayerSpec]:
         LayerSpec("s_v1_k1", 9, 17, v=1, k1=1),
         LayerSpec("s_v8_alloutlier", 64, 96, v=8, k1=256, n_out=96, v0=4, k0=4096),
         LayerSpec("s_v12_k4096", 60, 130, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192),
+        # group-wise codebooks (Sec. 3.1), with the parameter settings of the published 2-bit models
+        LayerSpec("s_v12_g4", 60, 134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4),
+        LayerSpec("s_v6_g16", 100, 333, v=6, k1=4096, n_out=3, v0=4, k0=8192, n_groups=16),
+        LayerSpec("s_v8_g3", 72, 200, v=8, k1=256, k2=16, n_groups=3),
     ]

@@ -52,11 +52,13 @@ def test_layer_weight_bytes_follow_the_bit_formulas(binding):
     # App. C.2: index bits log2(k)/v per weight and codebook bits (v0*k0 + v1*(k1+k2))*16
     for cfg in range(5):
         for s in synth.CONFIGS[cfg]["layers"]:
-            d = binding.make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype)
+            d = binding.make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype,
+                                  n_groups=s.n_groups)
             got = binding.vptq_layer_weight_bytes(d)
             exp = oracle.packed_bytes(s.R, s.Nc, s.k1) + (oracle.packed_bytes(s.R, s.Nc, s.k2) if s.k2 else 0) \
                 + (oracle.packed_bytes(s.R0, s.n_out, s.k0) if s.n_out else 0) \
-                + oracle.codebook_bits(s.v, s.k1, s.k2, s.n_out, s.v0, s.k0) / 8 + 4 * s.N
+                + (oracle.codebook_bits(s.v, s.k1, s.k2, 0, 0, 0) * max(1, s.n_groups)
+                   + (oracle.codebook_bits(s.v, 0, 0, s.n_out, s.v0, s.k0) if s.n_out else 0)) / 8 + 4 * s.N
             assert got == exp
     # the worked example of Sec. 2.2: 4096 x 4096, v = 8, k = 256, no scale/bias
     d = binding.make_desc(4096, 4096, 8, 256, flags=0)
