@@ -54,7 +54,7 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     "decode_smem_mma_kernel": 1.004,
 }
 
-ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
+ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
                    "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel"}
 
 
@@ -409,7 +409,7 @@ def extra_configs(vb, synth, peaks):
     """µs/call, effective weight GB/s (and TFLOP/s for the batched case) of the other workloads."""
     import torch
     res = {}
-    for cfg in (0, 1, 2, 4):
+    for cfg in (0, 1, 2, 4, 5):
         c = synth.CONFIGS[cfg]
         seen = set()
         for li, spec in enumerate(c["layers"]):

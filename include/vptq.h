@@ -217,7 +217,7 @@ const char *vptq_last_cuda_error(void);
  * is then invalid; the context stays usable), else VPTQ_OK.  A null workspace returns VPTQ_OK. */
 int vptq_workspace_status(const void *workspace, void *stream);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_fma",
- * "decode_smem_mma", "decode_l2_fma", "gemm_tcgen05".  For tests and benchmark logs. */
+ * "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05".  For tests and benchmark logs. */
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B);
 /* Number of kernels one vptq_linear call launches (scratch memsets are not counted). */
 int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B);

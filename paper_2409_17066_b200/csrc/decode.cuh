@@ -19,4 +19,9 @@ long long l2_fma_workspace_bytes(const LayerView &L, int B);
 int l2_fma_launches(const LayerView &L, int B);
 cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
 
+// codebooks in global memory, any even v <= 16, group-wise codebooks, FP32 FMAs, no scratch
+bool gl_fma_supported(const LayerView &L, int B);
+int gl_fma_launches(const LayerView &L, int B);
+cudaError_t launch_decode_gl_fma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
+
 }  // namespace vptq

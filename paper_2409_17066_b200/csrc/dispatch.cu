@@ -18,6 +18,7 @@ LinearPath choose_path(const LayerView &L, int B, int flags)
     if (smem_fma_supported(L, Bg)) return PATH_DECODE_SMEM_FMA;
     if (smem_mma_supported(L, Bg)) return PATH_DECODE_SMEM_MMA;
     if (l2_fma_supported(L, Bg)) return PATH_DECODE_L2_FMA;
+    if (gl_fma_supported(L, Bg)) return PATH_DECODE_GL_FMA;
     return PATH_GENERIC;
 }
 
@@ -27,6 +28,7 @@ const char *linear_path_name(const LayerView &L, int B, int flags)
     case PATH_DECODE_SMEM_FMA: return "decode_smem_fma";
     case PATH_DECODE_SMEM_MMA: return "decode_smem_mma";
     case PATH_DECODE_L2_FMA: return "decode_l2_fma";
+    case PATH_DECODE_GL_FMA: return "decode_gl_fma";
     case PATH_GEMM_TCGEN05: return "gemm_tcgen05";
     default: return "generic";
     }
@@ -38,6 +40,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
     case PATH_DECODE_SMEM_FMA: return 0;
     case PATH_DECODE_SMEM_MMA: return 0;
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
+    case PATH_DECODE_GL_FMA: return 0;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
     default: return generic_workspace_bytes(L, B);
     }
@@ -54,6 +57,8 @@ int linear_launches(const LayerView &L, int B, int flags)
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_launches(L, B);
     case PATH_DECODE_L2_FMA:
         return (groups - 1) * l2_fma_launches(L, DECODE_MAX_B) + l2_fma_launches(L, last);
+    case PATH_DECODE_GL_FMA:
+        return (groups - 1) * gl_fma_launches(L, DECODE_MAX_B) + gl_fma_launches(L, last);
     default: return generic_launches(L, B);
     }
 }
@@ -76,6 +81,7 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
             void *og = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
             if (path == PATH_DECODE_SMEM_FMA) e = launch_decode_smem_fma(L, xg, Bg, og, st);
             else if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, st);
+            else if (path == PATH_DECODE_GL_FMA) e = launch_decode_gl_fma(L, xg, Bg, og, st);
             else e = launch_decode_l2_fma(L, xg, Bg, og, ws, st);
         }
     }

@@ -72,7 +72,15 @@ def _c4(M, N, name):
     return LayerSpec(name, M, N, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32")
 
 
-# The five workloads: (list of layers, list of batch sizes)
+def _c5(M, N, name):
+    # App. B table, LLaMA-2-7B at 2.26 bit: v = 12, two 4096-entry codebooks per group, 4 groups,
+    # 1 % outlier columns with v0 = 4, k0 = 8192 (13-bit indices)
+    return LayerSpec(name, M, N, v=12, k1=4096, k2=4096,
+                     n_out=outlier_columns(N, 1.0), v0=4, k0=8192, n_groups=4)
+
+
+# The five workloads: (list of layers, list of batch sizes); number 5 is an addition: the parameter
+# setting of one of the paper's published 2-bit models (group-wise codebooks)
 CONFIGS: Dict[int, Dict] = {
     0: dict(name="tiny_256x512",
             layers=[LayerSpec("tiny", 256, 512, v=8, k1=256)],
@@ -89,6 +97,9 @@ CONFIGS: Dict[int, Dict] = {
                     _c3(1024, 8192, "v_proj"), _c3(8192, 8192, "o_proj"),
                     _c3(28672, 8192, "gate_proj"), _c3(28672, 8192, "up_proj"),
                     _c3(8192, 28672, "down_proj")],
+            batches=[1]),
+    5: dict(name="llama2_7b_published_2p26bit_setting",
+            layers=[_c5(4096, 4096, "q_proj"), _c5(11008, 4096, "gate_proj"), _c5(4096, 11008, "down_proj")],
             batches=[1]),
     4: dict(name="llama3_8b_mlp_prefill",
             layers=[_c4(14336, 4096, "gate_proj"), _c4(14336, 4096, "up_proj"),

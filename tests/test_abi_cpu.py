@@ -50,7 +50,7 @@ def test_format_arithmetic_matches_oracle(binding):
 
 def test_layer_weight_bytes_follow_the_bit_formulas(binding):
     # App. C.2: index bits log2(k)/v per weight and codebook bits (v0*k0 + v1*(k1+k2))*16
-    for cfg in range(5):
+    for cfg in sorted(synth.CONFIGS):
         for s in synth.CONFIGS[cfg]["layers"]:
             d = binding.make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype,
                                   n_groups=s.n_groups)
@@ -87,5 +87,5 @@ def test_argument_errors_need_no_gpu(binding):
     p2 = b.LayerPtrs(0x1008, 0x1000, None, None, None, None, 0x1000, 0x1000)
     assert b.lib.vptq_dequant(C.byref(d), C.byref(p2), 0x1000, None) == b.E_ALIGN
     assert b.lib.vptq_status_string(b.E_ALIGN).decode().startswith("a data pointer")
-    assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_fma", "decode_smem_mma", "decode_l2_fma", "gemm_tcgen05")
+    assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_fma", "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05")
     assert b.vptq_linear_launches(d, 1) >= 1
