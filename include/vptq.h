@@ -59,8 +59,6 @@ extern "C" {
 #define VPTQ_FLAG_SCALE_BIAS   1  /* scale and bias are present                                     */
 #define VPTQ_FLAG_SCALE_ROWS   2  /* scale/bias are per OUTPUT row ([M]) instead of per input column */
 #define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
-#define VPTQ_FLAG_CTA_PAIRS     8 /* batched path: pair two CTAs per 256-row tile (tcgen05 cta_group::2)
-                                     where the device runs such pairs; default is one CTA per tile   */
 
 /* Geometry of one quantized linear layer (App. C.1 names: v1,k1,k2 / N%,v0,k0). */
 typedef struct vptq_layer_desc {

@@ -51,7 +51,6 @@ struct LayerView {
     int G, cpg;            // column groups with codebooks of their own, columns per group (Sec. 3.1)
     int has_scale, scale_rows;
     int x_bf16, out_dtype;
-    int cta_pairs;         // batched path: CTA pairs requested
     Stream s1, s2, s0;
     const __half *c1, *c2, *c0;
     const __half *scale, *bias;

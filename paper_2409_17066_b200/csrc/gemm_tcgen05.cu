@@ -7,22 +7,26 @@
 //       centroid (8 consecutive output rows of one input column) = C1[i1] + C2[i2] per store,
 //       in the MN-major 128-byte-swizzled layout tcgen05.mma reads;
 //   B = x*s tile (FP16, scale folded into the activations by a pre-pass), 512 tokens x 32
-//       columns, K-major, loaded by TMA with the 64-byte swizzle (no multicast);
+//       columns, K-major with the 64-byte swizzle.  The pre-pass writes the activations as the
+//       shared-memory image of these tiles ([256-token half][k block] -> 16 KB, swizzle applied),
+//       so a tile half arrives by one linear bulk copy of whole 128-byte lines (a tiled TMA load of
+//       64-byte rows asks L2 for twice as many pieces);
 //   tcgen05.mma.cta_group::1.kind::f16, M = 128, N = 256 (two per token tile), K = 16.
 //
-// Warp roles (576 threads): warp 0 TMA loads of B; warp 1 TMEM allocation + MMA issue (one
-// thread); warps 2-9 dequant producers (a pair per k block: a1 unpack with the next visit's
+// Warp roles (640 threads): warp 0 bulk loads of B; warp 1 TMEM allocation + MMA issue (one
+// thread); warps 2-11 dequant producers (a pair per k block: a1 unpack with the next visit's
 // indices already in flight, a3 main lookup from the L2-resident codebook, a4 residual lookup
-// from shared memory, add, store); warps 10-17 epilogue (tcgen05.ld -> + bias term -> store or
-// red.add), two per TMEM lane quarter.
-// A and B have rings of their own: A is deep (the producers' gathers need about a microsecond),
-// B holds 32 KB per stage and is shallow.
-// CTA pairs (CG = 2): two CTAs of a cluster work on one 256-row tile with tcgen05.mma.cta_group::2:
-// each dequantises its own 128 rows and loads half of the tokens of every 256-token MMA (no TMA
-// multicast), the even CTA issues the MMAs for both, accumulators sit in each CTA's own TMEM.
-// That halves the activation traffic from L2 and the shared-memory traffic per MMA.  All
-// barriers the issuing thread waits on live in the even CTA (the odd CTA arrives remotely);
-// tcgen05.commit multicasts to both CTAs.  CG = 1 keeps everything in one CTA.
+// from shared memory, add, store); warps 12-19 epilogue (tcgen05.ld -> + bias term -> shared
+// memory -> TMA store or reduce-add), two per TMEM lane quarter.  Twenty warps are five per
+// scheduler: the register budget per thread is the same from 17 to 20 warps.
+// A and B have rings of their own: A has a stage per producer pair and one to spare (the
+// producers' gathers need a few microseconds), B holds 32 KB per stage and is shallow.
+// What bounds the k loop is the SM's request path to L2 (about one request per clock): per k block
+// 512 centroid reads and 256 lines of activations.  Two ways of sharing the activation tiles in a
+// CTA pair were measured and dropped: tcgen05 cta_group::2 (each CTA loads half of the tokens; the
+// pair advances at the pace of its slower half: 103 us against 88 us on the 14336 x 4096 layer at
+// 512 tokens) and forwarding the own half into the partner's shared memory (the forwarded bytes
+// load the same outgoing path: 117 us).
 // Persistent grid, one CTA per SM.  The work is the list of (tile, k block) units, tile =
 // (token tile, 128-row tile); with an FP32 output every CTA takes an equal, contiguous share of
 // the units, whatever tile they fall in (partial tiles meet in the output by red.add), so all
@@ -46,33 +50,28 @@ constexpr int TILE_N = 512;
 constexpr int MMA_N = 256;
 constexpr int A_STAGES = 6;                              // ring of dequantised weight tiles
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;       // 8 KB
-// ring of activation tiles: per CTA and stage 2 halves x (256 / CG tokens) x 32 columns
-template <int CG> struct BRing {
-    static constexpr int HALF_BYTES = (MMA_N / CG) * TILE_K * 2;     // 16 KB / 8 KB
-    static constexpr int STAGE_BYTES = 2 * HALF_BYTES;               // 32 KB / 16 KB
-    static constexpr int STAGES = CG == 1 ? 3 : 6;                   // 96 KB either way
-};
-constexpr int PAIRS = 4;                                 // producer warp pairs; pair p fills k blocks p, p+PAIRS, ...
+constexpr int B_STAGES = 3;                              // ring of activation tiles
+constexpr int B_HALF_BYTES = MMA_N * TILE_K * 2;         // 256 tokens x 32 columns: 16 KB, one bulk copy
+constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;          // 32 KB
+constexpr int PAIRS = 5;                                 // producer warp pairs; pair p fills k blocks p, p+PAIRS, ...
 constexpr int PRODUCER_WARPS = 2 * PAIRS;
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 16 * 32 * 4;                // one staged piece of the output: 16 tokens x 32 rows, FP32
 constexpr int EPI_STAGE_BYTES = EPI_WARPS * 2 * EPI_BUF_BYTES;   // two buffers per epilogue warp: 32 KB
 constexpr int CB2_REPLICAS = 4;                          // copies of a small residual table (16-byte skew)
 static_assert(A_STAGES >= PAIRS, "a producer pair needs a stage of its own");
-constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 448
+constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 640
 constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
 constexpr int A_LBO = 1024;   // bytes between the two 64-row blocks of the A stage
 constexpr int B_SBO = 512;    // bytes between consecutive 8-token groups of the B stage (8 x 64 B)
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
 
 constexpr int WS_STATUS_BYTES = 256;
-constexpr bool PREFER_CTA_PAIRS = false;
 
 struct GemmParams {
     LayerView L;
     void *out;
     int B;
-    int Npad;            // row stride of xs in elements
     int tiles_m, tiles_t, kb_total;
     int unit_gran;       // a CTA's share of the units is a multiple of this (1, or kb_total = whole tiles)
     long long units;     // tiles_m * tiles_t * kb_total
@@ -81,6 +80,7 @@ struct GemmParams {
     int tma_out;         // FP32 output written by TMA store / reduce from shared memory (needs M % 4 == 0)
     int *status;         // workspace status word
     const float *bterm;  // [B]
+    const uint8_t *xs;   // activation tile images, [ceil(B / 256)][kb_total][16 KB]
 };
 
 // ---- PTX wrappers ----------------------------------------------------------------------------
@@ -126,10 +126,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+// linear bulk copy global -> shared memory (16-byte aligned addresses, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout)
@@ -144,78 +145,33 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
 }
 constexpr uint32_t LAYOUT_SW128 = 2, LAYOUT_SW64 = 4;
 
-// kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128 * CG, N = 256
-template <int CG>
-__device__ __forceinline__ constexpr uint32_t idesc()
-{
-    return (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
-           ((uint32_t)(MMA_N >> 3) << 17) | ((uint32_t)((TILE_M * CG) >> 4) << 24);
-}
+// kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128, N = 256
+constexpr uint32_t IDESC = (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
+                           ((uint32_t)(MMA_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 
-template <int CG>
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
 {
-    if (CG == 1)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc<1>()), "r"(accumulate) : "memory");
-    else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc<2>()), "r"(accumulate) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(IDESC), "r"(accumulate) : "memory");
 }
 // The MMAs of one 32-column k block: two k16 steps x one or two 256-token halves, issued back to back.
 // `ad`/`bd` describe the k16 = 0 slice of the stage; the second slice lies 2 * A_SBO (A) and 32 bytes (B)
-// further, the second token half b_half_bytes further (descriptor address units are 16 bytes).
-template <int CG>
-__device__ __forceinline__ void umma_kblock(uint32_t d_tmem, uint64_t ad, uint64_t bd, uint32_t accumulate,
-                                            bool two_halves, int b_half_bytes)
+// further, the second token half B_HALF_BYTES further (descriptor address units are 16 bytes).
+__device__ __forceinline__ void umma_kblock(uint32_t d_tmem, uint64_t ad, uint64_t bd, uint32_t accumulate, bool two_halves)
 {
     const uint64_t ad1 = ad + (uint64_t)((2 * A_SBO) >> 4);
     const uint64_t bd1 = bd + 2u;
-    const uint64_t bh = (uint64_t)(b_half_bytes >> 4);
-    umma_f16<CG>(d_tmem, ad, bd, accumulate);
-    if (two_halves) umma_f16<CG>(d_tmem + MMA_N, ad, bd + bh, accumulate);
-    umma_f16<CG>(d_tmem, ad1, bd1, 1u);
-    if (two_halves) umma_f16<CG>(d_tmem + MMA_N, ad1, bd1 + bh, 1u);
+    const uint64_t bh = (uint64_t)(B_HALF_BYTES >> 4);
+    umma_f16(d_tmem, ad, bd, accumulate);
+    if (two_halves) umma_f16(d_tmem + MMA_N, ad, bd + bh, accumulate);
+    umma_f16(d_tmem, ad1, bd1, 1u);
+    if (two_halves) umma_f16(d_tmem + MMA_N, ad1, bd1 + bh, 1u);
 }
-// Arrive on the barrier once all MMAs issued so far have completed; with CG = 2 the arrival goes
-// to the barrier at the same offset in both CTAs of the pair.
-template <int CG>
+// Arrive on the barrier once all MMAs issued so far have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
-    if (CG == 1)
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-    else
-        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                     ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-// CG = 2: the copy lands in this CTA's shared memory and signals the barrier `bar` of the even CTA.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -254,13 +210,25 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-// ---- pre-pass: xs = fp16(x * s), bterm[t] = sum_n x[t][n] * b[n], status = 0; clears row t of an FP32
-//      output in which partial tiles are going to meet by red.add (zero_out != nullptr) -------------
+// ---- pre-pass: xs = fp16(x * s) written as tile images, bterm[t] = sum_n x[t][n] * b[n], status = 0; clears
+//      row t of an FP32 output in which partial tiles are going to meet by red.add (zero_out != nullptr).
+// Image of the tile half (256 tokens) x (k block of 32 columns): token r, 16-byte chunk q (8 columns) at
+//      (r / 8) * 512 + (r % 8) * 64 + ((q ^ ((r % 8) / 2)) * 16: the K-major 64-byte-swizzled operand layout.
+// One block per token of the padded range; tokens >= B and columns >= N are written as zeros. ---------------
 __global__ void __launch_bounds__(256)
-gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __half *__restrict__ xs,
+gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__restrict__ xs,
                     float *__restrict__ bterm, int *status, float *__restrict__ zero_out)
 {
     const int t = blockIdx.x;
+    const int kb_total = (L.N + TILE_K - 1) / TILE_K;
+    // where token t's 64 bytes of k block 0 start; the other k blocks follow at B_HALF_BYTES each
+    uint8_t *img_row = xs + (long long)(t / MMA_N) * kb_total * B_HALF_BYTES + ((t % MMA_N) >> 3) * B_SBO + (t & 7) * 64;
+    const int sw = (t & 7) >> 1;
+    if (t >= B) {
+        for (int q = threadIdx.x; q < 4 * kb_total; q += 256)
+            *reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
+        return;
+    }
     if (t == 0 && threadIdx.x == 0) *status = 0;
     if (zero_out != nullptr) {
         float *row = zero_out + (long long)t * L.M;
@@ -273,8 +241,11 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
     }
     float acc = 0.f;
     if ((L.N & 7) == 0) {
-        // 8 columns per thread and step, 128-bit loads and stores (Npad == N)
-        for (int n = 8 * threadIdx.x; n < L.N; n += 8 * 256) {
+        // 8 columns = one chunk per thread and step, 128-bit loads and stores
+        for (int n = 8 * threadIdx.x; n < kb_total * TILE_K; n += 8 * 256) {
+            const int q = n >> 3;
+            uint4 *dst = reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4));
+            if (n >= L.N) { *dst = make_uint4(0, 0, 0, 0); continue; }
             const uint4 xq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + (long long)t * L.N + n));
             uint4 sq = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u), bq = make_uint4(0, 0, 0, 0);
             if (L.has_scale) {
@@ -294,10 +265,10 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
                 ow[i] = *reinterpret_cast<const uint32_t *>(&o);
                 acc += xv.x * bv.x + xv.y * bv.y;
             }
-            *reinterpret_cast<uint4 *>(xs + (long long)t * Npad + n) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+            *dst = make_uint4(ow[0], ow[1], ow[2], ow[3]);
         }
     } else {
-        for (int n = threadIdx.x; n < Npad; n += 256) {
+        for (int n = threadIdx.x; n < kb_total * TILE_K; n += 256) {
             float xv = 0.f, sc = 1.f, bi = 0.f;
             if (n < L.N) {
                 xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
@@ -306,7 +277,9 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
                     bi = __half2float(__ldg(L.bias + n));
                 }
             }
-            xs[(long long)t * Npad + n] = __float2half_rn(xv * sc);
+            const int q = n >> 3;
+            *reinterpret_cast<__half *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4) + (n & 7) * 2) =
+                __float2half_rn(xv * sc);
             acc += xv * bi;
         }
     }
@@ -323,14 +296,9 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, int Npad, __
 }
 
 // ---- the GEMM ------------------------------------------------------------------------------------
-template <int CG>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
 {
-    constexpr int B_STAGES = BRing<CG>::STAGES;
-    constexpr int B_STAGE_BYTES = BRing<CG>::STAGE_BYTES;
-    constexpr int B_HALF_BYTES = BRing<CG>::HALF_BYTES;
-    constexpr int TILE_ROWS = TILE_M * CG;                   // output rows of a tile
     extern __shared__ uint8_t smem_raw[];
     const LayerView &L = P.L;
     // carve shared memory; swizzled operand stages need 1024-byte alignment
@@ -338,7 +306,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const uint32_t sA = base;                                   // A_STAGES x 8 KB
-    const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x (32 / CG) KB
+    const uint32_t sB = sA + A_STAGES * A_STAGE_BYTES;          // B_STAGES x 32 KB
     uint8_t *cb2_ptr = sm + A_STAGES * A_STAGE_BYTES + B_STAGES * B_STAGE_BYTES;
     const uint32_t sEpi = smem_addr(cb2_ptr + P.cb2_bytes);     // EPI_WARPS x 2 x 2 KB output staging
     uint8_t *misc = cb2_ptr + P.cb2_bytes + EPI_STAGE_BYTES;
@@ -355,33 +323,23 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // CG = 2: rank of this CTA in its pair; the even CTA (rank 0) issues the MMAs and owns the
-    // barriers the issuing thread waits on (fullA, fullB, accum_empty)
-    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
-    const bool leader = rank == 0;
-
     if (threadIdx.x == 0) {
         for (int s = 0; s < A_STAGES; s++) {
-            mbar_init(bar_fullA(s), 2 * CG);  // one arrival per producer warp of a pair, from every CTA
+            mbar_init(bar_fullA(s), 2);       // one arrival per producer warp of a pair
             mbar_init(bar_emptyA(s), 1);      // tcgen05.commit
         }
         for (int s = 0; s < B_STAGES; s++) {
-            mbar_init(bar_fullB(s), 1);       // the leader's expect_tx arrival
+            mbar_init(bar_fullB(s), 1);       // the expect_tx arrival
             mbar_init(bar_emptyB(s), 1);      // tcgen05.commit
         }
         mbar_init(bar_accum_full, 1);
-        mbar_init(bar_accum_empty, EPI_WARPS * CG);
+        mbar_init(bar_accum_empty, EPI_WARPS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        if (CG == 1) {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        } else {
-            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-        }
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // residual codebook -> shared memory (all threads)
     if (L.k2) {
@@ -401,16 +359,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
-    if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anybody arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // the barriers of the even CTA, as this CTA addresses them
-    auto leader_bar = [&](uint32_t bar) { return CG == 2 ? map_to_cta(bar, 0) : bar; };
-
-    // this worker's share of the (tile, k block) units: [u_begin, u_end), boundaries multiples of
-    // unit_gran; a worker is a CTA (CG = 1) or a CTA pair (CG = 2)
-    const long long n_workers = gridDim.x / CG, worker = blockIdx.x / CG;
+    // this CTA's share of the (tile, k block) units: [u_begin, u_end), boundaries multiples of unit_gran
+    const long long n_workers = gridDim.x, worker = blockIdx.x;
     const long long groups = P.units / P.unit_gran;
     const long long u_begin = groups * worker / n_workers * P.unit_gran;
     const long long u_end = groups * (worker + 1) / n_workers * P.unit_gran;
@@ -423,7 +376,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
     bool ok = true;
 
     if (warp == 0) {
-        // ================= TMA: B tiles (every CTA loads its own share of the tokens) =================
+        // ================= bulk copies: B tiles =================
         if (lane == 0) {
             int it = 0;
             uint32_t s = 0, ps = 1;                              // ring position, parity to wait for
@@ -433,16 +386,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
                 const int halves = (P.B - t0 > MMA_N) ? 2 : 1;
                 for (int kb = kb0; kb < kb1; kb++, it++, s = (s + 1 == B_STAGES ? 0 : s + 1), ps ^= (s == 0 ? 1u : 0u)) {
                     if (!(ok = mbar_wait(bar_emptyB(s), ps, abort_flag, P.status))) break;
-                    if (leader) mbar_expect_tx(bar_fullB(s), CG * halves * B_HALF_BYTES);
-                    for (int h = 0; h < halves; h++) {
-                        const uint32_t dst = sB + s * B_STAGE_BYTES + h * B_HALF_BYTES;
-                        const int tok = t0 + h * MMA_N + (int)rank * (MMA_N / CG);
-                        if (CG == 1) tma_load_2d(dst, &tmap_xs, bar_fullB(s), kb * TILE_K, tok);
-                        else tma_load_2d_pair(dst, &tmap_xs, leader_bar(bar_fullB(s)), kb * TILE_K, tok);
-                    }
+                    mbar_expect_tx(bar_fullB(s), halves * B_HALF_BYTES);
+                    for (int h = 0; h < halves; h++)
+                        bulk_load(sB + s * B_STAGE_BYTES + h * B_HALF_BYTES,
+                                  P.xs + ((long long)(2 * tt + h) * P.kb_total + kb) * B_HALF_BYTES, B_HALF_BYTES, bar_fullB(s));
                 }
             }
-            if (!ok && CG == 1) {
+            if (!ok) {
                 // abandoned: give copies still in flight a bounded time to land before the CTA exits
                 const int first = it > B_STAGES ? it - B_STAGES : 0;
                 for (int j = first; j < it; j++) {
@@ -452,8 +402,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issue (the even CTA issues for the pair) =================
-        if (lane == 0 && leader) {
+        // ================= MMA issue =================
+        if (lane == 0) {
             // One thread runs this loop as a serial instruction chain, so it is kept short: descriptors
             // are a constant plus a stage offset, stage numbers and parities are running counters, and the
             // MMAs of a k block go out in one asm block.
@@ -473,18 +423,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
                     // (stage offsets only touch the 14-bit address field of the descriptors: no carry)
                     const uint64_t ad = adesc0 + (uint64_t)((sa * A_STAGE_BYTES) >> 4);
                     const uint64_t bd = bdesc0 + (uint64_t)((sb * B_STAGE_BYTES) >> 4);
-                    umma_kblock<CG>(tmem_base, ad, bd, kb > kb0 ? 1u : 0u, two_halves, B_HALF_BYTES);
-                    umma_commit<CG>(bar_emptyA(sa));      // the stages may be refilled once these MMAs have read them
-                    umma_commit<CG>(bar_emptyB(sb));
+                    umma_kblock(tmem_base, ad, bd, kb > kb0 ? 1u : 0u, two_halves);
+                    umma_commit(bar_emptyA(sa));      // the stages may be refilled once these MMAs have read them
+                    umma_commit(bar_emptyB(sb));
                     if (++sa == A_STAGES) { sa = 0; pa ^= 1u; }
                     if (++sb == B_STAGES) { sb = 0; pb ^= 1u; }
                 }
-                if (ok) umma_commit<CG>(bar_accum_full);  // accumulators complete
+                if (ok) umma_commit(bar_accum_full);  // accumulators complete
                 seg_no++;
             }
         }
     } else if (warp < 2 + PRODUCER_WARPS) {
-        // ================= dequant producers: A tiles (every CTA its own 128 rows) =================
+        // ================= dequant producers: A tiles =================
         const int pw = warp - 2, pair = pw >> 1, half = pw & 1;
         const int c = lane & 7, grp = lane >> 3;             // row chunk within the 64-row block, 8-column group
         const uint4 *cb1 = reinterpret_cast<const uint4 *>(L.c1);
@@ -494,7 +444,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
         int it0 = 0;                                         // k blocks of earlier segments
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m;
-            const int vrow = mt * (TILE_ROWS / 8) + (int)rank * (TILE_M / 8) + 8 * half + c;
+            const int vrow = mt * (TILE_M / 8) + 8 * half + c;
             const bool row_ok = vrow < L.R;
             const uint8_t *row1 = L.s1.ptr + (long long)vrow * L.s1.stride;
             const uint8_t *row2 = L.k2 ? L.s2.ptr + (long long)vrow * L.s2.stride : nullptr;
@@ -565,10 +515,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
                 __syncwarp();
-                if (lane == 0) {
-                    if (CG == 1) mbar_arrive(bar_fullA(s));
-                    else mbar_arrive_cluster(leader_bar(bar_fullA(s)));
-                }
+                if (lane == 0) mbar_arrive(bar_fullA(s));
             }
             it0 += kb1 - kb0;
         }
@@ -583,7 +530,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m, tt = tile / P.tiles_m;
             const int t0 = tt * TILE_N;
-            const int m = mt * TILE_ROWS + (int)rank * TILE_M + 32 * q + lane;
+            const int m = mt * TILE_M + 32 * q + lane;
             const int t_cnt = min(TILE_N, P.B - t0);
             const bool partial = kb0 != 0 || kb1 != P.kb_total;
             // bias terms of this warp's 256 tokens, loaded before the wait (a load inside the drain would
@@ -602,7 +549,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
                 // output row: conflict free) and one lane hands it to TMA (store, or reduce-add for a partial
                 // tile); two staging buffers per warp, so the copy of one piece overlaps the next.
                 const uint32_t ebuf = sEpi + (uint32_t)(warp - (2 + PRODUCER_WARPS)) * (2 * EPI_BUF_BYTES);
-                const int m0 = mt * TILE_ROWS + (int)rank * TILE_M + 32 * q;
+                const int m0 = mt * TILE_M + 32 * q;
 #pragma unroll
                 for (int ci = 0; ci < MMA_N / 32; ci++) {    // unrolled: bt_chunk[] stays in registers
                     const int c0 = h * MMA_N + 32 * ci;
@@ -674,10 +621,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                if (CG == 1) mbar_arrive(bar_accum_empty);
-                else mbar_arrive_cluster(leader_bar(bar_accum_empty));
-            }
+            if (lane == 0) mbar_arrive(bar_accum_empty);
             seg_no++;
         }
         // the staging buffers must outlive the copies that read them, the copies must land before the end
@@ -685,16 +629,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_xs, const __grid_co
     }
 #undef FOR_EACH_SEGMENT
 
-    // ---- teardown: everybody (of both CTAs) meets, then the allocating warps free TMEM ---------------
+    // ---- teardown: everybody meets, then the allocating warp frees TMEM ---------------
     tc_fence_before();
     __syncwarp();
     __syncthreads();
-    if (CG == 2) cluster_sync_all();          // nobody leaves while its pair may still reach into it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
-        else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
     }
 }
 
@@ -718,8 +660,7 @@ EncodeTiledFn get_encode_fn()
 }
 
 struct GemmPlan {
-    int cg;              // CTAs per tile: 2 = CTA pairs (tcgen05 cta_group::2), 1 = single CTAs
-    int Npad, tiles_m, tiles_t, kb_total, unit_gran, grid, any_partial, cb2_rep, cb2_bytes;
+    int tiles_m, tiles_t, kb_total, unit_gran, grid, any_partial, cb2_rep, cb2_bytes;
     long long units;
     size_t smem;
     long long ws_bytes, off_bterm, off_xs;
@@ -737,55 +678,19 @@ int sm_count()
     return n;
 }
 
-template <int CG>
 size_t gemm_smem_bytes(int cb2_bytes)
 {
-    return 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)BRing<CG>::STAGES * BRing<CG>::STAGE_BYTES + cb2_bytes +
-           EPI_STAGE_BYTES + 8 * (2 * A_STAGES + 2 * BRing<CG>::STAGES + 2) + 16;
+    return 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)B_STAGES * B_STAGE_BYTES + cb2_bytes +
+           EPI_STAGE_BYTES + 8 * (2 * A_STAGES + 2 * B_STAGES + 2) + 16;
 }
 
-// How many CTA pairs of the cta_group::2 kernel the device runs at once (0: cannot).  Asked once.
-int max_active_pairs(int cb2_bytes)
-{
-    static int cached = -1;
-    if (cached >= 0) return cached;
-    int n = 0;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3(2 * sm_count(), 1, 1);
-    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = gemm_smem_bytes<2>(cb2_bytes > 0 ? cb2_bytes : 32768);
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    if (cudaFuncSetAttribute(gemm_tcgen05_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)cfg.dynamicSmemBytes) != cudaSuccess ||
-        cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<2>, &cfg) != cudaSuccess) {
-        (void)cudaGetLastError();
-        n = 0;
-    }
-    cached = n;
-    return cached;
-}
-
-GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
+GemmPlan plan_gemm(const LayerView &L, int B)
 {
     GemmPlan p;
-    const int G = sm_count();
+    int workers = sm_count();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
     p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? CB2_REPLICAS : 1) : 0;
-    // CTA pairs need the device to run (nearly) all its SMs as pairs and a layer with rows for them.
-    // Measured at 512 tokens on the 14336 x 4096 layer: 108 us with pairs, 94 us with single CTAs (the
-    // producers' centroid reads, not the activation traffic that pairs halve, hold the k loop back, and
-    // a pair advances at the pace of the slower of its two CTAs), so single CTAs are the default.
-    p.cg = 1;
-    int workers = G;
-    if ((PREFER_CTA_PAIRS || L.cta_pairs) && query_device && L.M > TILE_M) {
-        const int pairs = max_active_pairs(p.cb2_bytes);
-        if (2 * pairs >= G - 8) { p.cg = 2; workers = pairs; }
-    }
-    p.Npad = (L.N + 7) / 8 * 8;
-    p.tiles_m = ceil_div(L.M, TILE_M * p.cg);
+    p.tiles_m = ceil_div(L.M, TILE_M);
     p.tiles_t = ceil_div(B, TILE_N);
     p.kb_total = ceil_div(L.N, TILE_K);
     p.units = (long long)p.tiles_m * p.tiles_t * p.kb_total;
@@ -793,14 +698,15 @@ GemmPlan plan_gemm(const LayerView &L, int B, bool query_device)
     p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32) ? 1 : p.kb_total;
     const long long groups = p.units / p.unit_gran;
     if (groups < workers) workers = (int)groups;
-    p.grid = workers * p.cg;
+    p.grid = workers;
     p.any_partial = 0;
     for (int c = 1; c < workers; c++)
         if ((groups * c / workers * p.unit_gran) % p.kb_total != 0) p.any_partial = 1;
-    p.smem = p.cg == 2 ? gemm_smem_bytes<2>(p.cb2_bytes) : gemm_smem_bytes<1>(p.cb2_bytes);
+    p.smem = gemm_smem_bytes(p.cb2_bytes);
     p.off_bterm = WS_STATUS_BYTES;
     p.off_xs = p.off_bterm + ((long long)B * 4 + 255) / 256 * 256;
-    p.ws_bytes = p.off_xs + ((long long)B * p.Npad * 2 + 255) / 256 * 256;
+    // activation tile images: whole 256-token halves and whole k blocks
+    p.ws_bytes = p.off_xs + (long long)ceil_div(B, MMA_N) * p.kb_total * B_HALF_BYTES;
     return p;
 }
 
@@ -817,72 +723,50 @@ bool gemm_tcgen05_supported(const LayerView &L, int B)
 }
 
 // (the scratch layout does not depend on the device, so this query makes no CUDA call)
-long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B, false).ws_bytes; }
+long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B).ws_bytes; }
 
 int gemm_tcgen05_launches(const LayerView &, int) { return 2; }   // pre-pass + GEMM
 
 cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
 {
-    const GemmPlan pl = plan_gemm(L, B, true);
+    const GemmPlan pl = plan_gemm(L, B);
     uint8_t *w8 = reinterpret_cast<uint8_t *>(ws);
     int *status = reinterpret_cast<int *>(w8);
     float *bterm = reinterpret_cast<float *>(w8 + pl.off_bterm);
-    __half *xs = reinterpret_cast<__half *>(w8 + pl.off_xs);
-
-    EncodeTiledFn encode = get_encode_fn();
-    if (encode == nullptr) return cudaErrorNotSupported;
-    CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)L.N, (cuuint64_t)B};
-    const cuuint64_t gstride[1] = {(cuuint64_t)pl.Npad * 2};
-    const cuuint32_t box[2] = {TILE_K, (cuuint32_t)(MMA_N / pl.cg)};    // a CTA of a pair loads half the tokens of an MMA
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, xs, gdim, gstride, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    uint8_t *xs = w8 + pl.off_xs;
 
     // FP32 output with 16-byte aligned rows: the epilogue goes through shared memory and TMA
     const int tma_out = (L.out_dtype == VPTQ_DTYPE_FP32 && (L.M & 3) == 0) ? 1 : 0;
-    CUtensorMap tmap_out = tmap;                 // placeholder when unused
+    CUtensorMap tmap_out;
+    memset(&tmap_out, 0, sizeof(tmap_out));      // not read by the kernel when tma_out == 0
     if (tma_out) {
+        EncodeTiledFn encode = get_encode_fn();
+        if (encode == nullptr) return cudaErrorNotSupported;
         const cuuint64_t odim[2] = {(cuuint64_t)L.M, (cuuint64_t)B};
         const cuuint64_t ostride[1] = {(cuuint64_t)L.M * 4};
         const cuuint32_t obox[2] = {32, 16};
-        r = encode(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odim, ostride, obox, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        const cuuint32_t estr[2] = {1, 1};
+        const CUresult r = encode(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, odim, ostride, obox, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
 
     cudaError_t e;
-    gemm_prepass_kernel<<<B, 256, 0, st>>>(L, x, B, pl.Npad, xs, bterm, status,
-                                           pl.any_partial ? reinterpret_cast<float *>(out) : nullptr);
+    gemm_prepass_kernel<<<ceil_div(B, MMA_N) * MMA_N, 256, 0, st>>>(L, x, B, xs, bterm, status,
+                                                                   pl.any_partial ? reinterpret_cast<float *>(out) : nullptr);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     GemmParams P;
-    P.L = L; P.out = out; P.B = B; P.Npad = pl.Npad;
+    P.L = L; P.out = out; P.B = B;
     P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.kb_total = pl.kb_total;
     P.unit_gran = pl.unit_gran; P.units = pl.units;
     P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
-    P.status = status; P.bterm = bterm; P.tma_out = tma_out;
-    if (pl.cg == 1) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-        if (e != cudaSuccess) return e;
-        gemm_tcgen05_kernel<1><<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap, tmap_out, P);
-        return cudaGetLastError();
-    }
-    e = cudaFuncSetAttribute(gemm_tcgen05_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    P.status = status; P.bterm = bterm; P.xs = xs; P.tma_out = tma_out;
+    e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3(pl.grid, 1, 1);
-    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = pl.smem;
-    cfg.stream = st;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<2>, tmap, tmap_out, P);
+    gemm_tcgen05_kernel<<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap_out, P);
+    return cudaGetLastError();
 }
 
 }  // namespace vptq

@@ -34,7 +34,7 @@ int check_desc(const vptq_layer_desc *d)
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
         d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
-    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_CTA_PAIRS)) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC)) return VPTQ_E_UNSUPPORTED;
     if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
     return VPTQ_OK;
 }
@@ -75,7 +75,6 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     L.R0 = L.n_out ? ceil_div(L.M, L.v0) : 0;
     L.has_scale = (d->flags & VPTQ_FLAG_SCALE_BIAS) ? 1 : 0;
     L.scale_rows = (d->flags & VPTQ_FLAG_SCALE_ROWS) ? 1 : 0;
-    L.cta_pairs = (d->flags & VPTQ_FLAG_CTA_PAIRS) ? 1 : 0;
     L.x_bf16 = d->x_dtype == VPTQ_DTYPE_BF16;
     L.out_dtype = d->out_dtype;
     // stream geometry is part of the view even without pointers (path selection reads it)

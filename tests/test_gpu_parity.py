@@ -173,13 +173,10 @@ def test_linear_argument_errors(b):
     (136, 4100, 256, 40, "fp32"),    # few row tiles and many k blocks: K is split, partial sums meet by red.add
     (1024, 512, 256, 1100, "fp32"),  # three token tiles (the last one ragged)
 ])
-@pytest.mark.parametrize("pairs", [False, True], ids=["one_cta", "cta_pairs"])
-def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype, pairs):
+def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
     spec = synth.LayerSpec("g", M, N, v=8, k1=65536, k2=k2, x_dtype="bf16", out_dtype=out_dtype)
     d = synth.make_layer(spec, 76, B % 7, B)
     dl = b.DeviceLayer(d)
-    if pairs:       # two CTAs per 256-row tile (tcgen05 cta_group::2)
-        dl = dl.with_flags(dl.desc.flags | b.FLAG_CTA_PAIRS)
     assert b.vptq_linear_path(dl.desc, B) == "gemm_tcgen05"
     y_ref = oracle.Layer.from_synth(d).linear(d["x"])
     x = dl.upload_x(d["x"])
