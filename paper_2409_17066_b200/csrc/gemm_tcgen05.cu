@@ -29,8 +29,13 @@
 // load the same outgoing path: 117 us).
 // Persistent grid, one CTA per SM.  The work is the list of (tile, k block) units, tile =
 // (token tile, 128-row tile); with an FP32 output every CTA takes an equal, contiguous share of
-// the units, whatever tile they fall in (partial tiles meet in the output by red.add), so all
-// SMs stay busy; other output types are dealt out in whole tiles.
+// the units, whatever tile they fall in, so all SMs stay busy; other output types are dealt out in
+// whole tiles.  When a share is long (FLAG_ORDER_MIN_SHARE k blocks or more) the pieces of a split
+// tile meet in the output without a zero-fill: the piece that holds the tile's last k blocks is the
+// first thing its CTA works on, so it finishes early; it stores and then raises the tile's flag in
+// the workspace; the other pieces (the last thing their CTAs work on) wait for the flag (a bounded
+// wait that is normally over before it starts) and reduce-add.  With short shares all pieces end
+// together, so there the pre-pass clears the output and every piece reduce-adds.
 //
 // Every mbarrier wait is bounded: after about two seconds a waiter records VPTQ_E_TIMEOUT in
 // the status word of the workspace, raises a CTA-wide abort flag and every role leaves its
@@ -67,6 +72,7 @@ constexpr int B_SBO = 512;    // bytes between consecutive 8-token groups of the
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
 
 constexpr int WS_STATUS_BYTES = 256;
+constexpr int FLAG_ORDER_MIN_SHARE = 24;
 
 struct GemmParams {
     LayerView L;
@@ -77,9 +83,11 @@ struct GemmParams {
     long long units;     // tiles_m * tiles_t * kb_total
     int cb2_replicated;
     int cb2_bytes;
+    int flag_order;      // split tiles: 1 = last piece stores and raises a flag, the others wait and add; 0 = all add
     int tma_out;         // FP32 output written by TMA store / reduce from shared memory (needs M % 4 == 0)
     int *status;         // workspace status word
     const float *bterm;  // [B]
+    int *tile_flags;     // [tiles]: epilogue warps that have stored the piece with the tile's last k blocks
     const uint8_t *xs;   // activation tile images, [ceil(B / 256)][kb_total][16 KB]
 };
 
@@ -123,6 +131,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                 return false;
             }
         }
+    }
+}
+
+// Bounded wait until *flag >= target (set by another CTA of this grid; all CTAs of the grid are resident).
+__device__ __forceinline__ bool flag_wait(const int *flag, int target, volatile int *abort_flag, int *status)
+{
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (true) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v >= target) return true;
+        if ((++spins & 63u) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, VPTQ_E_TIMEOUT);
+                return false;
+            }
+        }
+        __nanosleep(64);
     }
 }
 
@@ -210,16 +239,18 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-// ---- pre-pass: xs = fp16(x * s) written as tile images, bterm[t] = sum_n x[t][n] * b[n], status = 0; clears
-//      row t of an FP32 output in which partial tiles are going to meet by red.add (zero_out != nullptr).
+// ---- pre-pass: xs = fp16(x * s) written as tile images, bterm[t] = sum_n x[t][n] * b[n], status = 0, tile
+//      flags = 0; clears row t of an FP32 output in which all pieces of split tiles reduce-add (zero_out != nullptr).
 // Image of the tile half (256 tokens) x (k block of 32 columns): token r, 16-byte chunk q (8 columns) at
 //      (r / 8) * 512 + (r % 8) * 64 + ((q ^ ((r % 8) / 2)) * 16: the K-major 64-byte-swizzled operand layout.
 // One block per token of the padded range; tokens >= B and columns >= N are written as zeros. ---------------
 __global__ void __launch_bounds__(256)
 gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__restrict__ xs,
-                    float *__restrict__ bterm, int *status, float *__restrict__ zero_out)
+                    float *__restrict__ bterm, int *status, int *__restrict__ tile_flags, int n_tiles,
+                    float *__restrict__ zero_out)
 {
     const int t = blockIdx.x;
+    for (int i = t * 256 + threadIdx.x; i < n_tiles; i += gridDim.x * 256) tile_flags[i] = 0;
     const int kb_total = (L.N + TILE_K - 1) / TILE_K;
     // where token t's 64 bytes of k block 0 start; the other k blocks follow at B_HALF_BYTES each
     uint8_t *img_row = xs + (long long)(t / MMA_N) * kb_total * B_HALF_BYTES + ((t % MMA_N) >> 3) * B_SBO + (t & 7) * 64;
@@ -532,7 +563,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
             const int t0 = tt * TILE_N;
             const int m = mt * TILE_M + 32 * q + lane;
             const int t_cnt = min(TILE_N, P.B - t0);
-            const bool partial = kb0 != 0 || kb1 != P.kb_total;
+            // a split tile: the piece with the last k blocks stores and announces it, the others add afterwards
+            const bool split = kb0 != 0 || kb1 != P.kb_total;
+            const bool add = P.flag_order ? kb1 != P.kb_total : split;
+            const bool announce = P.flag_order && kb0 != 0 && kb1 == P.kb_total;
             // bias terms of this warp's 256 tokens, loaded before the wait (a load inside the drain would
             // cost an L2 round trip under load): lane l holds token 32*i + l of chunk i
             float bt_chunk[MMA_N / 32];
@@ -544,6 +578,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
             ok = __all_sync(0xffffffffu, mbar_wait(bar_accum_full, seg_no & 1, abort_flag, P.status));
             if (!ok) break;
             tc_fence_after();
+            if (add && P.flag_order) {
+                ok = __all_sync(0xffffffffu, lane != 0 || flag_wait(P.tile_flags + tile, EPI_WARPS, abort_flag, P.status));
+                if (!ok) break;
+                asm volatile("fence.proxy.async;" ::: "memory");     // the reduce-adds below go through the async proxy
+            }
             if (P.tma_out) {
                 // FP32 output through shared memory: per 16 tokens a warp stages its [16][32] piece (lane =
                 // output row: conflict free) and one lane hands it to TMA (store, or reduce-add for a partial
@@ -575,7 +614,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
                             asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + j * 128u + lane * 4u), "r"(r[j]) : "memory");
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
-                        if (lane == 0 && m0 < L.M) tma_store_2d(&tmap_out, buf, m0, t0 + c1, partial);
+                        if (lane == 0 && m0 < L.M) tma_store_2d(&tmap_out, buf, m0, t0 + c1, add);
                         epi_piece++;
                     }
                 }
@@ -597,7 +636,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
                     if (fp32_out) {
                         // one element per token row; independent addresses, no serial pointer chain
                         float *p = reinterpret_cast<float *>(P.out) + (long long)(t0 + c0) * L.M + m;
-                        if (nt == 32 && !partial) {
+                        if (nt == 32 && !add) {
 #pragma unroll
                             for (int j = 0; j < 32; j++) p[(unsigned)j * Mu] = __uint_as_float(r[j]);
                         } else if (nt == 32) {
@@ -607,7 +646,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
 #pragma unroll
                             for (int j = 0; j < 32; j++) {
                                 if (j < nt) {
-                                    if (!partial) p[(unsigned)j * Mu] = __uint_as_float(r[j]);
+                                    if (!add) p[(unsigned)j * Mu] = __uint_as_float(r[j]);
                                     else atomicAdd(p + (unsigned)j * Mu, __uint_as_float(r[j]));
                                 }
                             }
@@ -622,6 +661,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_accum_empty);
+            if (announce) {
+                // this warp's part of the tile is in memory before the flag counts it
+                if (lane == 0) {
+                    if (P.tma_out) {
+                        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                    }
+                    __threadfence();
+                    atomicAdd(P.tile_flags + tile, 1);
+                }
+            }
             seg_no++;
         }
         // the staging buffers must outlive the copies that read them, the copies must land before the end
@@ -660,10 +710,10 @@ EncodeTiledFn get_encode_fn()
 }
 
 struct GemmPlan {
-    int tiles_m, tiles_t, kb_total, unit_gran, grid, any_partial, cb2_rep, cb2_bytes;
+    int tiles_m, tiles_t, kb_total, unit_gran, grid, any_split, flag_order, cb2_rep, cb2_bytes;
     long long units;
     size_t smem;
-    long long ws_bytes, off_bterm, off_xs;
+    long long ws_bytes, off_flags, off_bterm, off_xs;
 };
 
 int sm_count()
@@ -694,16 +744,18 @@ GemmPlan plan_gemm(const LayerView &L, int B)
     p.tiles_t = ceil_div(B, TILE_N);
     p.kb_total = ceil_div(L.N, TILE_K);
     p.units = (long long)p.tiles_m * p.tiles_t * p.kb_total;
-    // partial tiles meet in an FP32 output by red.add; other output types get whole tiles
+    // the pieces of a split tile meet in an FP32 output by red.add; other output types get whole tiles
     p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32) ? 1 : p.kb_total;
     const long long groups = p.units / p.unit_gran;
     if (groups < workers) workers = (int)groups;
     p.grid = workers;
-    p.any_partial = 0;
+    p.any_split = 0;
     for (int c = 1; c < workers; c++)
-        if ((groups * c / workers * p.unit_gran) % p.kb_total != 0) p.any_partial = 1;
+        if ((groups * c / workers * p.unit_gran) % p.kb_total != 0) p.any_split = 1;
+    p.flag_order = (p.any_split && p.units / workers >= FLAG_ORDER_MIN_SHARE) ? 1 : 0;
     p.smem = gemm_smem_bytes(p.cb2_bytes);
-    p.off_bterm = WS_STATUS_BYTES;
+    p.off_flags = WS_STATUS_BYTES;
+    p.off_bterm = p.off_flags + ((long long)p.tiles_m * p.tiles_t * 4 + 255) / 256 * 256;
     p.off_xs = p.off_bterm + ((long long)B * 4 + 255) / 256 * 256;
     // activation tile images: whole 256-token halves and whole k blocks
     p.ws_bytes = p.off_xs + (long long)ceil_div(B, MMA_N) * p.kb_total * B_HALF_BYTES;
@@ -732,6 +784,7 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     const GemmPlan pl = plan_gemm(L, B);
     uint8_t *w8 = reinterpret_cast<uint8_t *>(ws);
     int *status = reinterpret_cast<int *>(w8);
+    int *tile_flags = reinterpret_cast<int *>(w8 + pl.off_flags);
     float *bterm = reinterpret_cast<float *>(w8 + pl.off_bterm);
     uint8_t *xs = w8 + pl.off_xs;
 
@@ -753,8 +806,9 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     }
 
     cudaError_t e;
-    gemm_prepass_kernel<<<ceil_div(B, MMA_N) * MMA_N, 256, 0, st>>>(L, x, B, xs, bterm, status,
-                                                                   pl.any_partial ? reinterpret_cast<float *>(out) : nullptr);
+    gemm_prepass_kernel<<<ceil_div(B, MMA_N) * MMA_N, 256, 0, st>>>(
+        L, x, B, xs, bterm, status, tile_flags, pl.tiles_m * pl.tiles_t,
+        (pl.any_split && !pl.flag_order) ? reinterpret_cast<float *>(out) : nullptr);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     GemmParams P;
@@ -762,7 +816,7 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     P.tiles_m = pl.tiles_m; P.tiles_t = pl.tiles_t; P.kb_total = pl.kb_total;
     P.unit_gran = pl.unit_gran; P.units = pl.units;
     P.cb2_replicated = pl.cb2_rep; P.cb2_bytes = pl.cb2_bytes;
-    P.status = status; P.bterm = bterm; P.xs = xs; P.tma_out = tma_out;
+    P.status = status; P.bterm = bterm; P.xs = xs; P.tile_flags = tile_flags; P.flag_order = pl.flag_order; P.tma_out = tma_out;
     e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
     gemm_tcgen05_kernel<<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap_out, P);

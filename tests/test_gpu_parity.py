@@ -172,6 +172,8 @@ def test_linear_argument_errors(b):
     (264, 1030, 256, 300, "fp16"),   # residual codebook, both token halves, ragged everything
     (136, 4100, 256, 40, "fp32"),    # few row tiles and many k blocks: K is split, partial sums meet by red.add
     (1024, 512, 256, 1100, "fp32"),  # three token tiles (the last one ragged)
+    (1100, 13000, 256, 24, "fp32"),  # long shares of k blocks: the last piece of a split tile stores and raises
+                                     # the tile's flag, the other pieces wait for it and reduce-add
 ])
 def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
     spec = synth.LayerSpec("g", M, N, v=8, k1=65536, k2=k2, x_dtype="bf16", out_dtype=out_dtype)
