@@ -115,6 +115,9 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Wait until the preceding kernel of the stream (the pre-pass) has completed and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Bounded wait.  Returns false when the wait was abandoned (timeout here or abort raised elsewhere).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
@@ -127,6 +130,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1;
+                grid_dependency_wait();                  // the pre-pass clears the status word
                 atomicExch(status, VPTQ_E_TIMEOUT);
                 return false;
             }
@@ -147,6 +151,7 @@ __device__ __forceinline__ bool flag_wait(const int *flag, int target, volatile 
             if (*abort_flag) return false;
             if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1;
+                grid_dependency_wait();                  // the pre-pass clears the status word
                 atomicExch(status, VPTQ_E_TIMEOUT);
                 return false;
             }
@@ -244,19 +249,25 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
 // Image of the tile half (256 tokens) x (k block of 32 columns): token r, 16-byte chunk q (8 columns) at
 //      (r / 8) * 512 + (r % 8) * 64 + ((q ^ ((r % 8) / 2)) * 16: the K-major 64-byte-swizzled operand layout.
 // One block per token of the padded range; tokens >= B and columns >= N are written as zeros. ---------------
-__global__ void __launch_bounds__(256)
+constexpr int PRE_THREADS = 128;   // with 32 registers a block fits beside a resident GEMM CTA
+
+__global__ void __launch_bounds__(PRE_THREADS)
 gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__restrict__ xs,
                     float *__restrict__ bterm, int *status, int *__restrict__ tile_flags, int n_tiles,
                     float *__restrict__ zero_out)
 {
+    // the GEMM is launched as a programmatic dependent: its CTAs may become resident and run their set-up and
+    // first centroid reads as soon as every block of this grid has started; whatever reads this kernel's
+    // output waits for the whole grid (griddepcontrol.wait) first
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int t = blockIdx.x;
-    for (int i = t * 256 + threadIdx.x; i < n_tiles; i += gridDim.x * 256) tile_flags[i] = 0;
+    for (int i = t * PRE_THREADS + threadIdx.x; i < n_tiles; i += gridDim.x * PRE_THREADS) tile_flags[i] = 0;
     const int kb_total = (L.N + TILE_K - 1) / TILE_K;
     // where token t's 64 bytes of k block 0 start; the other k blocks follow at B_HALF_BYTES each
     uint8_t *img_row = xs + (long long)(t / MMA_N) * kb_total * B_HALF_BYTES + ((t % MMA_N) >> 3) * B_SBO + (t & 7) * 64;
     const int sw = (t & 7) >> 1;
     if (t >= B) {
-        for (int q = threadIdx.x; q < 4 * kb_total; q += 256)
+        for (int q = threadIdx.x; q < 4 * kb_total; q += PRE_THREADS)
             *reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
         return;
     }
@@ -265,15 +276,15 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
         float *row = zero_out + (long long)t * L.M;
         if ((L.M & 3) == 0) {
             float4 *r4 = reinterpret_cast<float4 *>(row);          // rows of M floats start 16-byte aligned
-            for (int i = threadIdx.x; i < (L.M >> 2); i += 256) r4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = threadIdx.x; i < (L.M >> 2); i += PRE_THREADS) r4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         } else {
-            for (int i = threadIdx.x; i < L.M; i += 256) row[i] = 0.f;
+            for (int i = threadIdx.x; i < L.M; i += PRE_THREADS) row[i] = 0.f;
         }
     }
     float acc = 0.f;
     if ((L.N & 7) == 0) {
         // 8 columns = one chunk per thread and step, 128-bit loads and stores
-        for (int n = 8 * threadIdx.x; n < kb_total * TILE_K; n += 8 * 256) {
+        for (int n = 8 * threadIdx.x; n < kb_total * TILE_K; n += 8 * PRE_THREADS) {
             const int q = n >> 3;
             uint4 *dst = reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4));
             if (n >= L.N) { *dst = make_uint4(0, 0, 0, 0); continue; }
@@ -299,7 +310,7 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
             *dst = make_uint4(ow[0], ow[1], ow[2], ow[3]);
         }
     } else {
-        for (int n = threadIdx.x; n < kb_total * TILE_K; n += 256) {
+        for (int n = threadIdx.x; n < kb_total * TILE_K; n += PRE_THREADS) {
             float xv = 0.f, sc = 1.f, bi = 0.f;
             if (n < L.N) {
                 xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
@@ -314,14 +325,14 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
             acc += xv * bi;
         }
     }
-    __shared__ float red[8];
+    __shared__ float red[PRE_THREADS / 32];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
     __syncthreads();
     if (threadIdx.x == 0) {
         float a = 0.f;
-        for (int w = 0; w < 8; w++) a += red[w];
+        for (int w = 0; w < PRE_THREADS / 32; w++) a += red[w];
         bterm[t] = a;
     }
 }
@@ -409,6 +420,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
     if (warp == 0) {
         // ================= bulk copies: B tiles =================
         if (lane == 0) {
+            grid_dependency_wait();                              // the tile images are the pre-pass's output
             int it = 0;
             uint32_t s = 0, ps = 1;                              // ring position, parity to wait for
             FOR_EACH_SEGMENT {
@@ -558,6 +570,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_out, GemmParams P)
         const unsigned Mu = (unsigned)L.M;
         int seg_no = 0;
         unsigned epi_piece = 0;                                  // staged pieces so far (buffer parity)
+        grid_dependency_wait();                                  // bias terms, tile flags and a cleared output come from the pre-pass
         FOR_EACH_SEGMENT {
             const int mt = tile % P.tiles_m, tt = tile / P.tiles_m;
             const int t0 = tt * TILE_N;
@@ -806,7 +819,7 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     }
 
     cudaError_t e;
-    gemm_prepass_kernel<<<ceil_div(B, MMA_N) * MMA_N, 256, 0, st>>>(
+    gemm_prepass_kernel<<<ceil_div(B, MMA_N) * MMA_N, PRE_THREADS, 0, st>>>(
         L, x, B, xs, bterm, status, tile_flags, pl.tiles_m * pl.tiles_t,
         (pl.any_split && !pl.flag_order) ? reinterpret_cast<float *>(out) : nullptr);
     e = cudaGetLastError();
@@ -819,8 +832,17 @@ cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *
     P.status = status; P.bterm = bterm; P.xs = xs; P.tile_flags = tile_flags; P.flag_order = pl.flag_order; P.tma_out = tma_out;
     e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    gemm_tcgen05_kernel<<<pl.grid, GEMM_THREADS, pl.smem, st>>>(tmap_out, P);
-    return cudaGetLastError();
+    // programmatic dependent launch: set-up and the producers' first reads overlap the pre-pass
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(pl.grid, 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel, tmap_out, P);
 }
 
 }  // namespace vptq
