@@ -249,7 +249,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
 // Image of the tile half (256 tokens) x (k block of 32 columns): token r, 16-byte chunk q (8 columns) at
 //      (r / 8) * 512 + (r % 8) * 64 + ((q ^ ((r % 8) / 2)) * 16: the K-major 64-byte-swizzled operand layout.
 // One block per token of the padded range; tokens >= B and columns >= N are written as zeros. ---------------
-constexpr int PRE_THREADS = 128;   // with 32 registers a block fits beside a resident GEMM CTA
+constexpr int PRE_THREADS = 128;
 
 __global__ void __launch_bounds__(PRE_THREADS)
 gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__restrict__ xs,
@@ -283,31 +283,46 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
     }
     float acc = 0.f;
     if ((L.N & 7) == 0) {
-        // 8 columns = one chunk per thread and step, 128-bit loads and stores
-        for (int n = 8 * threadIdx.x; n < kb_total * TILE_K; n += 8 * PRE_THREADS) {
-            const int q = n >> 3;
-            uint4 *dst = reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4));
-            if (n >= L.N) { *dst = make_uint4(0, 0, 0, 0); continue; }
-            const uint4 xq = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + (long long)t * L.N + n));
-            uint4 sq = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u), bq = make_uint4(0, 0, 0, 0);
-            if (L.has_scale) {
-                sq = __ldg(reinterpret_cast<const uint4 *>(L.scale + n));
-                bq = __ldg(reinterpret_cast<const uint4 *>(L.bias + n));
-            }
-            const uint32_t xw[4] = {xq.x, xq.y, xq.z, xq.w}, sw[4] = {sq.x, sq.y, sq.z, sq.w}, bw[4] = {bq.x, bq.y, bq.z, bq.w};
-            uint32_t ow[4];
+        // 8 columns = one chunk per thread and step, 128-bit loads and stores; the loads of four steps are
+        // issued together (a thread with one load in flight at a time leaves the memory system idle)
+        constexpr int UNROLL = 4;
+        const uint4 one = make_uint4(0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u), zero = make_uint4(0, 0, 0, 0);
+        for (int n0 = 8 * threadIdx.x; n0 < kb_total * TILE_K; n0 += UNROLL * 8 * PRE_THREADS) {
+            uint4 xq[UNROLL], sq[UNROLL], bq[UNROLL];
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-                float2 xv;
-                if (L.x_bf16) xv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xw[i]));
-                else xv = __half22float2(*reinterpret_cast<const __half2 *>(&xw[i]));
-                const float2 sv = __half22float2(*reinterpret_cast<const __half2 *>(&sw[i]));
-                const float2 bv = __half22float2(*reinterpret_cast<const __half2 *>(&bw[i]));
-                const __half2 o = __floats2half2_rn(xv.x * sv.x, xv.y * sv.y);
-                ow[i] = *reinterpret_cast<const uint32_t *>(&o);
-                acc += xv.x * bv.x + xv.y * bv.y;
+            for (int u = 0; u < UNROLL; u++) {
+                const int n = n0 + u * 8 * PRE_THREADS;
+                xq[u] = zero; sq[u] = one; bq[u] = zero;
+                if (n < L.N) {
+                    xq[u] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + (long long)t * L.N + n));
+                    if (L.has_scale) {
+                        sq[u] = __ldg(reinterpret_cast<const uint4 *>(L.scale + n));
+                        bq[u] = __ldg(reinterpret_cast<const uint4 *>(L.bias + n));
+                    }
+                }
             }
-            *dst = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+#pragma unroll
+            for (int u = 0; u < UNROLL; u++) {
+                const int n = n0 + u * 8 * PRE_THREADS;
+                if (n >= kb_total * TILE_K) break;
+                const uint32_t xw[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w}, sc[4] = {sq[u].x, sq[u].y, sq[u].z, sq[u].w},
+                               bw[4] = {bq[u].x, bq[u].y, bq[u].z, bq[u].w};
+                uint32_t ow[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {       // columns >= N were loaded as zeros: they store zeros and add nothing
+                    float2 xv;
+                    if (L.x_bf16) xv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xw[i]));
+                    else xv = __half22float2(*reinterpret_cast<const __half2 *>(&xw[i]));
+                    const float2 sv = __half22float2(*reinterpret_cast<const __half2 *>(&sc[i]));
+                    const float2 bv = __half22float2(*reinterpret_cast<const __half2 *>(&bw[i]));
+                    const __half2 o = __floats2half2_rn(xv.x * sv.x, xv.y * sv.y);
+                    ow[i] = *reinterpret_cast<const uint32_t *>(&o);
+                    acc += xv.x * bv.x + xv.y * bv.y;
+                }
+                const int q = n >> 3;
+                *reinterpret_cast<uint4 *>(img_row + (long long)(q >> 2) * B_HALF_BYTES + (((q & 3) ^ sw) << 4)) =
+                    make_uint4(ow[0], ow[1], ow[2], ow[3]);
+            }
         }
     } else {
         for (int n = threadIdx.x; n < kb_total * TILE_K; n += PRE_THREADS) {
