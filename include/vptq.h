@@ -157,6 +157,27 @@ int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
                 const vptq_layer_ptrs *p, void *out,
                 void *workspace, size_t workspace_bytes, void *stream);
 
+/* Several layers that read the SAME activations in one call (the q/k/v projections of an attention
+ * block, the gate/up projections of an MLP; the paper's decode loop, App. D.2, runs them one after
+ * the other): out_l = x * W_hat_l^T for l < n_layers <= VPTQ_MAX_FUSED_LAYERS.
+ *   descs, ptrs  host arrays of n_layers descriptors / pointer sets; all layers have the same N and
+ *                x_dtype (else VPTQ_E_SHAPE); M, codebooks, scale/bias and out_dtype are per layer
+ *   outs         host array of n_layers DEVICE pointers, outs[l] = [B][M_l] row-major
+ * When every layer takes the "decode_l2_fma" path (B <= 16) and whole vector rows of the layers spread
+ * evenly over the SMs, one kernel per token group serves all layers (no launch, prologue and ragged
+ * tail per layer; no scratch); otherwise the layers run one after the other on `stream`, sharing the
+ * workspace.  vptq_linear_fused_path() names which: "fused_decode_l2_fma" or "one_by_one".  Each
+ * layer's result is the one vptq_linear gives for it (same arithmetic, same summation order within a
+ * vector row).  Errors as for vptq_linear; nothing is launched when an argument is rejected. */
+#define VPTQ_MAX_FUSED_LAYERS 4
+int64_t vptq_linear_fused_workspace_bytes(const vptq_layer_desc *descs, int32_t n_layers, int32_t B);
+int vptq_linear_fused(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
+                      const void *x, int32_t B, void *const *outs,
+                      void *workspace, size_t workspace_bytes, void *stream);
+const char *vptq_linear_fused_path(const vptq_layer_desc *descs, int32_t n_layers, int32_t B);
+/* Number of kernels one vptq_linear_fused call launches. */
+int vptq_linear_fused_launches(const vptq_layer_desc *descs, int32_t n_layers, int32_t B);
+
 /* Same product with HOST activations and HOST result: copies x_host -> x_dev, runs
  * vptq_linear, copies out_dev -> out_host, all asynchronously on `stream` (the caller
  * synchronises the stream before reading out_host).  x_host/out_host should be pinned

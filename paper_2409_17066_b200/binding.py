@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from typing import Dict, Optional
+from typing import Dict, Optional, Sequence
 
 import numpy as np
 import torch
@@ -62,6 +62,11 @@ EXPORTS = {
     "vptq_linear_workspace_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                               C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "vptq_linear_fused_workspace_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32, C.c_int32]),
+    "vptq_linear_fused": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_int32, C.c_void_p, C.c_int32,
+                                    C.POINTER(C.c_void_p), C.c_void_p, C.c_size_t, C.c_void_p]),
+    "vptq_linear_fused_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32, C.c_int32]),
+    "vptq_linear_fused_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32, C.c_int32]),
     "vptq_linear_host_io": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                       C.c_void_p]),
@@ -169,6 +174,41 @@ def vptq_linear(desc: LayerDesc, x: torch.Tensor, ptrs: LayerPtrs, out: torch.Te
     _check(lib.vptq_linear(C.byref(desc), _ptr(x), B, C.byref(ptrs), _ptr(out),
                            _ptr(workspace), ws_bytes, _stream()))
     return out
+
+
+def _desc_array(descs: Sequence[LayerDesc]):
+    return (LayerDesc * len(descs))(*descs)
+
+
+def vptq_linear_fused_workspace_bytes(descs: Sequence[LayerDesc], B: int) -> int:
+    n = lib.vptq_linear_fused_workspace_bytes(_desc_array(descs), len(descs), B)
+    if n < 0:
+        raise VptqError(int(n))
+    return n
+
+
+def vptq_linear_fused(descs: Sequence[LayerDesc], ptrs: Sequence[LayerPtrs], x: torch.Tensor,
+                      outs: Sequence[torch.Tensor], workspace: Optional[torch.Tensor]) -> Sequence[torch.Tensor]:
+    """Several layers over the same activations in one call (q/k/v, gate/up)."""
+    n = len(descs)
+    assert len(ptrs) == n and len(outs) == n
+    B = x.shape[0]
+    assert x.is_cuda and x.is_contiguous() and tuple(x.shape) == (B, descs[0].N)
+    for d, o in zip(descs, outs):
+        assert o.is_cuda and o.is_contiguous() and tuple(o.shape) == (B, d.M) and o.dtype == _TORCH_DT[d.out_dtype]
+    out_ptrs = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vptq_linear_fused(_desc_array(descs), (LayerPtrs * n)(*ptrs), n, _ptr(x), B, out_ptrs,
+                                 _ptr(workspace), ws_bytes, _stream()))
+    return outs
+
+
+def vptq_linear_fused_path(descs: Sequence[LayerDesc], B: int) -> str:
+    return lib.vptq_linear_fused_path(_desc_array(descs), len(descs), B).decode()
+
+
+def vptq_linear_fused_launches(descs: Sequence[LayerDesc], B: int) -> int:
+    return lib.vptq_linear_fused_launches(_desc_array(descs), len(descs), B)
 
 
 def vptq_linear_host_io(desc: LayerDesc, x_host: torch.Tensor, ptrs: LayerPtrs, out_host: torch.Tensor,

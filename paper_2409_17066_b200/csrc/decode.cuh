@@ -18,6 +18,10 @@ bool l2_fma_supported(const LayerView &L, int B);
 long long l2_fma_workspace_bytes(const LayerView &L, int B);
 int l2_fma_launches(const LayerView &L, int B);
 cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
+// ... several layers that read the same activations in one launch per token group (no scratch)
+bool l2_fma_fused_supported(const LayerView *Ls, int n, int B);
+int l2_fma_fused_launches(int B);
+cudaError_t launch_decode_l2_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st);
 
 // codebooks in global memory, any even v <= 16, group-wise codebooks, FP32 FMAs, no scratch
 bool gl_fma_supported(const LayerView &L, int B);

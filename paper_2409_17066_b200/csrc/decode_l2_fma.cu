@@ -21,6 +21,10 @@
 //   balanced tasks are dealt out regardless of rows: partial sums meet in an FP32 scratch array
 //            through atomic adds, and a task counter per block of 16 vector rows tells which warp
 //            completed the block and so converts and stores it.
+// Fused launch (FUSED): up to MAX_FUSED layers that read the same activations (q/k/v, gate/up) in one
+// OWNER-mode grid; the CTAs are dealt out to the layers in proportion to their vector rows and each
+// CTA works on one layer exactly as in a launch of its own.  Small layers no longer pay a launch,
+// a prologue and a ragged tail each.
 #include "common.cuh"
 #include "decode.cuh"
 
@@ -32,11 +36,14 @@ constexpr int RB_ROWS = 16;                 // vector rows per completion counte
 constexpr int XS_BUDGET = 64 * 1024;        // bytes of staged activations per CTA
 constexpr int PART_BUDGET = 32 * 1024;      // bytes of per-row partial sums per CTA (OWNER mode)
 constexpr int WARPS_TB4 = 16;               // 4 tokens per launch need 128 registers per thread
+constexpr int MAX_FUSED = 4;                // layers of one fused launch
 
 struct L2FmaParams {
-    LayerView L;
+    LayerView L[MAX_FUSED];
+    void *out[MAX_FUSED];
+    int cta_begin[MAX_FUSED + 1];   // FUSED: layer l is the work of CTAs [cta_begin[l], cta_begin[l + 1])
+    int n_layers;
     const void *x;
-    void *out;
     int B;                 // tokens in this launch (<= TB)
     int slab_cols;         // columns per slab (multiple of 256); one slab of x*s is staged at a time
     int n_slabs;
@@ -80,13 +87,21 @@ __device__ __forceinline__ void act8_to_float(uint4 q, int is_bf16, float (&f)[8
     }
 }
 
-template <int TB, bool RES, bool OWNER, int WARPS>
+template <int TB, bool RES, bool OWNER, int WARPS, bool FUSED>
 __global__ void __launch_bounds__(WARPS * 32, 1)
-decode_l2_fma_kernel(L2FmaParams P)
+decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
 {
+    static_assert(!FUSED || OWNER, "a fused launch hands whole vector rows to CTAs");
     constexpr int THREADS = WARPS * 32;
     extern __shared__ __align__(16) uint8_t smem[];
-    const LayerView &L = P.L;
+    // the layer this CTA works on, and its place among that layer's CTAs
+    int li = 0;
+    if (FUSED)
+        while (li + 1 < P.n_layers && (int)blockIdx.x >= P.cta_begin[li + 1]) li++;
+    const LayerView &L = P.L[FUSED ? li : 0];
+    void *const out = P.out[FUSED ? li : 0];
+    const int bid = FUSED ? (int)blockIdx.x - P.cta_begin[li] : (int)blockIdx.x;
+    const int gdim = FUSED ? P.cta_begin[li + 1] - P.cta_begin[li] : (int)gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     __half *xs = reinterpret_cast<__half *>(smem);                                   // [TB][slab_cols]
@@ -96,11 +111,11 @@ decode_l2_fma_kernel(L2FmaParams P)
     float *part = reinterpret_cast<float *>(cb2 + (RES ? (size_t)L.k2 * (P.cb2_replicated ? 8 : 1) : 0));
 
     // rows of this CTA (OWNER) / rank among the CTAs of its slab (balanced)
-    const int r0 = OWNER ? (int)((long long)L.R * blockIdx.x / gridDim.x) : 0;
-    const int r1 = OWNER ? (int)((long long)L.R * (blockIdx.x + 1) / gridDim.x) : L.R;
-    const int my_slab = OWNER ? 0 : blockIdx.x % P.n_slabs;
-    const int grank = OWNER ? 0 : blockIdx.x / P.n_slabs;
-    const int gsize = OWNER ? 1 : (gridDim.x - my_slab + P.n_slabs - 1) / P.n_slabs;
+    const int r0 = OWNER ? (int)((long long)L.R * bid / gdim) : 0;
+    const int r1 = OWNER ? (int)((long long)L.R * (bid + 1) / gdim) : L.R;
+    const int my_slab = OWNER ? 0 : bid % P.n_slabs;
+    const int grank = OWNER ? 0 : bid / P.n_slabs;
+    const int gsize = OWNER ? 1 : (gdim - my_slab + P.n_slabs - 1) / P.n_slabs;
 
     // ---- residual codebook -> shared memory; clear the partial sums -----------------------------------
     if (RES) {
@@ -348,7 +363,7 @@ decode_l2_fma_kernel(L2FmaParams P)
                     for (int i = lane; i < n_m * P.B; i += 32) {
                         const int tt = i / n_m, mm = m_lo + i % n_m;
                         const float y = __ldcg(P.yacc + (long long)tt * L.M + mm) + bterm[tt];
-                        store_out(P.out, (long long)tt * L.M + mm, y, L.out_dtype);
+                        store_out(out, (long long)tt * L.M + mm, y, L.out_dtype);
                     }
                 }
             }
@@ -365,7 +380,7 @@ decode_l2_fma_kernel(L2FmaParams P)
         for (int i = threadIdx.x; i < n_m * P.B; i += THREADS) {
             const int t = i / n_m, ml = i % n_m;       // consecutive threads -> consecutive m
             const float y = part[((ml >> 3) * TB + t) * 8 + (ml & 7)] + bterm[t];
-            store_out(P.out, (long long)t * L.M + m_lo + ml, y, L.out_dtype);
+            store_out(out, (long long)t * L.M + m_lo + ml, y, L.out_dtype);
         }
     }
 }
@@ -374,6 +389,7 @@ struct L2Plan {
     int slab_cols, n_slabs, chunks_total, cb2_rep, grid, owner, part_floats, warps;
     size_t smem;
     long long ws_bytes, off_counters;
+    int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
 int l2_num_sms()
@@ -422,13 +438,62 @@ L2Plan plan_l2(const LayerView &L, int TB)
 
 int token_group(int B) { return B >= 4 ? 4 : (B >= 2 ? 2 : 1); }
 
-template <int TB, bool RES, bool OWNER, int WARPS>
+// A fused launch: the SMs are dealt out to the layers in proportion to their vector rows (every layer at
+// least one; leftover SMs go where the most rows per CTA remain).  False when the layers cannot share a
+// launch or whole rows would leave the SMs unevenly loaded.
+bool plan_l2_fused(const LayerView *Ls, int n, int TB, L2Plan *out)
+{
+    if (n < 2 || n > MAX_FUSED) return false;
+    for (int l = 1; l < n; l++)
+        if (Ls[l].N != Ls[0].N || Ls[l].x_bf16 != Ls[0].x_bf16 || Ls[l].k2 != Ls[0].k2) return false;
+    L2Plan p = plan_l2(Ls[0], TB);          // slab geometry, warps, residual table: functions of N, k2, TB
+    const int G = l2_num_sms();
+    long long rows = 0;
+    for (int l = 0; l < n; l++) rows += Ls[l].R;
+    if (rows < G) return false;
+    int ctas[MAX_FUSED], used = 0;
+    for (int l = 0; l < n; l++) {
+        ctas[l] = (int)((long long)G * Ls[l].R / rows);
+        if (ctas[l] < 1) ctas[l] = 1;
+        used += ctas[l];
+    }
+    if (used > G) return false;
+    for (; used < G; used++) {
+        int best = 0;
+        for (int l = 1; l < n; l++)
+            if ((long long)ceil_div(Ls[l].R, ctas[l]) * ctas[best] > (long long)ceil_div(Ls[best].R, ctas[best]) * ctas[l] ||
+                ceil_div(Ls[l].R, ctas[l]) > ceil_div(Ls[best].R, ctas[best]))
+                best = l;
+        ctas[best]++;
+    }
+    int rows_cta = 0;
+    p.cta_begin[0] = 0;
+    for (int l = 0; l < n; l++) {
+        rows_cta = rows_cta > ceil_div(Ls[l].R, ctas[l]) ? rows_cta : ceil_div(Ls[l].R, ctas[l]);
+        p.cta_begin[l + 1] = p.cta_begin[l] + ctas[l];
+    }
+    const double eff_cta = (double)rows / ((double)G * rows_cta);
+    const long long t_cta = (long long)rows_cta * (p.slab_cols / 256);
+    const double eff_warp = (double)t_cta / ((double)p.warps * (double)((t_cta + p.warps - 1) / p.warps));
+    p.part_floats = rows_cta * TB * 8;
+    if (eff_cta * eff_warp < 0.80 || (long long)p.part_floats * 4 > PART_BUDGET) return false;
+    p.owner = 1;
+    p.grid = G;
+    p.smem = (size_t)TB * p.slab_cols * 2 + 4 * 4 + (size_t)p.warps * 4 * 4 +
+             (size_t)Ls[0].k2 * 16 * (p.cb2_rep ? 8 : 1) + (size_t)p.part_floats * 4;
+    p.ws_bytes = 0;
+    p.off_counters = 0;
+    *out = p;
+    return true;
+}
+
+template <int TB, bool RES, bool OWNER, int WARPS, bool FUSED>
 cudaError_t launch_one(const L2FmaParams &P, const L2Plan &pl, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB, RES, OWNER, WARPS>,
+    cudaError_t e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    decode_l2_fma_kernel<TB, RES, OWNER, WARPS><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
+    decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -437,7 +502,9 @@ cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, in
                          void *ws, cudaStream_t st)
 {
     L2FmaParams P;
-    P.L = L; P.x = x; P.out = out; P.B = Bg;
+    memset(&P, 0, sizeof(P));
+    P.L[0] = L; P.out[0] = out; P.n_layers = 1; P.cta_begin[1] = pl.grid;
+    P.x = x; P.B = Bg;
     P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.chunks_total = pl.chunks_total;
     P.cb2_replicated = pl.cb2_rep; P.part_floats = pl.part_floats;
     P.yacc = nullptr; P.counters = nullptr;
@@ -448,8 +515,24 @@ cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, in
         if (e != cudaSuccess) return e;
     }
     const bool res = L.k2 > 0;
-    if (pl.owner) return res ? launch_one<TB, true, true, WARPS>(P, pl, st) : launch_one<TB, false, true, WARPS>(P, pl, st);
-    return res ? launch_one<TB, true, false, WARPS>(P, pl, st) : launch_one<TB, false, false, WARPS>(P, pl, st);
+    if (pl.owner) return res ? launch_one<TB, true, true, WARPS, false>(P, pl, st) : launch_one<TB, false, true, WARPS, false>(P, pl, st);
+    return res ? launch_one<TB, true, false, WARPS, false>(P, pl, st) : launch_one<TB, false, false, WARPS, false>(P, pl, st);
+}
+
+template <int TB, int WARPS>
+cudaError_t launch_group_fused(const LayerView *Ls, int n, const L2Plan &pl, const void *x, int Bg, void *const *outs,
+                               cudaStream_t st)
+{
+    L2FmaParams P;
+    memset(&P, 0, sizeof(P));
+    for (int l = 0; l < n; l++) { P.L[l] = Ls[l]; P.out[l] = outs[l]; }
+    for (int l = 0; l <= n; l++) P.cta_begin[l] = pl.cta_begin[l];
+    P.n_layers = n;
+    P.x = x; P.B = Bg;
+    P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.chunks_total = pl.chunks_total;
+    P.cb2_replicated = pl.cb2_rep; P.part_floats = pl.part_floats;
+    P.yacc = nullptr; P.counters = nullptr;
+    return Ls[0].k2 > 0 ? launch_one<TB, true, true, WARPS, true>(P, pl, st) : launch_one<TB, false, true, WARPS, true>(P, pl, st);
 }
 
 }  // namespace
@@ -490,6 +573,41 @@ cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void 
         if (TB == 4) e = launch_group<4, WARPS_TB4>(L, pl, xg, Bg, og, ws, st);
         else if (TB == 2) e = launch_group<2, 32>(L, pl, xg, Bg, og, ws, st);
         else e = launch_group<1, 32>(L, pl, xg, Bg, og, ws, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+bool l2_fma_fused_supported(const LayerView *Ls, int n, int B)
+{
+    if (B < 1 || B > 16) return false;
+    for (int l = 0; l < n; l++)
+        if (!l2_fma_supported(Ls[l], B)) return false;
+    L2Plan pl;
+    return plan_l2_fused(Ls, n, token_group(B), &pl);
+}
+
+int l2_fma_fused_launches(int B)
+{
+    const int TB = token_group(B);
+    return (B + TB - 1) / TB;
+}
+
+cudaError_t launch_decode_l2_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st)
+{
+    const int TB = token_group(B);
+    L2Plan pl;
+    if (!plan_l2_fused(Ls, n, TB, &pl)) return cudaErrorInvalidValue;
+    for (int t0 = 0; t0 < B; t0 += TB) {
+        const int Bg = (B - t0 < TB) ? (B - t0) : TB;
+        const void *xg = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * Ls[0].N * 2;
+        void *og[MAX_FUSED];
+        for (int l = 0; l < n; l++)
+            og[l] = reinterpret_cast<uint8_t *>(outs[l]) + (size_t)t0 * Ls[l].M * (Ls[l].out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
+        cudaError_t e;
+        if (TB == 4) e = launch_group_fused<4, WARPS_TB4>(Ls, n, pl, xg, Bg, og, st);
+        else if (TB == 2) e = launch_group_fused<2, 32>(Ls, n, pl, xg, Bg, og, st);
+        else e = launch_group_fused<1, 32>(Ls, n, pl, xg, Bg, og, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

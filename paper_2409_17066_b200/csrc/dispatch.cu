@@ -89,4 +89,47 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
     return e == cudaSuccess ? VPTQ_OK : VPTQ_E_CUDA;
 }
 
+// ---- several layers that read the same activations ---------------------------------------------------
+
+bool fused_path_available(const LayerView *Ls, const int *flags, int n, int B)
+{
+    if (n < 2 || B > DECODE_MAX_B) return false;
+    for (int l = 0; l < n; l++)
+        if (choose_path(Ls[l], B, flags[l]) != PATH_DECODE_L2_FMA) return false;
+    return l2_fma_fused_supported(Ls, n, B);
+}
+
+long long linear_fused_workspace_bytes(const LayerView *Ls, const int *flags, int n, int B)
+{
+    if (fused_path_available(Ls, flags, n, B)) return 0;
+    long long need = 0;       // one layer after the other on the stream: they share the scratch
+    for (int l = 0; l < n; l++) {
+        const long long w = linear_workspace_bytes(Ls[l], B, flags[l]);
+        if (w > need) need = w;
+    }
+    return need;
+}
+
+int linear_fused_launches(const LayerView *Ls, const int *flags, int n, int B)
+{
+    if (fused_path_available(Ls, flags, n, B)) return l2_fma_fused_launches(B);
+    int total = 0;
+    for (int l = 0; l < n; l++) total += linear_launches(Ls[l], B, flags[l]);
+    return total;
+}
+
+int linear_fused_dispatch(const LayerView *Ls, const int *flags, int n, const void *x, int B, void *const *outs,
+                          void *ws, cudaStream_t st, cudaError_t *cuda_err)
+{
+    if (fused_path_available(Ls, flags, n, B)) {
+        *cuda_err = launch_decode_l2_fma_fused(Ls, n, x, B, outs, st);
+        return *cuda_err == cudaSuccess ? VPTQ_OK : VPTQ_E_CUDA;
+    }
+    for (int l = 0; l < n; l++) {
+        const int rc = linear_dispatch(Ls[l], flags[l], x, B, outs[l], ws, st, cuda_err);
+        if (rc != VPTQ_OK) return rc;
+    }
+    return VPTQ_OK;
+}
+
 }  // namespace vptq

@@ -210,6 +210,78 @@ int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
     return rc;
 }
 
+// descriptors (and pointers) of a fused call -> views; VPTQ_OK or the first error
+static int fused_views(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers, int32_t B,
+                       LayerView *Ls, int *flags)
+{
+    if (descs == nullptr) return VPTQ_E_NULL;
+    if (n_layers < 1 || n_layers > VPTQ_MAX_FUSED_LAYERS || B <= 0) return VPTQ_E_SHAPE;
+    for (int l = 0; l < n_layers; l++) {
+        int rc = check_desc(&descs[l]);
+        if (rc != VPTQ_OK) return rc;
+        if (descs[l].N != descs[0].N || descs[l].x_dtype != descs[0].x_dtype) return VPTQ_E_SHAPE;
+        if (ptrs != nullptr) {
+            rc = check_ptrs(&descs[l], &ptrs[l]);
+            if (rc != VPTQ_OK) return rc;
+        }
+        Ls[l] = make_view(&descs[l], ptrs != nullptr ? &ptrs[l] : nullptr);
+        flags[l] = descs[l].flags;
+    }
+    return VPTQ_OK;
+}
+
+int64_t vptq_linear_fused_workspace_bytes(const vptq_layer_desc *descs, int32_t n_layers, int32_t B)
+{
+    LayerView Ls[VPTQ_MAX_FUSED_LAYERS];
+    int flags[VPTQ_MAX_FUSED_LAYERS];
+    const int rc = fused_views(descs, nullptr, n_layers, B, Ls, flags);
+    if (rc != VPTQ_OK) return rc;
+    return linear_fused_workspace_bytes(Ls, flags, n_layers, B);
+}
+
+int vptq_linear_fused(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
+                      const void *x, int32_t B, void *const *outs,
+                      void *workspace, size_t workspace_bytes, void *stream)
+{
+    LayerView Ls[VPTQ_MAX_FUSED_LAYERS];
+    int flags[VPTQ_MAX_FUSED_LAYERS];
+    if (ptrs == nullptr || outs == nullptr || x == nullptr) return VPTQ_E_NULL;
+    const int rc = fused_views(descs, ptrs, n_layers, B, Ls, flags);
+    if (rc != VPTQ_OK) return rc;
+    if (!aligned16(x)) return VPTQ_E_ALIGN;
+    for (int l = 0; l < n_layers; l++) {
+        if (outs[l] == nullptr) return VPTQ_E_NULL;
+        if (!aligned16(outs[l])) return VPTQ_E_ALIGN;
+    }
+    const long long need = linear_fused_workspace_bytes(Ls, flags, n_layers, B);
+    if (need > 0) {
+        if (workspace == nullptr || (long long)workspace_bytes < need) return VPTQ_E_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return VPTQ_E_ALIGN;
+    }
+    cudaError_t e = cudaSuccess;
+    const int rc2 = linear_fused_dispatch(Ls, flags, n_layers, x, B, outs, workspace,
+                                          reinterpret_cast<cudaStream_t>(stream), &e);
+    if (rc2 == VPTQ_E_CUDA) return cuda_fail(e);
+    return rc2;
+}
+
+int vptq_linear_fused_launches(const vptq_layer_desc *descs, int32_t n_layers, int32_t B)
+{
+    LayerView Ls[VPTQ_MAX_FUSED_LAYERS];
+    int flags[VPTQ_MAX_FUSED_LAYERS];
+    const int rc = fused_views(descs, nullptr, n_layers, B, Ls, flags);
+    if (rc != VPTQ_OK) return rc;
+    return linear_fused_launches(Ls, flags, n_layers, B);
+}
+
+const char *vptq_linear_fused_path(const vptq_layer_desc *descs, int32_t n_layers, int32_t B)
+{
+    LayerView Ls[VPTQ_MAX_FUSED_LAYERS];
+    int flags[VPTQ_MAX_FUSED_LAYERS];
+    if (fused_views(descs, nullptr, n_layers, B, Ls, flags) != VPTQ_OK) return "invalid";
+    return fused_path_available(Ls, flags, n_layers, B) ? "fused_decode_l2_fma" : "one_by_one";
+}
+
 int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
                         const vptq_layer_ptrs *p, void *out_host,
                         void *x_dev, void *out_dev,

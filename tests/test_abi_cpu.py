@@ -89,3 +89,32 @@ def test_argument_errors_need_no_gpu(binding):
     assert b.lib.vptq_status_string(b.E_ALIGN).decode().startswith("a data pointer")
     assert b.vptq_linear_path(d, 1) in ("generic", "decode_smem_fma", "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05")
     assert b.vptq_linear_launches(d, 1) >= 1
+
+
+def test_fused_call_argument_errors_and_path_names(binding):
+    b = binding
+    q = b.make_desc(8192, 8192, 8, 65536, 256)
+    kv = b.make_desc(1024, 8192, 8, 65536, 256)
+    arr = (b.LayerDesc * 3)(q, kv, kv)
+    assert b.lib.vptq_linear_fused_workspace_bytes(None, 3, 1) == b.E_NULL
+    assert b.lib.vptq_linear_fused_workspace_bytes(arr, 0, 1) == b.E_SHAPE
+    assert b.lib.vptq_linear_fused_workspace_bytes(arr, 5, 1) == b.E_SHAPE
+    assert b.lib.vptq_linear_fused_workspace_bytes(arr, 3, 0) == b.E_SHAPE
+    other_n = (b.LayerDesc * 2)(q, b.make_desc(1024, 4096, 8, 65536, 256))
+    assert b.lib.vptq_linear_fused_workspace_bytes(other_n, 2, 1) == b.E_SHAPE
+    assert b.lib.vptq_linear_fused(arr, None, 3, None, 1, None, None, 0, None) == b.E_NULL
+    # three projections of an attention block over the same input: one launch, no scratch
+    assert b.vptq_linear_fused_path([q, kv, kv], 1) == "fused_decode_l2_fma"
+    assert b.vptq_linear_fused_workspace_bytes([q, kv, kv], 1) == 0
+    assert b.vptq_linear_fused_launches([q, kv, kv], 1) == 1
+    assert b.vptq_linear_fused_launches([q, kv, kv], 6) == 2          # token groups of 4
+    # layers that take another kernel family run one after the other and share the scratch
+    small = b.make_desc(11008, 4096, 6, 4096, 256, n_outlier=41, v0=4, k0=4096)
+    assert b.vptq_linear_fused_path([small, small], 1) == "one_by_one"
+    assert b.vptq_linear_fused_launches([small, small], 1) == 2 * b.vptq_linear_launches(small, 1)
+    # a single layer, or many tokens, is not fused either
+    assert b.vptq_linear_fused_path([q], 1) == "one_by_one"
+    assert b.vptq_linear_fused_path([q, kv], 64) == "one_by_one"
+    assert b.vptq_linear_fused_workspace_bytes([q, kv], 64) == max(b.vptq_linear_workspace_bytes(q, 64),
+                                                                  b.vptq_linear_workspace_bytes(kv, 64))
+

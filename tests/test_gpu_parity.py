@@ -190,3 +190,51 @@ def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
     g = dl.with_flags(dl.desc.flags | b.FLAG_FORCE_GENERIC)
     yg = g.linear(x).float().cpu().numpy()
     assert rel_err(y.float().cpu().numpy(), yg.astype(np.float64)) <= TOL
+
+
+# ------------------------------------------------------------------ several layers over the same activations
+
+def _fused_case(b, specs, B, seed):
+    ds = [synth.make_layer(sp, seed + 7 * i, 3, B) for i, sp in enumerate(specs)]
+    for d in ds[1:]:
+        d["x"] = ds[0]["x"]                                  # the layers of a fused call read the same x
+    dls = [b.DeviceLayer(d) for d in ds]
+    x = dls[0].upload_x(ds[0]["x"])
+    descs = [dl.desc for dl in dls]
+    outs = [torch.full((B, dl.spec.M), float("nan"), dtype=b._TORCH_DT[dl.desc.out_dtype], device="cuda") for dl in dls]
+    need = b.vptq_linear_fused_workspace_bytes(descs, B)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda") if need else None
+    b.vptq_linear_fused(descs, [dl.ptrs for dl in dls], x, outs, ws)
+    return ds, dls, x, outs
+
+
+@pytest.mark.parametrize("Ms,N,k2,B,out_dtypes", [
+    ((4096, 1024, 1024), 4096, 256, 1, ("fp16", "fp16", "fp16")),   # q/k/v shaped
+    ((4100, 1000, 1024), 4096, 256, 3, ("fp32", "fp16", "fp16")),   # ragged rows, 3 tokens, mixed output types
+    ((2048, 2048), 4096, 0, 5, ("fp16", "fp16")),                   # gate/up shaped, no residual, two token groups
+    ((2900, 600), 4360, 256, 2, ("fp16", "fp32")),                  # ragged rows and a ragged last chunk of columns
+])
+def test_linear_fused_matches_oracle_and_single_calls(b, Ms, N, k2, B, out_dtypes):
+    specs = [synth.LayerSpec("f%d" % i, M, N, v=8, k1=65536, k2=k2, x_dtype="bf16", out_dtype=od)
+             for i, (M, od) in enumerate(zip(Ms, out_dtypes))]
+    ds, dls, x, outs = _fused_case(b, specs, B, 311)
+    assert b.vptq_linear_fused_path([dl.desc for dl in dls], B) == "fused_decode_l2_fma"
+    tb = 4 if B >= 4 else 2 if B >= 2 else 1                 # tokens per launch
+    assert b.vptq_linear_fused_launches([dl.desc for dl in dls], B) == (B + tb - 1) // tb
+    for d, dl, y in zip(ds, dls, outs):
+        y = y.float().cpu().numpy()
+        assert np.isfinite(y).all()
+        assert rel_err(y, oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+        y1 = dl.linear(x).float().cpu().numpy()              # the layer's own launch: same arithmetic
+        assert rel_err(y, y1.astype(np.float64)) <= 1e-3 * TOL + (4e-3 if dl.desc.out_dtype != b.DTYPE_FP32 else 0)
+
+
+def test_linear_fused_runs_other_kernel_families_one_by_one(b):
+    spec = {sp.name: sp for sp in synth.small_specs()}["s_v6_full"]
+    specs = [spec, spec]
+    B = 2
+    ds, dls, x, outs = _fused_case(b, specs, B, 17)
+    assert b.vptq_linear_fused_path([dl.desc for dl in dls], B) == "one_by_one"
+    for d, y in zip(ds, outs):
+        assert rel_err(y.float().cpu().numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+
