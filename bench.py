@@ -55,7 +55,10 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
 }
 
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
-                   "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel"}
+                   "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel",
+                   "fused_decode_l2_fma": "decode_l2_fma_kernel"}
+# projections of a decoder layer that read the same activations
+FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
 
 
 def read_traffic(kernel: str, algorithmic_bytes_per_launch: float):
@@ -220,17 +223,37 @@ def run_ours(args):
         l.extend(l[0].clone_streams() for _ in range(copies - 1))
     xs = [layers[i][0].upload_x(xs_np[i]) for i in range(len(layers))]
     outs = [torch.empty((B, l[0].spec.M), dtype=vb._TORCH_DT[l[0].desc.out_dtype], device="cuda") for l in layers]
-    launches_per_step = sum(vb.vptq_linear_launches(l[0].desc, B) for l in layers)
-    paths = sorted({vb.vptq_linear_path(l[0].desc, B) for l in layers})
+    # calls of a step: projections that read the same activations (q/k/v, gate/up) go through one
+    # vptq_linear_fused call where the library serves them with one launch, the rest through vptq_linear
+    calls, li = [], 0
+    names = [l[0].spec.name for l in layers]
+    while li < len(layers):
+        group = next((g for g in FUSE_GROUPS if tuple(names[li:li + len(g)]) == g), None)
+        if group is not None and not args.no_fuse and \
+                vb.vptq_linear_fused_path([layers[j][0].desc for j in range(li, li + len(group))], B) == "fused_decode_l2_fma":
+            idx = list(range(li, li + len(group)))
+            calls.append((idx, [vb.FusedLayers([layers[j][c] for j in idx]) for c in range(copies)]))
+        else:
+            idx = [li]
+            calls.append((idx, None))
+        li += len(idx)
+    call_names = ["+".join(names[j] for j in idx) + f"_{idx[0]}" for idx, _ in calls]
+    launches_per_step = sum(f[0].launches(B) if f is not None else vb.vptq_linear_launches(layers[idx[0]][0].desc, B)
+                            for idx, f in calls)
+    paths = sorted({f[0].path(B) if f is not None else vb.vptq_linear_path(layers[idx[0]][0].desc, B)
+                    for idx, f in calls})
 
     def step(i, events=None):
         c = i % copies
-        for li, l in enumerate(layers):
+        for ci, (idx, fused) in enumerate(calls):
             if events is not None:
-                events[li][0].record()
-            l[c].linear(xs[li], outs[li])
+                events[ci][0].record()
+            if fused is not None:
+                fused[c].linear(xs[idx[0]], [outs[j] for j in idx])     # the group's common input
+            else:
+                layers[idx[0]][c].linear(xs[idx[0]], outs[idx[0]])
             if events is not None:
-                events[li][1].record()
+                events[ci][1].record()
 
     def barrier():
         if world > 1:
@@ -249,7 +272,7 @@ def run_ours(args):
     # per-call events on every `stride`-th step only (at most ~200 steps), to keep the stream tight
     stride = max(1, args.steps // 200)
     per_call = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                 for _ in layers] if i % stride == 0 else None for i in range(args.steps)]
+                 for _ in calls] if i % stride == 0 else None for i in range(args.steps)]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
@@ -271,13 +294,13 @@ def run_ours(args):
     # per-launch durations of the dominant kernel (all seven calls run the same kernel family)
     call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call if pc is not None]
     n_ev = len(call_ms)
-    layer_ms = [statistics.mean(call_ms[i][li] for i in range(n_ev)) for li in range(len(layers))]
+    layer_ms = [statistics.mean(call_ms[i][ci] for i in range(n_ev)) for ci in range(len(calls))]
     kern_ms_per_step = sum(layer_ms)
     achieved = step_bytes / (kern_ms_per_step * 1e-3) / 1e9
-    per_layer = {layers[li][0].spec.name + f"_{li}": {
-        "us": 1e3 * layer_ms[li],
-        "GBps": layers[li][0].weight_bytes() / (1e-3 * layer_ms[li]) / 1e9}
-        for li in range(len(layers))}
+    per_layer = {call_names[ci]: {
+        "us": 1e3 * layer_ms[ci],
+        "GBps": sum(layers[j][0].weight_bytes() for j in calls[ci][0]) / (1e-3 * layer_ms[ci]) / 1e9}
+        for ci in range(len(calls))}
 
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     xh = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in xs_np]
@@ -285,10 +308,17 @@ def run_ours(args):
     h2d = sum(x.numel() * x.element_size() for x in xh)
     d2h = sum(o.numel() * o.element_size() for o in oh)
 
+    # (a fused call copies its common input once)
+    h2d = sum(xh[idx[0]].numel() * xh[idx[0]].element_size() for idx, _ in calls)
+
     def step_e2e(i):
         c = i % copies
-        for li, l in enumerate(layers):
-            vb.vptq_linear_host_io(l[c].desc, xh[li], l[c].ptrs, oh[li], xs[li], outs[li], l[c].workspace(B))
+        for idx, fused in calls:
+            if fused is not None:
+                fused[c].linear_host_io(xh[idx[0]], [oh[j] for j in idx], xs[idx[0]], [outs[j] for j in idx])
+            else:
+                l = layers[idx[0]][c]
+                vb.vptq_linear_host_io(l.desc, xh[idx[0]], l.ptrs, oh[idx[0]], xs[idx[0]], outs[idx[0]], l.workspace(B))
         torch.cuda.synchronize()     # the step's result is on the host
 
     for i in range(3):
@@ -309,12 +339,13 @@ def run_ours(args):
     e2e_value = world * step_bytes / (e2e_ms * 1e-3) / 1e9
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "us_per_call_mean": 1e3 * ms_step / len(layers),
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "us_per_call_mean": 1e3 * ms_step / len(calls),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": WORKLOAD if default_case else
                        f"config{cfg_id}_{'+'.join(l[0].spec.name for l in layers)}_B{B} (profiling case, not the headline workload)",
-                       "batch": B, "calls_per_step": len(layers),
+                       "batch": B, "linear_layers_per_step": len(layers), "calls_per_step": len(calls),
+                       "calls": call_names,
                        "compressed_bytes_per_step": step_bytes, "kernel_paths": paths,
                        "l2": f"inputs larger than L2: {copies} copies of the {step_bytes / 1e6:.0f} MB index streams walked alternately",
                        "multi_gpu": "replicas only (no sharding, no collective)"},
@@ -455,6 +486,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-fuse", action="store_true", help="one vptq_linear call per layer (no vptq_linear_fused)")
     ap.add_argument("--cfg", type=int, default=WORKLOAD_CFG,
                     help="workload number (default: the headline workload); others are profiling cases")
     ap.add_argument("--layers", default="", help="comma-separated layer names to keep (profiling cases)")

@@ -188,6 +188,13 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
                         void *x_dev, void *out_dev,
                         void *workspace, size_t workspace_bytes, void *stream);
 
+/* vptq_linear_fused with HOST activations and HOST results: one copy of x_host -> x_dev, the fused
+ * call, one copy outs_dev[l] -> outs_host[l] per layer, all asynchronous on `stream`. */
+int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
+                              const void *x_host, int32_t B, void *const *outs_host,
+                              void *x_dev, void *const *outs_dev,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- the same product for callers that cannot allocate device memory ---------------- */
 
 /* The paper has no counterpart to this entry point; it exists for integration reasons only.

@@ -67,6 +67,9 @@ EXPORTS = {
                                     C.POINTER(C.c_void_p), C.c_void_p, C.c_size_t, C.c_void_p]),
     "vptq_linear_fused_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32, C.c_int32]),
     "vptq_linear_fused_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32, C.c_int32]),
+    "vptq_linear_fused_host_io": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_int32, C.c_void_p, C.c_int32,
+                                            C.POINTER(C.c_void_p), C.c_void_p, C.POINTER(C.c_void_p), C.c_void_p,
+                                            C.c_size_t, C.c_void_p]),
     "vptq_linear_host_io": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                       C.c_void_p]),
@@ -328,3 +331,48 @@ class DeviceLayer:
         if out is None:
             out = torch.empty((B, self.spec.M), dtype=_TORCH_DT[self.desc.out_dtype], device=self.device)
         return vptq_linear(self.desc, x, self.ptrs, out, self.workspace(B))
+
+
+class FusedLayers:
+    """Several DeviceLayers that read the same activations (q/k/v, gate/up): keeps the argument arrays of
+    vptq_linear_fused so that a call costs no more host time than vptq_linear."""
+
+    def __init__(self, dls: Sequence[DeviceLayer]):
+        self.dls = list(dls)
+        self.n = len(self.dls)
+        self.descs = _desc_array([d.desc for d in self.dls])
+        self.ptrs = (LayerPtrs * self.n)(*[d.ptrs for d in self.dls])
+        self._ws: Dict[int, Optional[torch.Tensor]] = {}
+
+    def path(self, B: int) -> str:
+        return lib.vptq_linear_fused_path(self.descs, self.n, B).decode()
+
+    def launches(self, B: int) -> int:
+        return lib.vptq_linear_fused_launches(self.descs, self.n, B)
+
+    def workspace(self, B: int) -> Optional[torch.Tensor]:
+        if B not in self._ws:
+            need = lib.vptq_linear_fused_workspace_bytes(self.descs, self.n, B)
+            if need < 0:
+                raise VptqError(int(need))
+            self._ws[B] = torch.empty(need, dtype=torch.uint8, device=self.dls[0].device) if need else None
+        return self._ws[B]
+
+    def linear(self, x: torch.Tensor, outs: Sequence[torch.Tensor]) -> Sequence[torch.Tensor]:
+        B = x.shape[0]
+        ws = self.workspace(B)
+        out_ptrs = (C.c_void_p * self.n)(*[o.data_ptr() for o in outs])
+        _check(lib.vptq_linear_fused(self.descs, self.ptrs, self.n, _ptr(x), B, out_ptrs, _ptr(ws),
+                                     0 if ws is None else ws.numel(), _stream()))
+        return outs
+
+    def linear_host_io(self, x_host: torch.Tensor, outs_host: Sequence[torch.Tensor], x_dev: torch.Tensor,
+                       outs_dev: Sequence[torch.Tensor]) -> Sequence[torch.Tensor]:
+        B = x_host.shape[0]
+        ws = self.workspace(B)
+        oh = (C.c_void_p * self.n)(*[o.data_ptr() for o in outs_host])
+        od = (C.c_void_p * self.n)(*[o.data_ptr() for o in outs_dev])
+        _check(lib.vptq_linear_fused_host_io(self.descs, self.ptrs, self.n, _ptr(x_host), B, oh, _ptr(x_dev), od,
+                                             _ptr(ws), 0 if ws is None else ws.numel(), _stream()))
+        return outs_host
+

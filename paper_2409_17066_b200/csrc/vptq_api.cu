@@ -303,6 +303,32 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
     return VPTQ_OK;
 }
 
+int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
+                              const void *x_host, int32_t B, void *const *outs_host,
+                              void *x_dev, void *const *outs_dev,
+                              void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (descs == nullptr || x_host == nullptr || outs_host == nullptr || x_dev == nullptr || outs_dev == nullptr)
+        return VPTQ_E_NULL;
+    if (n_layers < 1 || n_layers > VPTQ_MAX_FUSED_LAYERS || B <= 0) return VPTQ_E_SHAPE;
+    for (int l = 0; l < n_layers; l++) {
+        const int rc = check_desc(&descs[l]);
+        if (rc != VPTQ_OK) return rc;
+        if (outs_host[l] == nullptr || outs_dev[l] == nullptr) return VPTQ_E_NULL;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)B * descs[0].N * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int rc = vptq_linear_fused(descs, ptrs, n_layers, x_dev, B, outs_dev, workspace, workspace_bytes, stream);
+    if (rc != VPTQ_OK) return rc;
+    for (int l = 0; l < n_layers; l++) {
+        const size_t ob = (size_t)B * descs[l].M * (descs[l].out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
+        e = cudaMemcpyAsync(outs_host[l], outs_dev[l], ob, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return VPTQ_OK;
+}
+
 const char *vptq_status_string(int code)
 {
     switch (code) {
