@@ -46,8 +46,8 @@ def read_peaks():
 # in proportion to the packed index streams, so it is scaled by the bytes a launch processes).
 # An entry is removed (-> null in the output) when its kernel changes after the capture.
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
-    # profiles/decode_l2_fma_kernel_config3_gate_proj_B1.md: (89.22 + 2.77) MB DRAM / 89.24 MB algorithmic
-    "decode_l2_fma_kernel": 1.031,
+    # profiles/decode_l2_fma_kernel_config3_gate_up_fused_B1.md: (178.44 + 3.68) MB DRAM / 178.33 MB algorithmic
+    "decode_l2_fma_kernel": 1.021,
     # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.95 MB
     "decode_smem_fma_kernel": 1.003,
     # profiles/decode_smem_mma_kernel_config2_gate_proj_B8.md: 19.09 MB / 19.0 MB
