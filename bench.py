@@ -117,6 +117,30 @@ def dist_env():
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
+# Replicas only: every rank runs the whole workload on weights of its own, nothing crosses ranks but
+# the timing.  The three helpers below are all there is to the N > 1 path.
+
+def replica_layer_ordinal(li: int, rank: int) -> int:
+    """Seed ordinal of layer `li` on replica `rank` (every replica has weights of its own)."""
+    return li + 100 * rank
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's time (all ranks get it)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbps(step_bytes_per_rank: float, world: int, ms_step_max: float) -> float:
+    """Bytes all replicas processed per step over the slowest replica's step time."""
+    return world * step_bytes_per_rank / (ms_step_max * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------------------ reference arm
 
 def oracle_sample_rate(layers_np, rows_per_layer, B=1):
@@ -210,7 +234,7 @@ def run_ours(args):
     for li, spec in enumerate(cfg["layers"]):
         if keep is not None and spec.name not in keep:
             continue
-        d = synth.make_layer(spec, cfg_id, li + 100 * rank, B)
+        d = synth.make_layer(spec, cfg_id, replica_layer_ordinal(li, rank), B)
         dl = vb.DeviceLayer(d)
         layers.append([dl])
         xs_np.append(d["x"])
@@ -283,13 +307,9 @@ def run_ours(args):
     ms_total = ev0.elapsed_time(ev1)
     time.sleep(0.2)
     clocks = sampler.stop()
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, "cuda")
     ms_step = ms_total / args.steps
-    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    value = whole_job_gbps(step_bytes, world, ms_step)
 
     # per-launch durations of the dominant kernel (all seven calls run the same kernel family)
     call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call if pc is not None]
@@ -331,12 +351,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / args.steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * step_bytes / (e2e_ms * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
+    e2e_value = whole_job_gbps(step_bytes, world, e2e_ms)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "us_per_call_mean": 1e3 * ms_step / len(calls),
