@@ -47,8 +47,9 @@ def unpack(packed: np.ndarray, rows: int, cols: int, k: int) -> np.ndarray:
 
 
 def dequant(M, N, v, c1, idx1, c2=None, idx2=None, n_out=0, v0=0, c0=None, idx0=None,
-            scale=None, bias=None, scale_axis=0, n_groups=1) -> np.ndarray:
-    """float16 [M][N] from integer index matrices and float16 tables."""
+            scale=None, bias=None, scale_axis=0, n_groups=1, col_perm=None) -> np.ndarray:
+    """float16 [M][N] from integer index matrices and float16 tables.  col_perm (Sec. 3.2.3): stored column j
+    is column col_perm[j] of the result."""
     W = np.zeros((M, N), dtype=np.float32)
     m = np.arange(M)
     if n_out < N:
@@ -75,7 +76,12 @@ def dequant(M, N, v, c1, idx1, c2=None, idx2=None, n_out=0, v0=0, c0=None, idx0=
             W = (W * s[:, None]).astype(np.float32)
             W = (W + bb[:, None]).astype(np.float32)
     with np.errstate(over="ignore"):
-        return W.astype(np.float16)
+        W16 = W.astype(np.float16)
+    if col_perm is None:
+        return W16
+    out = np.empty_like(W16)
+    out[:, np.asarray(col_perm)] = W16
+    return out
 
 
 def linear(W16: np.ndarray, x_f64: np.ndarray) -> np.ndarray:
@@ -86,4 +92,5 @@ def linear(W16: np.ndarray, x_f64: np.ndarray) -> np.ndarray:
 def dequant_from_synth(d, scale_axis=0) -> np.ndarray:
     s = d["spec"]
     return dequant(s.M, s.N, s.v, d["c1"], d["idx1"], d["c2"], d["idx2"], s.n_out, s.v0,
-                   d["c0"], d["idx0"], d["scale"], d["bias"], scale_axis, getattr(s, "n_groups", 1))
+                   d["c0"], d["idx0"], d["scale"], d["bias"], scale_axis, getattr(s, "n_groups", 1),
+                   d.get("col_perm"))

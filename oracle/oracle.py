@@ -28,7 +28,7 @@ class _Layer(C.Structure):
                 ("idx1", C.c_void_p), ("c1", C.c_void_p),
                 ("idx2", C.c_void_p), ("c2", C.c_void_p),
                 ("idx0", C.c_void_p), ("c0", C.c_void_p),
-                ("scale", C.c_void_p), ("bias", C.c_void_p)]
+                ("scale", C.c_void_p), ("bias", C.c_void_p), ("col_perm", C.c_void_p)]
 
 
 _lib.oracle_half_to_float.restype = C.c_float
@@ -120,7 +120,7 @@ class Layer:
 
     def __init__(self, M, N, v, k1, c1, idx1_packed, k2=0, c2=None, idx2_packed=None,
                  n_out=0, v0=0, k0=0, c0=None, idx0_packed=None,
-                 scale=None, bias=None, scale_axis=0, n_groups=1):
+                 scale=None, bias=None, scale_axis=0, n_groups=1, col_perm=None):
         def u16(a):
             return None if a is None else np.ascontiguousarray(a).view(np.uint16).reshape(-1).copy()
 
@@ -143,10 +143,14 @@ class Layer:
         if has_scale:
             assert self._keep["scale"].size == (M if scale_axis else N)
             assert self._keep["bias"].size == (M if scale_axis else N)
+        # stored column j is input feature col_perm[j] (Sec. 3.2.3: outlier columns lie where the quantizer found them)
+        self._keep["col_perm"] = None if col_perm is None else np.ascontiguousarray(col_perm, dtype=np.int32).copy()
+        if col_perm is not None:
+            assert self._keep["col_perm"].shape == (N,)
         p = lambda n: (self._keep[n].ctypes.data if self._keep[n] is not None else None)
         self.c = _Layer(M, N, v, k1, k2, n_out, v0, k0, int(has_scale), scale_axis, G,
                         p("idx1"), p("c1"), p("idx2"), p("c2"), p("idx0"), p("c0"),
-                        p("scale"), p("bias"))
+                        p("scale"), p("bias"), p("col_perm"))
 
     @classmethod
     def from_synth(cls, d, scale_axis=0):
@@ -157,7 +161,7 @@ class Layer:
                    n_out=s.n_out, v0=s.v0, k0=s.k0, c0=d["c0"],
                    idx0_packed=pack(d["idx0"], s.k0) if s.n_out else None,
                    scale=d["scale"], bias=d["bias"], scale_axis=scale_axis,
-                   n_groups=getattr(s, "n_groups", 1))
+                   n_groups=getattr(s, "n_groups", 1), col_perm=d.get("col_perm"))
 
     def dequant(self) -> np.ndarray:
         """W16 [M][N] as numpy float16 (bit-exact definition of the restored weight)."""

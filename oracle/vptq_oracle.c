@@ -19,14 +19,20 @@
  *   - outlier columns use their own table with their own vector length
  *     (Sec. 3.2.3; App. C.1 "Parameter Description"), and have no residual stage
  *     (Algorithm 2 order; index-bit formula of App. C.2);
+ *   - which columns are outlier columns is the quantizer's choice (Sec. 3.2.3: the
+ *     columns with the largest Hessian diagonal; Algorithm 2 "selects outlier
+ *     columns"), so they may lie anywhere in the matrix: the layer may carry a
+ *     column order, col_perm, that says which input feature each stored column is;
  *   - the weights are restored to FP16 and then multiplied (App. D.2).
  *   - size accounting: compression ratio / equivalent bit width (Sec. 2.2) and
  *     the index-bit / codebook-bit formulas (App. C.2).
  *
  * Not stated by the paper, defined by this project (parity unpinned by the
  * paper, consistency-checked only): the per-input-channel scale and bias and
- * their FP32 operation order, the bit-packed index stream, and "the first
- * n_out columns are the outlier columns".
+ * their FP32 operation order, the bit-packed index stream, "the first n_out
+ * STORED columns are the outlier columns", and the form of the column order
+ * (an explicit list of N input-feature numbers; scale and bias follow the
+ * stored order).
  *
  * Arithmetic: lookup sum, scale and bias in FP32 with three separately rounded
  * operations (build with -ffp-contract=off), result rounded to FP16
@@ -189,12 +195,23 @@ typedef struct oracle_layer {
     const uint16_t *c2;      /* [n_groups][k2][v]                                   */
     const uint8_t *idx0;     /* packed [ceil(M/v0)][n_out], b(k0) bits (n_out > 0)  */
     const uint16_t *c0;      /* [k0][v0]                                            */
-    const uint16_t *scale;   /* fp16 bits, [N] (axis 0) or [M] (axis 1)             */
+    const uint16_t *scale;   /* fp16 bits, [N] (axis 0, stored column order) or [M] (axis 1) */
     const uint16_t *bias;
+    const int32_t *col_perm; /* NULL, or [N]: stored column j is input feature col_perm[j]
+                                (a permutation of 0..N-1; Sec. 3.2.3)                */
 } oracle_layer;
 
-/* One restored weight, FP16 bits.  Returns 0xFFFF-coded error through *err when an
- * index is out of range (corrupt stream): the tests treat that as a failure. */
+/* Input feature of stored column j; -1 when the list names a feature outside [0,N). */
+static int32_t feature_of(const oracle_layer *L, int32_t j)
+{
+    if (L->col_perm == NULL) return j;
+    int32_t f = L->col_perm[j];
+    return (f < 0 || f >= L->N) ? -1 : f;
+}
+
+/* One restored weight, FP16 bits: row m of STORED column n (its place in W is column
+ * feature_of(n)).  Sets *err when an index is out of range (corrupt stream): the tests
+ * treat that as a failure. */
 static uint16_t restore_weight(const oracle_layer *L, int32_t m, int32_t n, int *err)
 {
     float t;
@@ -242,8 +259,11 @@ int oracle_dequant(const oracle_layer *L, uint16_t *W16)
 #pragma omp parallel for schedule(static) reduction(|:bad)
     for (int32_t m = 0; m < L->M; m++) {
         int err = 0;
-        for (int32_t n = 0; n < L->N; n++)
-            W16[(int64_t)m * L->N + n] = restore_weight(L, m, n, &err);
+        for (int32_t n = 0; n < L->N; n++) {
+            int32_t f = feature_of(L, n);
+            if (f < 0) { err = 1; continue; }
+            W16[(int64_t)m * L->N + f] = restore_weight(L, m, n, &err);
+        }
         bad |= err;
     }
     return bad ? -1 : 0;
@@ -256,8 +276,11 @@ int oracle_dequant_rows(const oracle_layer *L, const int32_t *rows, int32_t n_ro
 #pragma omp parallel for schedule(static) reduction(|:bad)
     for (int32_t i = 0; i < n_rows; i++) {
         int err = 0;
-        for (int32_t n = 0; n < L->N; n++)
-            Wrows[(int64_t)i * L->N + n] = restore_weight(L, rows[i], n, &err);
+        for (int32_t n = 0; n < L->N; n++) {
+            int32_t f = feature_of(L, n);
+            if (f < 0) { err = 1; continue; }
+            Wrows[(int64_t)i * L->N + f] = restore_weight(L, rows[i], n, &err);
+        }
         bad |= err;
     }
     return bad ? -1 : 0;
@@ -278,8 +301,12 @@ int oracle_linear_rows(const oracle_layer *L, const uint16_t *x, int32_t B, int 
     for (int32_t i = 0; i < n_rows; i++) {
         int err = 0;
         int32_t m = rows ? rows[i] : i;
-        uint16_t *w = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)L->N);
-        for (int32_t n = 0; n < L->N; n++) w[n] = restore_weight(L, m, n, &err);
+        uint16_t *w = (uint16_t *)calloc((size_t)L->N, sizeof(uint16_t));
+        for (int32_t n = 0; n < L->N; n++) {
+            int32_t f = feature_of(L, n);
+            if (f < 0) { err = 1; continue; }
+            w[f] = restore_weight(L, m, n, &err);          /* row m of W, in input-feature order */
+        }
         for (int32_t t = 0; t < B; t++) {
             double acc = 0.0;
             for (int32_t n = 0; n < L->N; n++)

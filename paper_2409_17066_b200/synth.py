@@ -21,7 +21,7 @@ import numpy as np
 BASE_SEED = 240917066
 
 # tensor ordinals inside a layer (part of the seed)
-T_IDX1, T_IDX2, T_IDX0, T_C1, T_C2, T_C0, T_SCALE, T_BIAS, T_X = range(9)
+T_IDX1, T_IDX2, T_IDX0, T_C1, T_C2, T_C0, T_SCALE, T_BIAS, T_X, T_PERM = range(10)
 
 
 @dataclasses.dataclass(frozen=True)
@@ -40,6 +40,8 @@ class LayerSpec:
     out_dtype: str = "fp16"   # "fp16" | "bf16" | "fp32"
     has_scale: bool = True
     n_groups: int = 1         # column groups with codebooks of their own (Sec. 3.1 / App. B table)
+    permuted: bool = False    # the stored columns are a seeded permutation of the input features (Sec. 3.2.3:
+                              # the outlier columns lie where the quantizer found them, not in front)
 
     @property
     def R(self) -> int:
@@ -169,8 +171,16 @@ def make_x(spec: LayerSpec, config: int, layer: int, B: int) -> np.ndarray:
 def make_layer(spec: LayerSpec, config: int, layer: int, B: int, dist: str = "uniform") -> Dict:
     idx1, idx2, idx0 = make_indices(spec, config, layer, dist)
     c1, c2, c0, scale, bias = make_tables(spec, config, layer)
-    return dict(spec=spec, idx1=idx1, idx2=idx2, idx0=idx0, c1=c1, c2=c2, c0=c0,
-                scale=scale, bias=bias, x=make_x(spec, config, layer, B), B=B)
+    d = dict(spec=spec, idx1=idx1, idx2=idx2, idx0=idx0, c1=c1, c2=c2, c0=c0,
+             scale=scale, bias=bias, x=make_x(spec, config, layer, B), B=B)
+    if spec.permuted:
+        d["col_perm"] = make_col_perm(spec, config, layer)
+    return d
+
+
+def make_col_perm(spec: LayerSpec, config: int, layer: int) -> np.ndarray:
+    """Input feature of every stored column: a seeded permutation of 0..N-1 (int32)."""
+    return _rng(config, layer, T_PERM).permutation(spec.N).astype(np.int32)
 
 
 def small_specs() -> List[LayerSpec]:
@@ -191,4 +201,8 @@ def small_specs() -> List[LayerSpec]:
         LayerSpec("s_v12_g4", 60, 134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4),
         LayerSpec("s_v6_g16", 100, 333, v=6, k1=4096, n_out=3, v0=4, k0=8192, n_groups=16),
         LayerSpec("s_v8_g3", 72, 200, v=8, k1=256, k2=16, n_groups=3),
+        # outlier columns anywhere in the matrix (Sec. 3.2.3): the stored columns are a permutation of the inputs
+        LayerSpec("s_v6_perm", 130, 700, v=6, k1=4096, k2=256, n_out=7, v0=4, k0=4096, permuted=True),
+        LayerSpec("s_v8_res_perm", 264, 1030, v=8, k1=65536, k2=256, permuted=True),
+        LayerSpec("s_v12_g4_perm", 60, 134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4, permuted=True),
     ]

@@ -398,3 +398,50 @@ def test_grouped_layers_vs_numpy_statement_and_group_boundaries(G):
     others = np.setdiff1d(np.arange(spec.n_out, spec.N), cols)
     bias = d["bias"].astype(np.float32)[others]
     assert np.array_equal(W0[:, others].astype(np.float32), np.broadcast_to(bias.astype(np.float16).astype(np.float32), (spec.M, others.size)))
+
+
+# ---------------------------------------------------------------- outlier columns anywhere (Sec. 3.2.3)
+
+def test_column_order_special_cases():
+    # Sec. 3.2.3 / Algorithm 2: the quantizer selects the outlier columns, so the stored column order is
+    # a list of input features.  Identity order: nothing changes.  Reversed order: the mirror image.
+    spec = synth.LayerSpec("p", 24, 30, v=8, k1=256, k2=16, n_out=5, v0=4, k0=16)
+    d = synth.make_layer(spec, 98, 0, 2)
+    W = _layer(d).dequant()
+    ident = dict(d, col_perm=np.arange(30, dtype=np.int32))
+    assert np.array_equal(_layer(ident).dequant().view(np.uint16), W.view(np.uint16))
+    assert np.array_equal(_layer(ident).linear(d["x"]), _layer(d).linear(d["x"]))
+    rev = dict(d, col_perm=np.arange(29, -1, -1, dtype=np.int32))
+    assert np.array_equal(_layer(rev).dequant().view(np.uint16), W[:, ::-1].view(np.uint16))
+    # the first n_out STORED columns are the outlier columns: they land on the features the list names
+    perm = np.random.default_rng(5).permutation(30).astype(np.int32)
+    Wp = _layer(dict(d, col_perm=perm)).dequant()
+    for j in range(30):
+        assert np.array_equal(Wp[:, perm[j]].view(np.uint16), W[:, j].view(np.uint16))
+    for m in range(24):
+        for j in range(5):      # scale and bias follow the stored order
+            t = np.float32(d["c0"][d["idx0"][m // 4, j], m % 4]) * np.float32(d["scale"][j])
+            t = np.float32(t) + np.float32(d["bias"][j])
+            assert Wp[m, perm[j]].view(np.uint16) == np.float16(t).view(np.uint16)
+
+
+def test_column_order_is_a_reordering_of_the_activations():
+    # y = sum_j x[perm[j]] * W_stored[:, j]: the permuted layer on x equals the plain layer on x[:, perm]
+    spec = synth.LayerSpec("q", 40, 52, v=8, k1=256, k2=16, n_out=3, v0=4, k0=16, permuted=True)
+    d = synth.make_layer(spec, 99, 0, 3)
+    perm = d["col_perm"]
+    assert sorted(perm.tolist()) == list(range(52))
+    plain = {k: v for k, v in d.items() if k != "col_perm"}
+    y = _layer(d).linear(d["x"])
+    y_plain = _layer(plain).linear(np.ascontiguousarray(d["x"][:, perm]))
+    assert np.max(np.abs(y - y_plain)) <= 1e-12 * np.max(np.abs(y_plain))
+    assert np.max(np.abs(y - _layer(plain).linear(d["x"]))) > 1e-3      # and it does matter
+    # matmul over the restored matrix (library routine)
+    W = _layer(d).dequant()
+    assert np.allclose(y, mini.linear(W, d["x"].astype(np.float64)), rtol=0, atol=1e-12)
+    # a list that names a feature outside [0, N) is a corrupt layer
+    bad = dict(d, col_perm=np.where(np.arange(52) == 7, 52, perm).astype(np.int32))
+    with pytest.raises(ValueError):
+        _layer(bad).dequant()
+    with pytest.raises(ValueError):
+        _layer(bad).linear(d["x"])
