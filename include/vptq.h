@@ -59,6 +59,7 @@ extern "C" {
 #define VPTQ_FLAG_SCALE_BIAS   1  /* scale and bias are present                                     */
 #define VPTQ_FLAG_SCALE_ROWS   2  /* scale/bias are per OUTPUT row ([M]) instead of per input column */
 #define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
+#define VPTQ_FLAG_COL_PERM      8 /* the layer has a stored column order (vptq_layer_ptrs.col_perm)   */
 
 /* Geometry of one quantized linear layer (App. C.1 names: v1,k1,k2 / N%,v0,k0). */
 typedef struct vptq_layer_desc {
@@ -76,7 +77,7 @@ typedef struct vptq_layer_desc {
                             shorter), each with main/residual codebooks of its own; 0 or 1 = one   */
 } vptq_layer_desc;
 
-/* The nine format pointers of a layer, in the order of the paper's format statement.
+/* The format pointers of a layer, in the order of the paper's format statement.
  *   packed_idx       packed [ceil(M/v)][N-n_outlier], b(k1) bits       (required unless n_outlier == N)
  *   codebook         fp16 [n_groups][k1][v]                             (required unless n_outlier == N)
  *   res_idx          packed, same shape, b(k2) bits                     (required iff k2 > 0)
@@ -84,7 +85,17 @@ typedef struct vptq_layer_desc {
  *   outlier_idx      packed [ceil(M/v0)][n_outlier], b(k0) bits         (required iff n_outlier > 0)
  *   outlier_codebook fp16 [k0][v0]                                      (required iff n_outlier > 0)
  *   scale, bias      fp16 [N] (or [M] with VPTQ_FLAG_SCALE_ROWS)        (required iff VPTQ_FLAG_SCALE_BIAS)
- * A pointer that is not required may be null and is never read. */
+ *   col_perm         int32 [N], a permutation of 0..N-1                 (required iff VPTQ_FLAG_COL_PERM)
+ * A pointer that is not required may be null and is never read.
+ *
+ * col_perm is the stored column order.  The quantizer picks the outlier columns where the Hessian
+ * diagonal is largest (Sec. 3.2.3; Algorithm 2 "selects outlier columns"), so they lie anywhere in the
+ * matrix, while the format keeps them in front: stored column j (an outlier column for j < n_outlier)
+ * is input feature col_perm[j], i.e. W_hat[m][col_perm[j]] = value restored for stored column j, and
+ * vptq_linear multiplies stored column j with x[t][col_perm[j]].  scale and bias (per input column)
+ * follow the stored order.  Without the flag the order is the identity.  Entries outside [0,N) are clamped to N-1 on the
+ * device (like indices beyond a codebook), never dereferenced out of bounds; a list that is not a
+ * permutation gives a well-defined but meaningless result. */
 typedef struct vptq_layer_ptrs {
     const uint8_t *packed_idx;
     const void    *codebook;
@@ -94,6 +105,7 @@ typedef struct vptq_layer_ptrs {
     const void    *outlier_codebook;
     const void    *scale;
     const void    *bias;
+    const int32_t *col_perm;
 } vptq_layer_ptrs;
 
 /* ---- format arithmetic (host only, no CUDA call) ---------------------------------- */

@@ -29,7 +29,7 @@ E_NULL, E_SHAPE, E_ALIGN, E_UNSUPPORTED, E_WORKSPACE, E_INDEX_RANGE, E_CUDA, E_T
 E_SCRATCH_LIMIT = -9
 NOALLOC_SCRATCH_BYTES = 1 << 20
 DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
-FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC = 1, 2, 4
+FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC, FLAG_COL_PERM = 1, 2, 4, 8
 
 _DT = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, "fp32": DTYPE_FP32}
 _TORCH_DT = {DTYPE_FP16: torch.float16, DTYPE_BF16: torch.bfloat16, DTYPE_FP32: torch.float32}
@@ -48,7 +48,7 @@ class LayerPtrs(C.Structure):
     _fields_ = [("packed_idx", C.c_void_p), ("codebook", C.c_void_p),
                 ("res_idx", C.c_void_p), ("res_codebook", C.c_void_p),
                 ("outlier_idx", C.c_void_p), ("outlier_codebook", C.c_void_p),
-                ("scale", C.c_void_p), ("bias", C.c_void_p)]
+                ("scale", C.c_void_p), ("bias", C.c_void_p), ("col_perm", C.c_void_p)]
 
 
 EXPORTS = {
@@ -275,14 +275,18 @@ class DeviceLayer:
         self.idx0 = vptq_pack(up(d["idx0"]), s.k0) if s.n_out else None
         self.c1, self.c2, self.c0 = up(d["c1"]), up(d["c2"]), up(d["c0"])
         self.scale, self.bias = up(d["scale"]), up(d["bias"])
+        self.col_perm = up(d.get("col_perm"))          # int32 [N] or None: stored column order
         if flags is None:
             flags = FLAG_SCALE_BIAS if d["scale"] is not None else 0
             if scale_rows:
                 flags |= FLAG_SCALE_ROWS
+            if self.col_perm is not None:
+                flags |= FLAG_COL_PERM
         self.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags,
                               getattr(s, "n_groups", 1))
         self.ptrs = LayerPtrs(_ptr(self.idx1), _ptr(self.c1), _ptr(self.idx2), _ptr(self.c2),
-                              _ptr(self.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias))
+                              _ptr(self.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias),
+                              _ptr(self.col_perm))
         self._ws: Dict[int, Optional[torch.Tensor]] = {}
         self.device = dev
 
@@ -304,7 +308,8 @@ class DeviceLayer:
         other.idx2 = None if self.idx2 is None else self.idx2.clone()
         other.idx0 = None if self.idx0 is None else self.idx0.clone()
         other.ptrs = LayerPtrs(_ptr(other.idx1), _ptr(self.c1), _ptr(other.idx2), _ptr(self.c2),
-                               _ptr(other.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias))
+                               _ptr(other.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias),
+                               _ptr(self.col_perm))
         return other
 
     def weight_bytes(self) -> int:

@@ -54,6 +54,7 @@ struct LayerView {
     Stream s1, s2, s0;
     const __half *c1, *c2, *c0;
     const __half *scale, *bias;
+    const int *perm;       // nullptr, or [N]: stored column n is input feature perm[n] (Sec. 3.2.3)
 };
 
 #ifdef __CUDACC__
@@ -74,6 +75,14 @@ __device__ __forceinline__ int load_index(const uint8_t *row, int c, int bits)
 }
 
 __device__ __forceinline__ int clamp_index(int i, int k) { return i < k ? i : k - 1; }
+
+// Input feature of stored column n.  A list entry outside [0, N) is clamped, as indices are.
+__device__ __forceinline__ int in_col(const LayerView &L, int n)
+{
+    if (L.perm == nullptr) return n;
+    const unsigned f = (unsigned)__ldg(L.perm + n);
+    return (int)(f < (unsigned)L.N ? f : (unsigned)(L.N - 1));
+}
 
 __device__ __forceinline__ float load_act(const void *x, long long i, int is_bf16)
 {

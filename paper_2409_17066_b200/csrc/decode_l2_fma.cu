@@ -167,7 +167,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
             float bacc[TB];
 #pragma unroll
             for (int t = 0; t < TB; t++) bacc[t] = 0.f;
-            if ((L.N & 7) == 0) {
+            if ((L.N & 7) == 0 && L.perm == nullptr) {
                 // 8 columns per thread and step, 128-bit loads (rows of x start 16-byte aligned)
                 for (int n = b_begin + 8 * threadIdx.x; n < b_end; n += 8 * THREADS) {
                     float sc[8], bi[8];
@@ -210,7 +210,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
                     const bool mine = n >= c_begin && n < c_end;
 #pragma unroll
                     for (int t = 0; t < TB; t++) {
-                        const float xv = t < P.B ? load_act(P.x, (long long)t * L.N + n, L.x_bf16) : 0.f;
+                        const float xv = t < P.B ? load_act(P.x, (long long)t * L.N + in_col(L, n), L.x_bf16) : 0.f;
                         if (mine) xs[t * P.slab_cols + (n - c_begin)] = __float2half_rn(xv * sc);
                         bacc[t] += xv * bi;
                     }

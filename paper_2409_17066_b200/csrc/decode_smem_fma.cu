@@ -207,7 +207,7 @@ decode_smem_fma_kernel(SmemFmaParams P)
                 const bool mine = c >= c_begin && c < c_end;
 #pragma unroll
                 for (int t = 0; t < TB; t++) {
-                    const float xv = t < P.B ? load_act(P.x, (long long)t * L.N + n, L.x_bf16) : 0.f;
+                    const float xv = t < P.B ? load_act(P.x, (long long)t * L.N + in_col(L, n), L.x_bf16) : 0.f;
                     const __half hv = __float2half_rn(xv * sc);
                     if (c < 0) xs_out[t * P.n_out_pad + n] = hv;
                     else if (mine) xs[t * P.slab_cols + (c - c_begin)] = hv;

@@ -140,6 +140,16 @@ __device__ __forceinline__ void load_xs16(const SmemMmaParams &P, int t, int n0,
 {
     const LayerView &L = P.L;
     uint32_t xw[8];
+    if (L.perm != nullptr) {
+        // a stored column order: the 16 activations are gathered one by one
+        const uint16_t *xr = reinterpret_cast<const uint16_t *>(P.x) + (long long)t * L.N;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const uint32_t lo = n0 + 2 * i < n_end ? __ldg(xr + in_col(L, n0 + 2 * i)) : 0u;
+            const uint32_t hi = n0 + 2 * i + 1 < n_end ? __ldg(xr + in_col(L, n0 + 2 * i + 1)) : 0u;
+            xw[i] = lo | (hi << 16);
+        }
+    } else
     load16_elems(reinterpret_cast<const uint16_t *>(P.x), (long long)t * L.N + n0,
                  (long long)t * L.N + n_end, xw);
     const bool scaled = L.has_scale && !L.scale_rows;
@@ -248,7 +258,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
                 float bn = L.scale_rows ? 1.f : __half2float(__ldg(L.bias + n));
 #pragma unroll
                 for (int t = 0; t < TP; t++)
-                    if (t < P.B) acc[t] += load_act(P.x, (long long)t * L.N + n, L.x_bf16) * bn;
+                    if (t < P.B) acc[t] += load_act(P.x, (long long)t * L.N + in_col(L, n), L.x_bf16) * bn;
             }
         }
 #pragma unroll
@@ -405,7 +415,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
                         float xv[4];
 #pragma unroll
                         for (int t = 0; t < 4; t++)
-                            xv[t] = (t0 + t < P.B) ? load_act(P.x, (long long)(t0 + t) * L.N + n, L.x_bf16) * sc : 0.f;
+                            xv[t] = (t0 + t < P.B) ? load_act(P.x, (long long)(t0 + t) * L.N + in_col(L, n), L.x_bf16) * sc : 0.f;
 #pragma unroll
                         for (int j = 0; j < 8; j++) {
                             if (j < L.v0) {

@@ -58,7 +58,7 @@ dequant_kernel(LayerView L, __half *__restrict__ W)
             s = __half2float(__ldg(L.scale + m));
             b = __half2float(__ldg(L.bias + m));
         }
-        W[(long long)m * L.N + n] = finish_weight(t, L.has_scale, s, b);
+        W[(long long)m * L.N + in_col(L, n)] = finish_weight(t, L.has_scale, s, b);
     }
 }
 

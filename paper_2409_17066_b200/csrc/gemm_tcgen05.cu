@@ -282,7 +282,7 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
         }
     }
     float acc = 0.f;
-    if ((L.N & 7) == 0) {
+    if ((L.N & 7) == 0 && L.perm == nullptr) {
         // 8 columns = one chunk per thread and step, 128-bit loads and stores; the loads of four steps are
         // issued together (a thread with one load in flight at a time leaves the memory system idle)
         constexpr int UNROLL = 4;
@@ -328,7 +328,7 @@ gemm_prepass_kernel(LayerView L, const void *__restrict__ x, int B, uint8_t *__r
         for (int n = threadIdx.x; n < kb_total * TILE_K; n += PRE_THREADS) {
             float xv = 0.f, sc = 1.f, bi = 0.f;
             if (n < L.N) {
-                xv = load_act(x, (long long)t * L.N + n, L.x_bf16);
+                xv = load_act(x, (long long)t * L.N + in_col(L, n), L.x_bf16);
                 if (L.has_scale) {
                     sc = __half2float(__ldg(L.scale + n));
                     bi = __half2float(__ldg(L.bias + n));

@@ -53,7 +53,7 @@ linear_generic_kernel(LayerView L, const void *__restrict__ x, int B, void *__re
             }
 #pragma unroll
             for (int t = 0; t < GEN_TB; t++)
-                if (t0 + t < B) acc[t] += load_act(x, (long long)(t0 + t) * L.N + n, L.x_bf16) * w;
+                if (t0 + t < B) acc[t] += load_act(x, (long long)(t0 + t) * L.N + in_col(L, n), L.x_bf16) * w;
         }
 #pragma unroll
         for (int t = 0; t < GEN_TB; t++) {

@@ -34,7 +34,7 @@ int check_desc(const vptq_layer_desc *d)
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
         d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
-    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC)) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM)) return VPTQ_E_UNSUPPORTED;
     if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
     return VPTQ_OK;
 }
@@ -47,6 +47,10 @@ int check_ptrs(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     if (has_main && d->k2 > 0 && (p->res_idx == nullptr || p->res_codebook == nullptr)) return VPTQ_E_NULL;
     if (d->n_outlier > 0 && (p->outlier_idx == nullptr || p->outlier_codebook == nullptr)) return VPTQ_E_NULL;
     if ((d->flags & VPTQ_FLAG_SCALE_BIAS) && (p->scale == nullptr || p->bias == nullptr)) return VPTQ_E_NULL;
+    if (d->flags & VPTQ_FLAG_COL_PERM) {
+        if (p->col_perm == nullptr) return VPTQ_E_NULL;
+        if (!aligned16(p->col_perm)) return VPTQ_E_ALIGN;
+    }
     const void *all[8] = {has_main ? p->packed_idx : nullptr, has_main ? p->codebook : nullptr,
                           (has_main && d->k2 > 0) ? p->res_idx : nullptr,
                           (has_main && d->k2 > 0) ? p->res_codebook : nullptr,
@@ -87,6 +91,7 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
         L.c0 = L.n_out ? reinterpret_cast<const __half *>(p->outlier_codebook) : nullptr;
         L.scale = L.has_scale ? reinterpret_cast<const __half *>(p->scale) : nullptr;
         L.bias = L.has_scale ? reinterpret_cast<const __half *>(p->bias) : nullptr;
+        L.perm = (d->flags & VPTQ_FLAG_COL_PERM) ? reinterpret_cast<const int *>(p->col_perm) : nullptr;
     }
     return L;
 }
@@ -125,6 +130,7 @@ int64_t vptq_layer_weight_bytes(const vptq_layer_desc *d)
     }
     if (L.n_out) bytes += (int64_t)L.R0 * row_bytes(L.n_out, L.k0) + 2LL * L.k0 * L.v0;
     if (L.has_scale) bytes += 4LL * (L.scale_rows ? L.M : L.N);
+    if (d->flags & VPTQ_FLAG_COL_PERM) bytes += 4LL * L.N;
     return bytes;
 }
 

@@ -192,6 +192,21 @@ def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
     assert rel_err(y.float().cpu().numpy(), yg.astype(np.float64)) <= TOL
 
 
+def test_linear_batched_tcgen05_with_a_stored_column_order(b):
+    # Sec. 3.2.3: stored column j is input feature col_perm[j]; the pre-pass gathers the activations
+    spec = synth.LayerSpec("gp", 264, 1032, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32", permuted=True)
+    B = 40
+    d = synth.make_layer(spec, 77, 1, B)
+    dl = b.DeviceLayer(d)
+    assert dl.desc.flags & b.FLAG_COL_PERM and b.vptq_linear_path(dl.desc, B) == "gemm_tcgen05"
+    y = dl.linear(dl.upload_x(d["x"])).float().cpu().numpy()
+    assert b.vptq_workspace_status(dl.workspace(B)) == b.OK
+    assert rel_err(y, oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+    # the same layer without its column order gives another result: the order is really applied
+    plain = {k: v for k, v in d.items() if k != "col_perm"}
+    assert rel_err(y, oracle.Layer.from_synth(plain).linear(d["x"])) > 100 * TOL
+
+
 # ------------------------------------------------------------------ several layers over the same activations
 
 def _fused_case(b, specs, B, seed):
