@@ -64,6 +64,11 @@ _lib.oracle_equivalent_bits_grouped.argtypes = [C.c_int32] * 9
 for _n in ("oracle_index_bits_total", "oracle_equivalent_bits", "oracle_compression_ratio"):
     getattr(_lib, _n).restype = C.c_double
     getattr(_lib, _n).argtypes = [C.c_int32] * 8
+_lib.oracle_assign.restype = None
+_lib.oracle_assign.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
+_lib.oracle_assign_some.restype = None
+_lib.oracle_assign_some.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                    C.c_void_p, C.c_int32, C.c_void_p]
 _lib.oracle_num_threads.restype = C.c_int
 _lib.oracle_set_num_threads.argtypes = [C.c_int]
 
@@ -193,6 +198,25 @@ class Layer:
                                    y.ctypes.data) != 0:
             raise ValueError("index out of range in packed stream")
         return y
+
+
+def assign(W16: np.ndarray, v: int, codebook: np.ndarray, vectors=None) -> np.ndarray:
+    """Eq. 2: index of the nearest centroid for every length-v vector (v consecutive rows of a column) of the
+    float16 matrix W16 [M][N]; codebook float16 [k][v].  Returns int32 [ceil(M/v)][N], or, with `vectors`
+    (flat numbers r * N + n), the indices of those vectors only."""
+    Wb = np.ascontiguousarray(W16, dtype=np.float16).view(np.uint16)
+    Cb = np.ascontiguousarray(codebook, dtype=np.float16).view(np.uint16)
+    M, N = Wb.shape
+    k = Cb.shape[0]
+    assert Cb.shape == (k, v)
+    if vectors is None:
+        idx = np.empty((-(-M // v), N), dtype=np.int32)
+        _lib.oracle_assign(Wb.ctypes.data, M, N, v, Cb.ctypes.data, k, idx.ctypes.data)
+        return idx
+    vec = np.ascontiguousarray(vectors, dtype=np.int64)
+    idx = np.empty(vec.size, dtype=np.int32)
+    _lib.oracle_assign_some(Wb.ctypes.data, M, N, v, Cb.ctypes.data, k, vec.ctypes.data, vec.size, idx.ctypes.data)
+    return idx
 
 
 def codebook_bits(v, k1, k2=0, n_out=0, v0=0, k0=0) -> float:

@@ -25,7 +25,11 @@
  *     column order, col_perm, that says which input feature each stored column is;
  *   - the weights are restored to FP16 and then multiplied (App. D.2).
  *   - size accounting: compression ratio / equivalent bit width (Sec. 2.2) and
- *     the index-bit / codebook-bit formulas (App. C.2).
+ *     the index-bit / codebook-bit formulas (App. C.2);
+ *   - the quantizer's assignment step (Eq. 2): every vector of the reshaped weight
+ *     matrix takes the index of the centroid at the smallest Euclidean distance
+ *     (oracle_assign below; the Hessian-driven parts of Algorithms 1 and 2 are not
+ *     here).
  *
  * Not stated by the paper, defined by this project (parity unpinned by the
  * paper, consistency-checked only): the per-input-channel scale and bias and
@@ -46,6 +50,7 @@
 #include <stddef.h>
 #include <stdlib.h>
 #include <string.h>
+#include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -322,6 +327,60 @@ int oracle_linear_rows(const oracle_layer *L, const uint16_t *x, int32_t B, int 
 int oracle_linear(const oracle_layer *L, const uint16_t *x, int32_t B, int x_is_bf16, double *y)
 {
     return oracle_linear_rows(L, x, B, x_is_bf16, NULL, L->M, y);
+}
+
+/* ------------------------------------------------------------------ */
+/* Assignment step of the quantizer (Eq. 2)                            */
+/* ------------------------------------------------------------------ */
+
+/* Squared Euclidean distance between vector (r, n) of W and centroid i, over the components
+ * that exist (the last vector row is short when v does not divide M).
+ * Floating point decides an integer here, so the arithmetic is fixed: FP32, components in
+ * ascending order, each step d = fma(t, t, d) with t = x_j - c_j rounded to FP32. */
+static float sq_distance(const uint16_t *W, int32_t M, int32_t N, int32_t v, int32_t r, int32_t n,
+                         const uint16_t *C, int32_t i)
+{
+    float d = 0.0f;
+    for (int32_t j = 0; j < v && r * v + j < M; j++) {
+        float x = oracle_half_to_float(W[(int64_t)(r * v + j) * N + n]);
+        float c = oracle_half_to_float(C[(int64_t)i * v + j]);
+        float t = x - c;
+        d = fmaf(t, t, d);
+    }
+    return d;
+}
+
+/* Eq. 2 for one vector: argmin_i || v - C_i ||^2; of equal distances the lowest index wins;
+ * a distance that is NaN never wins (all NaN: index 0). */
+static int32_t nearest_centroid(const uint16_t *W, int32_t M, int32_t N, int32_t v, int32_t r, int32_t n,
+                                const uint16_t *C, int32_t k)
+{
+    int32_t best = 0;
+    float best_d = INFINITY;
+    for (int32_t i = 0; i < k; i++) {
+        float d = sq_distance(W, M, N, v, r, n, C, i);
+        if (d < best_d) { best_d = d; best = i; }
+    }
+    return best;
+}
+
+/* idx [ceil(M/v)][N]: vectors are v consecutive rows of one column (Sec. 3.1, Algorithm 1). */
+void oracle_assign(const uint16_t *W, int32_t M, int32_t N, int32_t v, const uint16_t *C, int32_t k, int32_t *idx)
+{
+    int32_t R = (M + v - 1) / v;
+#pragma omp parallel for schedule(static)
+    for (int32_t r = 0; r < R; r++)
+        for (int32_t n = 0; n < N; n++)
+            idx[(int64_t)r * N + n] = nearest_centroid(W, M, N, v, r, n, C, k);
+}
+
+/* The same for selected vectors only: vec[i] = r * N + n. */
+void oracle_assign_some(const uint16_t *W, int32_t M, int32_t N, int32_t v, const uint16_t *C, int32_t k,
+                        const int64_t *vec, int32_t n_vec, int32_t *idx)
+{
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int32_t i = 0; i < n_vec; i++)
+        idx[i] = nearest_centroid(W, M, N, v, (int32_t)(vec[i] / N), (int32_t)(vec[i] % N), C, k);
 }
 
 /* ------------------------------------------------------------------ */

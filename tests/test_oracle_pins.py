@@ -445,3 +445,67 @@ def test_column_order_is_a_reordering_of_the_activations():
         _layer(bad).dequant()
     with pytest.raises(ValueError):
         _layer(bad).linear(d["x"])
+
+
+# ---------------------------------------------------------------- assignment step of the quantizer (Eq. 2)
+
+def _dist64(W, v, C):
+    """All squared distances in float64: [R][N][k] (M divisible by v)."""
+    M, N = W.shape
+    X = W.astype(np.float64).reshape(M // v, v, N).transpose(0, 2, 1)          # [R][N][v]
+    return ((X[:, :, None, :] - C.astype(np.float64)[None, None, :, :]) ** 2).sum(axis=3)
+
+
+def test_assign_is_the_nearest_centroid_brute_force():
+    rng = np.random.default_rng(11)
+    for v, k, M, N in ((8, 64, 32, 20), (6, 50, 36, 17), (2, 7, 10, 9), (12, 33, 24, 5), (1, 5, 6, 6)):
+        W = rng.normal(0, 1, (M, N)).astype(np.float16)
+        C = rng.normal(0, 1, (k, v)).astype(np.float16)
+        idx = oracle.assign(W, v, C)
+        D = _dist64(W, v, C)
+        best = D.min(axis=2)
+        chosen = np.take_along_axis(D, idx[:, :, None].astype(np.int64), axis=2)[:, :, 0]
+        # the chosen centroid is a nearest one (FP32 rounding may only swap near-ties) ...
+        assert np.all(chosen <= best * (1 + 1e-5) + 1e-12)
+        # ... and THE nearest one wherever the runner-up is clearly farther
+        second = np.partition(D, 1, axis=2)[:, :, 1]
+        clear = second > best * (1 + 1e-4) + 1e-9
+        assert clear.mean() > 0.9
+        assert np.array_equal(idx[clear], D.argmin(axis=2)[clear])
+
+
+def test_assign_special_cases():
+    rng = np.random.default_rng(12)
+    # every vector IS a centroid: the assignment returns it (distance 0), so assign(dequant(I)) = I
+    C = rng.normal(0, 1, (40, 8)).astype(np.float16)
+    I = rng.integers(0, 40, (5, 13)).astype(np.int32)
+    W = mini.dequant(40, 13, 8, C, I)
+    assert np.array_equal(oracle.assign(W, 8, C), I)
+    # equal distances: the lowest index wins (a duplicated centroid; a point half way between two)
+    C2 = np.concatenate([C[:3], C[:3], C[3:]])
+    assert np.array_equal(oracle.assign(W, 8, C2), np.where(I >= 3, I + 3, I))
+    mid = oracle.assign(np.zeros((2, 1), np.float16), 2, np.array([[1, 0], [-1, 0], [0, 1]], np.float16))
+    assert mid.tolist() == [[0]]
+    # v = 1 with a sorted grid of centroids: rounding to the nearest grid point (closed form)
+    grid = np.arange(-4, 5, dtype=np.float16).reshape(9, 1)
+    x = np.array([[-3.75, -0.25, 0.0, 0.26, 1.49, 1.51, 3.9, 7.0, -9.0]], np.float16)
+    want = np.clip(np.rint(x.astype(np.float64)), -4, 4).astype(np.int32) + 4
+    assert np.array_equal(oracle.assign(x, 1, grid), want)
+    # k = 1: always index 0
+    assert not oracle.assign(W, 8, C[:1]).any()
+
+
+def test_assign_ragged_last_vector_row_ignores_missing_components():
+    rng = np.random.default_rng(13)
+    v, k, M, N = 8, 30, 21, 11                       # last vector row has 5 of 8 components
+    W = rng.normal(0, 1, (M, N)).astype(np.float16)
+    C = rng.normal(0, 1, (k, v)).astype(np.float16)
+    idx = oracle.assign(W, v, C)
+    assert idx.shape == (3, N)
+    Wp = np.concatenate([W, np.zeros((3, N), np.float16)])
+    assert np.array_equal(idx[:2], oracle.assign(Wp, v, C)[:2])
+    # the short row is the assignment against the first 5 components of every centroid
+    assert np.array_equal(idx[2:], oracle.assign(W[16:], 5, np.ascontiguousarray(C[:, :5])))
+    # selected vectors only
+    vec = np.array([0, N - 1, N, 2 * N + 3], np.int64)
+    assert np.array_equal(oracle.assign(W, v, C, vec), idx.reshape(-1)[vec])
