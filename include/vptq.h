@@ -245,6 +245,22 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
 int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
                         const vptq_layer_ptrs *p, void *out, void *stream);
 
+/* ---- the quantizer's assignment step -------------------------------------------------- */
+
+/* Eq. 2: idx[r][n] = argmin_i || W[r*v .. r*v+v-1][n] - C_i ||^2 for every length-v vector of the
+ * weight matrix (v consecutive rows of one column: Sec. 3.1, Algorithm 1), i.e. the index matrix that
+ * vptq_pack packs and vptq_dequant looks up again.  (With a Hessian-weighted objective the weight of a
+ * vector's column is common to all its distances and does not change the argmin: Sec. 3.2.1 moves the
+ * weights into the k-means centroid update, which this library does not have.)
+ *   W        fp16 [M][N] row-major (device)      codebook  fp16 [k][v] (device)
+ *   idx      int32 [ceil(M/v)][N] (device, written)
+ * Arithmetic, fixed because it decides an integer: FP32, components in ascending order,
+ * d = fma(t, t, d) with t = x_j - c_j; of equal distances the lowest index wins; a NaN distance never
+ * wins (all NaN: index 0); components beyond row M-1 (short last vector row) are left out.
+ * 1 <= v <= 32, 1 <= k <= 65536, else VPTQ_E_SHAPE / VPTQ_E_UNSUPPORTED.  Asynchronous on `stream`. */
+int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
+                int32_t *idx, void *stream);
+
 /* ---- diagnostics ------------------------------------------------------------------ */
 
 const char *vptq_status_string(int code);

@@ -59,6 +59,7 @@ EXPORTS = {
     "vptq_pack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
+    "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "vptq_linear_workspace_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                               C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -158,6 +159,18 @@ def vptq_dequant(desc: LayerDesc, ptrs: LayerPtrs, W_out: torch.Tensor) -> torch
     assert tuple(W_out.shape) == (desc.M, desc.N)
     _check(lib.vptq_dequant(C.byref(desc), C.byref(ptrs), _ptr(W_out), _stream()))
     return W_out
+
+
+def vptq_assign(W: torch.Tensor, v: int, codebook: torch.Tensor) -> torch.Tensor:
+    """Eq. 2: int32 [ceil(M/v)][N] index of the nearest centroid of every length-v vector of W (fp16 [M][N])."""
+    assert W.is_cuda and W.dtype == torch.float16 and W.dim() == 2 and W.is_contiguous()
+    assert codebook.is_cuda and codebook.dtype == torch.float16 and codebook.is_contiguous()
+    M, N = W.shape
+    k = codebook.shape[0]
+    assert tuple(codebook.shape) == (k, v)
+    idx = torch.empty((-(-M // v), N), dtype=torch.int32, device=W.device)
+    _check(lib.vptq_assign(_ptr(W), M, N, v, _ptr(codebook), k, _ptr(idx), _stream()))
+    return idx
 
 
 def vptq_linear_workspace_bytes(desc: LayerDesc, B: int) -> int:

@@ -104,6 +104,9 @@ cudaError_t launch_pack(const int32_t *idx, int rows, int cols, int k, uint8_t *
 cudaError_t launch_unpack(const uint8_t *packed, int rows, int cols, int k, int32_t *idx,
                           cudaStream_t st);
 cudaError_t launch_dequant(const LayerView &L, __half *W, cudaStream_t st);
+// assignment step of the quantizer (Eq. 2): idx [ceil(M/v)][N]
+bool assign_supported(int v, int k);
+cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st);
 
 // generic fallback linear (any geometry, any B): workspace = B*M floats
 long long generic_workspace_bytes(const LayerView &L, int B);

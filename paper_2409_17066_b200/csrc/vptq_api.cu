@@ -184,6 +184,21 @@ int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, void *W_
     return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 
+int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
+                int32_t *idx, void *stream)
+{
+    if (M < 0 || N < 0 || v < 1 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (!assign_supported(v, k)) return VPTQ_E_UNSUPPORTED;
+    if (M == 0 || N == 0) return VPTQ_OK;
+    if (W == nullptr || codebook == nullptr || idx == nullptr) return VPTQ_E_NULL;
+    if ((reinterpret_cast<uintptr_t>(W) & 1u) || (reinterpret_cast<uintptr_t>(codebook) & 1u) ||
+        (reinterpret_cast<uintptr_t>(idx) & 3u)) return VPTQ_E_ALIGN;
+    cudaError_t e = launch_assign(reinterpret_cast<const __half *>(W), M, N, v,
+                                  reinterpret_cast<const __half *>(codebook), k, idx,
+                                  reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
+}
+
 int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B)
 {
     int rc = check_desc(desc);

@@ -253,3 +253,34 @@ def test_linear_fused_runs_other_kernel_families_one_by_one(b):
     for d, y in zip(ds, outs):
         assert rel_err(y.float().cpu().numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
 
+
+
+# ------------------------------------------------------------------ assignment step of the quantizer (Eq. 2)
+
+@pytest.mark.parametrize("M,N,v,k", [
+    (136, 520, 8, 4096),       # several blocks, several codebook chunks
+    (130, 333, 6, 4096),       # v = 6 (padded to 8 components), ragged last vector row (130 = 21 * 6 + 4)
+    (60, 134, 12, 1000),       # v = 12 (padded to 16), a short last chunk
+    (34, 77, 2, 16),
+    (9, 17, 1, 1),
+    (16, 64, 8, 65536),        # the largest table, few vectors
+    (70, 50, 24, 300),         # v > 16
+])
+def test_assign_is_bit_identical_to_the_oracle(b, M, N, v, k):
+    rng = np.random.default_rng(1000 * v + k)
+    W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
+    Cb = rng.normal(0, 0.02, (k, v)).astype(np.float16)
+    idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda()).cpu().numpy()
+    assert np.array_equal(idx, oracle.assign(W, v, Cb))
+
+
+def test_assign_then_pack_and_dequant_reproduce_the_matrix(b):
+    # a matrix built from centroids goes through assign -> pack -> dequant unchanged (distinct centroids)
+    spec = synth.LayerSpec("enc", 264, 300, v=8, k1=4096, has_scale=False)
+    d = synth.make_layer(spec, 78, 0, 1)
+    dl = b.DeviceLayer(d)
+    W = dl.dequant()
+    idx = b.vptq_assign(W, 8, dl.c1)
+    again = b.vptq_pack(idx, spec.k1)
+    assert torch.equal(again, dl.idx1) or np.array_equal(
+        oracle.Layer.from_synth(dict(d, idx1=idx.cpu().numpy())).dequant().view(np.uint16), W.cpu().numpy().view(np.uint16))
