@@ -491,7 +491,38 @@ def extra_configs(vb, synth, peaks):
                 res[key] = r
             del variants, base, d
             torch.cuda.empty_cache()
+    res.update(encoder_assign(vb, synth))
     return res
+
+
+def encoder_assign(vb, synth):
+    """The quantizer's assignment step (Eq. 2) on a matrix of the size of config 1's layer: every one of the
+    2.1 M vectors against all 65536 centroids.  Bound by the FP32 pipes: one subtract and one fma per
+    component and centroid; peak = SMs x 128 FP32 lanes x SM clock instructions per second."""
+    import numpy as np
+    import torch
+    M, N, v, k = 4096, 4096, 8, 65536
+    rng = np.random.default_rng(synth.BASE_SEED + 77)
+    W = torch.from_numpy(rng.normal(0, 0.02, (M, N)).astype(np.float16)).cuda()
+    Cb = torch.from_numpy(rng.normal(0, 0.02, (k, v)).astype(np.float16)).cuda()
+    vb.vptq_assign(W, v, Cb)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        vb.vptq_assign(W, v, Cb)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 3
+    props = torch.cuda.get_device_properties(0)
+    pairs = (M // v) * N * k * v                                   # (subtract, fma) pairs
+    peak = props.multi_processor_count * 128 * 1.965e9             # FP32 instructions per second at the maximum SM clock
+    return {"encoder_assign_4096x4096_v8_k65536": {
+        "ms": ms, "G_distances_per_s": (M // v) * N * k / (ms * 1e-3) / 1e9,
+        "roofline": {"bound": "alu", "achieved": 2 * pairs / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
+                     "unit": "T FP32 instructions/s (one subtract and one fma per component)",
+                     "frac": 2 * pairs / (ms * 1e-3) / peak,
+                     "peak_source": "148 SMs x 128 FP32 lanes x 1.965 GHz (unit counts and maximum clock)"}}}
 
 
 def main():

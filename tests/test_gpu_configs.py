@@ -65,3 +65,17 @@ def test_config_layer(b, cfg, li):
         assert rel_err(y_rows, y_ref) <= TOL, (cfg, spec.name, B, b.vptq_linear_path(dl.desc, B))
         # a property that holds at any size: the whole output has the scale the samples have
         assert float(y.float().abs().max()) <= 3.0 * np.max(np.abs(y_ref)) + 1e-6
+
+
+def test_assign_full_size_sampled(b):
+    """Eq. 2 on a matrix of the size of config 1's layer, in the launch configuration the benchmark times:
+    all 2.1 M vectors against 65536 centroids on the GPU, 1500 sampled vectors through the oracle."""
+    M, N, v, k = 4096, 4096, 8, 65536
+    rng = np.random.default_rng(synth.BASE_SEED + 77)
+    W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
+    Cb = rng.normal(0, 0.02, (k, v)).astype(np.float16)
+    idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda()).cpu().numpy().reshape(-1)
+    n_vec = (M // v) * N
+    vec = np.unique(np.concatenate([np.random.default_rng(5).integers(0, n_vec, 1500), [0, n_vec - 1, N - 1, N]]))
+    assert np.array_equal(idx[vec], oracle.assign(W, v, Cb, vec))
+    assert idx.min() >= 0 and idx.max() < k
