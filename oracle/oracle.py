@@ -69,6 +69,11 @@ _lib.oracle_assign.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_
 _lib.oracle_assign_some.restype = None
 _lib.oracle_assign_some.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
                                     C.c_void_p, C.c_int32, C.c_void_p]
+_lib.oracle_kmeans_update.restype = None
+_lib.oracle_kmeans_update.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                      C.c_int32, C.c_void_p]
+_lib.oracle_distortion.restype = C.c_double
+_lib.oracle_distortion.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.oracle_num_threads.restype = C.c_int
 _lib.oracle_set_num_threads.argtypes = [C.c_int]
 
@@ -217,6 +222,31 @@ def assign(W16: np.ndarray, v: int, codebook: np.ndarray, vectors=None) -> np.nd
     idx = np.empty(vec.size, dtype=np.int32)
     _lib.oracle_assign_some(Wb.ctypes.data, M, N, v, Cb.ctypes.data, k, vec.ctypes.data, vec.size, idx.ctypes.data)
     return idx
+
+
+def kmeans_update(W16: np.ndarray, v: int, idx: np.ndarray, codebook: np.ndarray, h=None) -> np.ndarray:
+    """Weighted k-means centroid update (Sec. 3.2.1): the weighted mean of the vectors assigned to every
+    centroid (weights h[N] per column, None = 1); components that received no weight keep their old value.
+    Returns the new float16 [k][v] codebook."""
+    Wb = np.ascontiguousarray(W16, dtype=np.float16).view(np.uint16)
+    Cb = np.ascontiguousarray(codebook, dtype=np.float16).view(np.uint16).copy()
+    ib = np.ascontiguousarray(idx, dtype=np.int32)
+    M, N = Wb.shape
+    hb = None if h is None else np.ascontiguousarray(h, dtype=np.float32)
+    _lib.oracle_kmeans_update(Wb.ctypes.data, M, N, v, ib.ctypes.data, None if hb is None else hb.ctypes.data,
+                              Cb.shape[0], Cb.ctypes.data)
+    return Cb.view(np.float16)
+
+
+def distortion(W16: np.ndarray, v: int, idx: np.ndarray, codebook: np.ndarray, h=None) -> float:
+    """sum_n h_n ||x - C_idx||^2 over all vectors, float64."""
+    Wb = np.ascontiguousarray(W16, dtype=np.float16).view(np.uint16)
+    Cb = np.ascontiguousarray(codebook, dtype=np.float16).view(np.uint16)
+    ib = np.ascontiguousarray(idx, dtype=np.int32)
+    M, N = Wb.shape
+    hb = None if h is None else np.ascontiguousarray(h, dtype=np.float32)
+    return float(_lib.oracle_distortion(Wb.ctypes.data, M, N, v, ib.ctypes.data,
+                                        None if hb is None else hb.ctypes.data, Cb.ctypes.data))
 
 
 def codebook_bits(v, k1, k2=0, n_out=0, v0=0, k0=0) -> float:

@@ -383,6 +383,55 @@ void oracle_assign_some(const uint16_t *W, int32_t M, int32_t N, int32_t v, cons
         idx[i] = nearest_centroid(W, M, N, v, (int32_t)(vec[i] / N), (int32_t)(vec[i] % N), C, k);
 }
 
+/* Centroid update of (weighted) k-means (Sec. 2.2 "k-means ... to build a codebook"; Sec. 3.2.1: the
+ * diagonal term of the proxy error, sum_n h_nn ||dW[:,n]||^2, is a weighted k-means problem whose
+ * weight is the Hessian diagonal of the vector's column).  With the assignment fixed, the minimiser of
+ * sum h_n ||x - C_i||^2 over C_i is the weighted mean of the vectors assigned to i:
+ *   C_i[j] = sum h_n x_j / sum h_n   over the vectors (r, n) with idx[r][n] = i that have component j
+ * (the short last vector row has no components beyond row M-1).  FP64 sums, result rounded to FP16.
+ * h == NULL means all weights 1.  A component that received no weight keeps its old value. */
+void oracle_kmeans_update(const uint16_t *W, int32_t M, int32_t N, int32_t v, const int32_t *idx,
+                          const float *h, int32_t k, uint16_t *C)
+{
+    int32_t R = (M + v - 1) / v;
+    double *sum = (double *)calloc((size_t)k * v, sizeof(double));
+    double *wsum = (double *)calloc((size_t)k * v, sizeof(double));
+    for (int32_t r = 0; r < R; r++)
+        for (int32_t n = 0; n < N; n++) {
+            int32_t i = idx[(int64_t)r * N + n];
+            if (i < 0 || i >= k) continue;
+            double w = h ? (double)h[n] : 1.0;
+            for (int32_t j = 0; j < v && r * v + j < M; j++) {
+                sum[(int64_t)i * v + j] += w * (double)oracle_half_to_float(W[(int64_t)(r * v + j) * N + n]);
+                wsum[(int64_t)i * v + j] += w;
+            }
+        }
+    for (int64_t e = 0; e < (int64_t)k * v; e++)
+        if (wsum[e] > 0.0) C[e] = oracle_float_to_half((float)(sum[e] / wsum[e]));
+    free(sum);
+    free(wsum);
+}
+
+/* Weighted distortion sum_n h_n ||x - C_idx||^2 in FP64 (the quantity a k-means step must not increase). */
+double oracle_distortion(const uint16_t *W, int32_t M, int32_t N, int32_t v, const int32_t *idx,
+                         const float *h, const uint16_t *C)
+{
+    int32_t R = (M + v - 1) / v;
+    double total = 0.0;
+    for (int32_t r = 0; r < R; r++)
+        for (int32_t n = 0; n < N; n++) {
+            int32_t i = idx[(int64_t)r * N + n];
+            double w = h ? (double)h[n] : 1.0, d = 0.0;
+            for (int32_t j = 0; j < v && r * v + j < M; j++) {
+                double t = (double)oracle_half_to_float(W[(int64_t)(r * v + j) * N + n]) -
+                           (double)oracle_half_to_float(C[(int64_t)i * v + j]);
+                d += t * t;
+            }
+            total += w * d;
+        }
+    return total;
+}
+
 /* ------------------------------------------------------------------ */
 /* Size accounting                                                     */
 /* ------------------------------------------------------------------ */

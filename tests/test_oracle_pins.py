@@ -509,3 +509,52 @@ def test_assign_ragged_last_vector_row_ignores_missing_components():
     # selected vectors only
     vec = np.array([0, N - 1, N, 2 * N + 3], np.int64)
     assert np.array_equal(oracle.assign(W, v, C, vec), idx.reshape(-1)[vec])
+
+
+# ---------------------------------------------------------------- k-means centroid update (Sec. 3.2.1)
+
+def test_kmeans_update_is_the_weighted_mean():
+    rng = np.random.default_rng(21)
+    v, k, M, N = 4, 6, 16, 9
+    W = rng.normal(0, 1, (M, N)).astype(np.float16)
+    C = rng.normal(0, 1, (k, v)).astype(np.float16)
+    idx = rng.integers(0, k - 1, (M // v, N)).astype(np.int32)        # centroid k-1 gets no vector
+    h = rng.uniform(0.1, 3.0, N).astype(np.float32)
+    for weights in (None, h):
+        new = oracle.kmeans_update(W, v, idx, C, weights)
+        X = W.astype(np.float64).reshape(M // v, v, N).transpose(0, 2, 1)          # [R][N][v]
+        hw = np.ones(N) if weights is None else weights.astype(np.float64)
+        for i in range(k - 1):
+            sel = idx == i
+            wsel = np.broadcast_to(hw[None, :], idx.shape)[sel]
+            want = (X[sel] * wsel[:, None]).sum(0) / wsel.sum()
+            assert np.array_equal(new[i].view(np.uint16), want.astype(np.float32).astype(np.float16).view(np.uint16))
+        assert np.array_equal(new[k - 1].view(np.uint16), C[k - 1].view(np.uint16))     # empty cluster: unchanged
+    # one vector per centroid: the centroid becomes that vector, whatever its weight
+    W1 = rng.normal(0, 1, (4, 5)).astype(np.float16)
+    new = oracle.kmeans_update(W1, 4, np.arange(5, dtype=np.int32).reshape(1, 5), np.zeros((5, 4), np.float16), h[:5])
+    assert np.array_equal(new.view(np.uint16), np.ascontiguousarray(W1.T).view(np.uint16))
+
+
+def test_a_kmeans_step_never_increases_the_weighted_distortion():
+    # Lloyd iteration on a synthetic matrix with H = diag(h): both half steps are minimisations
+    rng = np.random.default_rng(22)
+    v, k, M, N = 8, 32, 64, 40
+    W = rng.normal(0, 1, (M, N)).astype(np.float16)
+    C = W[:v * 4, :8].reshape(4, v, 8).transpose(0, 2, 1).reshape(32, v).copy()       # 32 vectors of W as seeds
+    h = rng.uniform(0.2, 5.0, N).astype(np.float32)
+    idx = oracle.assign(W, v, C)
+    prev = oracle.distortion(W, v, idx, C, h)
+    for _ in range(6):
+        C = oracle.kmeans_update(W, v, idx, C, h)
+        after_update = oracle.distortion(W, v, idx, C, h)
+        assert after_update <= prev * (1 + 2e-3)          # centroids are rounded to FP16
+        idx = oracle.assign(W, v, C)
+        after_assign = oracle.distortion(W, v, idx, C, h)
+        assert after_assign <= after_update * (1 + 1e-6)
+        prev = after_assign
+    # ragged last vector row: components beyond M are neither read nor written
+    Wr = W[:61]
+    idx_r = oracle.assign(Wr, v, C)
+    Cr = oracle.kmeans_update(Wr, v, idx_r, C, h)
+    assert oracle.distortion(Wr, v, idx_r, Cr, h) <= oracle.distortion(Wr, v, idx_r, C, h) * (1 + 2e-3)
