@@ -261,6 +261,22 @@ int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
 int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
                 int32_t *idx, void *stream);
 
+/* Centroid update of (weighted) k-means (Sec. 2.2: k-means builds the codebook; Sec. 3.2.1: the diagonal
+ * term of the proxy error is a weighted k-means problem, the weight of a vector being the Hessian
+ * diagonal of its column): with the assignment `idx` fixed,
+ *   codebook[i][j] = sum h_n x_j / sum h_n   over the vectors (r, n) with idx[r][n] = i that have
+ * component j (x = W[r*v + j][n], h_n = col_weight[n], or 1 when col_weight is null); a component that
+ * received no weight keeps its old value, an index outside [0,k) takes no part.  vptq_assign followed
+ * by this call is one Lloyd iteration.
+ *   W fp16 [M][N], idx int32 [ceil(M/v)][N], col_weight fp32 [N] or null, codebook fp16 [k][v]
+ *   (read and written), workspace of vptq_kmeans_update_workspace_bytes(v, k) bytes (all device).
+ * Sums are FP32 atomics: the result agrees with the FP64 weighted mean to FP32 summation error (then
+ * rounded to FP16), not bit for bit, and may differ from run to run in the last FP16 bit. */
+int64_t vptq_kmeans_update_workspace_bytes(int32_t v, int32_t k);
+int vptq_kmeans_update(const void *W, int32_t M, int32_t N, int32_t v, const int32_t *idx,
+                       const float *col_weight, int32_t k, void *codebook,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- diagnostics ------------------------------------------------------------------ */
 
 const char *vptq_status_string(int code);

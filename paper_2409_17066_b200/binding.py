@@ -60,6 +60,9 @@ EXPORTS = {
     "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
     "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "vptq_kmeans_update_workspace_bytes": (C.c_int64, [C.c_int32, C.c_int32]),
+    "vptq_kmeans_update": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                     C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "vptq_linear_workspace_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_int32, C.POINTER(LayerPtrs),
                               C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -171,6 +174,23 @@ def vptq_assign(W: torch.Tensor, v: int, codebook: torch.Tensor) -> torch.Tensor
     idx = torch.empty((-(-M // v), N), dtype=torch.int32, device=W.device)
     _check(lib.vptq_assign(_ptr(W), M, N, v, _ptr(codebook), k, _ptr(idx), _stream()))
     return idx
+
+
+def vptq_kmeans_update(W: torch.Tensor, v: int, idx: torch.Tensor, codebook: torch.Tensor,
+                       col_weight: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Weighted k-means centroid update (Sec. 3.2.1), in place on `codebook` (fp16 [k][v])."""
+    assert W.is_cuda and W.dtype == torch.float16 and W.is_contiguous()
+    assert idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()
+    assert codebook.is_cuda and codebook.dtype == torch.float16 and codebook.is_contiguous()
+    assert col_weight is None or (col_weight.is_cuda and col_weight.dtype == torch.float32 and col_weight.is_contiguous())
+    M, N = W.shape
+    k = codebook.shape[0]
+    assert tuple(codebook.shape) == (k, v) and tuple(idx.shape) == (-(-M // v), N)
+    need = lib.vptq_kmeans_update_workspace_bytes(v, k)
+    ws = torch.empty(need, dtype=torch.uint8, device=W.device)
+    _check(lib.vptq_kmeans_update(_ptr(W), M, N, v, _ptr(idx), _ptr(col_weight), k, _ptr(codebook),
+                                  _ptr(ws), need, _stream()))
+    return codebook
 
 
 def vptq_linear_workspace_bytes(desc: LayerDesc, B: int) -> int:

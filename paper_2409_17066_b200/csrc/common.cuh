@@ -106,6 +106,10 @@ cudaError_t launch_unpack(const uint8_t *packed, int rows, int cols, int k, int3
 cudaError_t launch_dequant(const LayerView &L, __half *W, cudaStream_t st);
 // assignment step of the quantizer (Eq. 2): idx [ceil(M/v)][N]
 bool assign_supported(int v, int k);
+// (weighted) k-means centroid update (Sec. 3.2.1); workspace = 2*k*v floats
+long long kmeans_update_workspace_bytes(int v, int k);
+cudaError_t launch_kmeans_update(const __half *W, int M, int N, int v, const int *idx, const float *h, int k,
+                                 __half *C, void *ws, cudaStream_t st);
 cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st);
 
 // generic fallback linear (any geometry, any B): workspace = B*M floats

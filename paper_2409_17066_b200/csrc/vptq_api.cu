@@ -199,6 +199,29 @@ int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *code
     return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 
+int64_t vptq_kmeans_update_workspace_bytes(int32_t v, int32_t k)
+{
+    if (v < 1 || v > 32 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    return kmeans_update_workspace_bytes(v, k);
+}
+
+int vptq_kmeans_update(const void *W, int32_t M, int32_t N, int32_t v, const int32_t *idx,
+                       const float *col_weight, int32_t k, void *codebook,
+                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (M < 0 || N < 0 || v < 1 || v > 32 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (codebook == nullptr) return VPTQ_E_NULL;
+    if (M > 0 && N > 0 && (W == nullptr || idx == nullptr)) return VPTQ_E_NULL;
+    if (workspace == nullptr || (long long)workspace_bytes < kmeans_update_workspace_bytes(v, k)) return VPTQ_E_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(W) & 1u) || (reinterpret_cast<uintptr_t>(codebook) & 1u) ||
+        (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(col_weight) & 3u) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 3u)) return VPTQ_E_ALIGN;
+    cudaError_t e = launch_kmeans_update(reinterpret_cast<const __half *>(W), M, N, v, idx, col_weight, k,
+                                         reinterpret_cast<__half *>(codebook), workspace,
+                                         reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
+}
+
 int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B)
 {
     int rc = check_desc(desc);

@@ -284,3 +284,43 @@ def test_assign_then_pack_and_dequant_reproduce_the_matrix(b):
     again = b.vptq_pack(idx, spec.k1)
     assert torch.equal(again, dl.idx1) or np.array_equal(
         oracle.Layer.from_synth(dict(d, idx1=idx.cpu().numpy())).dequant().view(np.uint16), W.cpu().numpy().view(np.uint16))
+
+
+# ------------------------------------------------------------------ k-means centroid update (Sec. 3.2.1)
+
+@pytest.mark.parametrize("M,N,v,k,weighted", [
+    (136, 520, 8, 4096, True),      # sums straight into the workspace
+    (130, 333, 6, 300, True),       # shared-memory copy per block, ragged last vector row
+    (64, 40, 8, 32, False),         # unweighted
+    (60, 134, 12, 5000, True),
+])
+def test_kmeans_update_matches_the_weighted_mean(b, M, N, v, k, weighted):
+    rng = np.random.default_rng(7 * k + v)
+    W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
+    Cb = rng.normal(0, 0.02, (k, v)).astype(np.float16)
+    h = rng.uniform(0.2, 5.0, N).astype(np.float32) if weighted else None
+    idx = oracle.assign(W, v, Cb)
+    want = oracle.kmeans_update(W, v, idx, Cb, h).astype(np.float64)
+    got = b.vptq_kmeans_update(torch.from_numpy(W).cuda(), v, torch.from_numpy(idx).cuda(), torch.from_numpy(Cb).cuda(),
+                               None if h is None else torch.from_numpy(h).cuda()).cpu().numpy().astype(np.float64)
+    # FP32 atomic sums against the FP64 mean: at most the last FP16 bit
+    assert np.all(np.abs(got - want) <= 2.0 ** -10 * np.abs(want) + 1e-7)
+    # centroids nobody was assigned to are untouched, bit for bit
+    unused = np.setdiff1d(np.arange(k), np.unique(idx))
+    assert np.array_equal(got[unused], Cb[unused].astype(np.float64))
+
+
+def test_lloyd_iterations_on_the_gpu_decrease_the_distortion(b):
+    rng = np.random.default_rng(23)
+    v, k, M, N = 8, 256, 256, 300
+    W = rng.normal(0, 1, (M, N)).astype(np.float16)
+    h = rng.uniform(0.2, 5.0, N).astype(np.float32)
+    Wd, hd = torch.from_numpy(W).cuda(), torch.from_numpy(h).cuda()
+    Cd = torch.from_numpy(rng.normal(0, 1, (k, v)).astype(np.float16)).cuda()
+    prev = None
+    for _ in range(5):
+        idx = b.vptq_assign(Wd, v, Cd)
+        b.vptq_kmeans_update(Wd, v, idx, Cd, hd)
+        dist = oracle.distortion(W, v, idx.cpu().numpy(), Cd.cpu().numpy(), h)
+        assert prev is None or dist <= prev * (1 + 2e-3)
+        prev = dist
