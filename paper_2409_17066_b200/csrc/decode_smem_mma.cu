@@ -136,11 +136,14 @@ __device__ __forceinline__ void load16_elems(const uint16_t *__restrict__ base, 
 
 // 16 scaled activations (x*s, FP16) for token t, absolute columns [n0, n0+16); columns at or
 // beyond n_end read as zero.
+// (PERM: the layer has a stored column order; a template parameter so that the plain case keeps its
+// loads free of branches and the compiler can issue them together)
+template <bool PERM>
 __device__ __forceinline__ void load_xs16(const SmemMmaParams &P, int t, int n0, int n_end, uint32_t (&hw)[8])
 {
     const LayerView &L = P.L;
     uint32_t xw[8];
-    if (L.perm != nullptr) {
+    if (PERM) {
         // a stored column order: the 16 activations are gathered one by one
         const uint16_t *xr = reinterpret_cast<const uint16_t *>(P.x) + (long long)t * L.N;
 #pragma unroll
@@ -221,7 +224,7 @@ __device__ __forceinline__ void decode8(uint4 q, int bits, int k, uint32_t (&w)[
     for (int i = 0; i < 4; i++) w[i] = __vminu2(w[i], lim);
 }
 
-template <int NT>   // NT = 1: up to 8 tokens, NT = 2: up to 16 tokens
+template <int NT, bool PERM>   // NT = 1: up to 8 tokens, NT = 2: up to 16 tokens
 __global__ void __launch_bounds__(THREADS, 1)
 decode_smem_mma_kernel(SmemMmaParams P)
 {
@@ -258,7 +261,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
                 float bn = L.scale_rows ? 1.f : __half2float(__ldg(L.bias + n));
 #pragma unroll
                 for (int t = 0; t < TP; t++)
-                    if (t < P.B) acc[t] += load_act(P.x, (long long)t * L.N + in_col(L, n), L.x_bf16) * bn;
+                    if (t < P.B) acc[t] += load_act(P.x, (long long)t * L.N + (PERM ? in_col(L, n) : n), L.x_bf16) * bn;
             }
         }
 #pragma unroll
@@ -305,7 +308,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
                         const int t = g + 8 * th;
                         uint32_t hw[8];
                         if (t < P.B && n0 < n_end) {
-                            load_xs16(P, t, n0, n_end, hw);
+                            load_xs16<PERM>(P, t, n0, n_end, hw);
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; i++) hw[i] = 0u;
@@ -415,7 +418,7 @@ decode_smem_mma_kernel(SmemMmaParams P)
                         float xv[4];
 #pragma unroll
                         for (int t = 0; t < 4; t++)
-                            xv[t] = (t0 + t < P.B) ? load_act(P.x, (long long)(t0 + t) * L.N + in_col(L, n), L.x_bf16) * sc : 0.f;
+                            xv[t] = (t0 + t < P.B) ? load_act(P.x, (long long)(t0 + t) * L.N + (PERM ? in_col(L, n) : n), L.x_bf16) * sc : 0.f;
 #pragma unroll
                         for (int j = 0; j < 8; j++) {
                             if (j < L.v0) {
@@ -487,6 +490,24 @@ static int num_sms()
     return g_num_sms;
 }
 
+namespace {
+template <int NT>
+cudaError_t launch_variant(const SmemMmaParams &P, bool perm, int grid, size_t smem, cudaStream_t st)
+{
+    cudaError_t e;
+    if (perm) {
+        e = cudaFuncSetAttribute(decode_smem_mma_kernel<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        decode_smem_mma_kernel<NT, true><<<grid, THREADS, smem, st>>>(P);
+    } else {
+        e = cudaFuncSetAttribute(decode_smem_mma_kernel<NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        decode_smem_mma_kernel<NT, false><<<grid, THREADS, smem, st>>>(P);
+    }
+    return cudaGetLastError();
+}
+}  // namespace
+
 cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st)
 {
     SmemMmaParams P;
@@ -505,17 +526,8 @@ cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, voi
     P.rows_per_pass = rpp;
     const int grid = ceil_div(L.R, P.rows_per_cta);
     const size_t smem = (size_t)P.cb1_bytes + P.cb2_bytes + (size_t)rpp * per_row + (TP + WARPS * TP) * 4;
-    cudaError_t e;
-    if (NT == 1) {
-        e = cudaFuncSetAttribute(decode_smem_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        decode_smem_mma_kernel<1><<<grid, THREADS, smem, st>>>(P);
-    } else {
-        e = cudaFuncSetAttribute(decode_smem_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        decode_smem_mma_kernel<2><<<grid, THREADS, smem, st>>>(P);
-    }
-    return cudaGetLastError();
+    return NT == 1 ? launch_variant<1>(P, L.perm != nullptr, grid, smem, st)
+                   : launch_variant<2>(P, L.perm != nullptr, grid, smem, st);
 }
 
 }  // namespace vptq
