@@ -50,8 +50,8 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     "decode_l2_fma_kernel": 1.021,
     # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.95 MB
     "decode_smem_fma_kernel": 1.003,
-    # profiles/decode_smem_mma_kernel_config2_gate_proj_B8.md: 19.09 MB / 19.0 MB
-    "decode_smem_mma_kernel": 1.004,
+    # profiles/decode_smem_mma_kernel_config2_gate_proj_B8.md: 19.10 MB / 19.0 MB
+    "decode_smem_mma_kernel": 1.005,
 }
 
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
