@@ -257,9 +257,19 @@ int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
  * Arithmetic, fixed because it decides an integer: FP32, components in ascending order,
  * d = fma(t, t, d) with t = x_j - c_j; of equal distances the lowest index wins; a NaN distance never
  * wins (all NaN: index 0); components beyond row M-1 (short last vector row) are left out.
+ * Two kernels give these same indices: "assign_fp32" evaluates the definition for every pair;
+ * "assign_tcgen05" (v <= 14, v divides M, k >= 1024, at least 4096 vectors) computes
+ * ||c||^2 - 2 x.c on the tensor cores only to find, per vector, the group of 32 centroids that holds
+ * the minimum, evaluates that group by the definition, and hands every vector whose candidate group is
+ * not clearly the only one (within a bound on the tensor core's rounding) to the first kernel.
+ * vptq_assign_path() names the kernel; VPTQ_FLAG_FORCE_GENERIC in `flags` selects "assign_fp32".
+ * The tensor-core kernel needs a workspace of vptq_assign_workspace_bytes() bytes (256-byte aligned;
+ * its first int32 is a status word read by vptq_workspace_status()); the other needs none.
  * 1 <= v <= 32, 1 <= k <= 65536, else VPTQ_E_SHAPE / VPTQ_E_UNSUPPORTED.  Asynchronous on `stream`. */
+const char *vptq_assign_path(int32_t M, int32_t N, int32_t v, int32_t k, int32_t flags);
+int64_t vptq_assign_workspace_bytes(int32_t M, int32_t N, int32_t v, int32_t k, int32_t flags);
 int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
-                int32_t *idx, void *stream);
+                int32_t *idx, int32_t flags, void *workspace, size_t workspace_bytes, void *stream);
 
 /* Centroid update of (weighted) k-means (Sec. 2.2: k-means builds the codebook; Sec. 3.2.1: the diagonal
  * term of the proxy error is a weighted k-means problem, the weight of a vector being the Hessian

@@ -59,7 +59,10 @@ EXPORTS = {
     "vptq_pack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
-    "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
+                              C.c_void_p, C.c_size_t, C.c_void_p]),
+    "vptq_assign_workspace_bytes": (C.c_int64, [C.c_int32] * 5),
+    "vptq_assign_path": (C.c_char_p, [C.c_int32] * 5),
     "vptq_kmeans_update_workspace_bytes": (C.c_int64, [C.c_int32, C.c_int32]),
     "vptq_kmeans_update": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -164,15 +167,29 @@ def vptq_dequant(desc: LayerDesc, ptrs: LayerPtrs, W_out: torch.Tensor) -> torch
     return W_out
 
 
-def vptq_assign(W: torch.Tensor, v: int, codebook: torch.Tensor) -> torch.Tensor:
-    """Eq. 2: int32 [ceil(M/v)][N] index of the nearest centroid of every length-v vector of W (fp16 [M][N])."""
+def vptq_assign_path(M: int, N: int, v: int, k: int, flags: int = 0) -> str:
+    return lib.vptq_assign_path(M, N, v, k, flags).decode()
+
+
+def vptq_assign(W: torch.Tensor, v: int, codebook: torch.Tensor, flags: int = 0,
+                workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Eq. 2: int32 [ceil(M/v)][N] index of the nearest centroid of every length-v vector of W (fp16 [M][N]).
+    flags = FLAG_FORCE_GENERIC selects the plain FP32 kernel; both kernels give the same indices."""
     assert W.is_cuda and W.dtype == torch.float16 and W.dim() == 2 and W.is_contiguous()
     assert codebook.is_cuda and codebook.dtype == torch.float16 and codebook.is_contiguous()
     M, N = W.shape
     k = codebook.shape[0]
     assert tuple(codebook.shape) == (k, v)
     idx = torch.empty((-(-M // v), N), dtype=torch.int32, device=W.device)
-    _check(lib.vptq_assign(_ptr(W), M, N, v, _ptr(codebook), k, _ptr(idx), _stream()))
+    need = lib.vptq_assign_workspace_bytes(M, N, v, k, flags)
+    if need < 0:
+        raise VptqError(int(need))
+    if need and workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=W.device)
+    _check(lib.vptq_assign(_ptr(W), M, N, v, _ptr(codebook), k, _ptr(idx), flags, _ptr(workspace),
+                           0 if workspace is None else workspace.numel(), _stream()))
+    if need:
+        _check(lib.vptq_workspace_status(_ptr(workspace), _stream()))
     return idx
 
 

@@ -13,6 +13,7 @@
 // same centroid (broadcast).  The work is n_vectors * k * v subtract + fma pairs: bound by the FP32
 // pipes, not by memory (the codebook is re-read from L2 once per block).
 #include "common.cuh"
+#include "assign.cuh"
 
 namespace vptq {
 
@@ -24,12 +25,20 @@ constexpr int CHUNK_FLOATS = 4096;        // 16 KB of shared memory: CHUNK_FLOAT
 template <int VMAX>
 __global__ void __launch_bounds__(ASSIGN_THREADS)
 assign_kernel(const __half *__restrict__ W, int M, int N, int v, const __half *__restrict__ C, int k,
-              int *__restrict__ idx, long long n_vectors)
+              int *__restrict__ idx, long long n_vectors, const int *__restrict__ list, const int *__restrict__ count)
 {
     constexpr int CHUNK = CHUNK_FLOATS / VMAX;
     __shared__ __align__(16) float cb[CHUNK_FLOATS];
-    const long long g = (long long)blockIdx.x * ASSIGN_THREADS + threadIdx.x;
-    const bool valid = g < n_vectors;
+    // all vectors, or (list != nullptr) the vectors list[0 .. *count) only
+    const long long slot = (long long)blockIdx.x * ASSIGN_THREADS + threadIdx.x;
+    long long g = slot;
+    bool valid = slot < n_vectors;
+    if (list != nullptr) {
+        const int cnt = __ldg(count);
+        if ((long long)blockIdx.x * ASSIGN_THREADS >= cnt) return;       // the whole block has nothing to do
+        valid = slot < cnt;
+        g = valid ? __ldg(list + slot) : 0;
+    }
     const int r = valid ? (int)(g / N) : 0, n = valid ? (int)(g % N) : 0;
     const int vlen = min(v, M - r * v);              // components of this vector that exist
     float x[VMAX];
@@ -79,18 +88,24 @@ assign_kernel(const __half *__restrict__ W, int M, int N, int v, const __half *_
 
 bool assign_supported(int v, int k) { return v >= 1 && v <= 32 && k >= 1 && k <= 65536; }
 
-cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st)
+cudaError_t launch_assign_listed(const __half *W, int M, int N, int v, const __half *C, int k, int *idx,
+                                 const int *list, const int *count, long long n_vectors, cudaStream_t st)
 {
-    const long long n_vectors = (long long)ceil_div(M, v) * N;
     if (n_vectors == 0) return cudaSuccess;
+    // (with a list the grid is sized for the worst case, every vector listed; blocks beyond the count return at once)
     const long long blocks = (n_vectors + ASSIGN_THREADS - 1) / ASSIGN_THREADS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     const dim3 grid((unsigned)blocks);
-    if (v <= 4) assign_kernel<4><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
-    else if (v <= 8) assign_kernel<8><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
-    else if (v <= 16) assign_kernel<16><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
-    else assign_kernel<32><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
+    if (v <= 4) assign_kernel<4><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
+    else if (v <= 8) assign_kernel<8><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
+    else if (v <= 16) assign_kernel<16><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
+    else assign_kernel<32><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
     return cudaGetLastError();
+}
+
+cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st)
+{
+    return launch_assign_listed(W, M, N, v, C, k, idx, nullptr, nullptr, (long long)ceil_div(M, v) * N, st);
 }
 
 }  // namespace vptq

@@ -1,0 +1,450 @@
+// Assignment step of the quantizer (Eq. 2) on the tensor cores, with the result of the FP32 definition.
+//
+// The squared distance is ||c||^2 - 2 x.c + ||x||^2, and the first two terms are a contraction over the
+// vector's components: D[vector][centroid] = A * B^T with
+//   A row (a vector):   x_0 .. x_{v-1}, 0 .., 1, 1          (16 FP16 values, K = 16)
+//   B row (a centroid): -2c_0 .. -2c_{v-1}, 0 .., hi, lo     hi + lo = ||c||^2 split into two FP16 values
+// One tcgen05.mma (M = 128 vectors, N = 128 centroids, K = 16) gives 16 K approximate distances.  They
+// only FILTER: per vector the kernel keeps the smallest and the second smallest minimum over groups of
+// 32 centroids and the group of the smallest.  Then the 32 centroids of that group are evaluated with
+// the arithmetic that defines the result (FP32 fma chain, lowest index wins: the same code as the plain
+// kernel), and a vector whose two group minima are closer than a bound on the filter's error is put on
+// a list; the plain kernel scans all centroids for the vectors on the list.  The indices are therefore
+// those of the FP32 definition, bit for bit, whatever the tensor core's summation order.
+//   bound: |filter - (definition - ||x||^2)| <= 2^-18 (||x||^2 + max ||c||^2) (FP16 split of the norm,
+//   FP32 accumulation of 10 products, rounding of the fma chain); the margin tested is 2^-14 of it.
+//
+// Persistent grid, one CTA per SM, 256 vectors (two A tiles) per step.  Warp 0 streams the prepared
+// centroid tiles (4 KB, shared-memory image with the 32-byte swizzle applied by the preparation kernel)
+// with linear bulk copies into a ring; warp 1 issues the MMAs (two per centroid tile, fresh accumulators
+// in one of two TMEM buffers); warps 2-9 write the A tiles of a step, then drain the accumulators: a lane
+// owns one vector, reads 32 distances per tcgen05.ld and keeps its two running minima (35 instructions
+// per 32 distances: the epilogue, not the tensor core, bounds the kernel).
+// Every mbarrier wait is bounded; a wait that gives up sets the status word of the workspace.
+#include "common.cuh"
+#include "assign.cuh"
+
+namespace vptq {
+
+namespace {
+
+constexpr int KT = 128;                       // centroids per tile (N of the MMA)
+constexpr int ROW_BYTES = 32;                 // K = 16 FP16 values
+constexpr int TILE_BYTES = KT * ROW_BYTES;    // 4 KB: an A tile (128 vectors) or a B tile (128 centroids)
+constexpr int B_STAGES = 8;
+constexpr int EPI_WARPS = 8;
+constexpr int SCAN_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int STEP_VECTORS = 256;             // two A tiles
+constexpr int GROUP = 32;                     // centroids per candidate group (one tcgen05.ld)
+constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
+constexpr float PAD_NORM = 60000.f;           // norm of the padding rows of the last centroid tile: never the minimum
+constexpr float MARGIN = 1.0f / 16384.0f;     // 2^-14
+
+struct ScanParams {
+    const __half *W;
+    int M, N, v, k;
+    const __half *C;          // [k][v]
+    const uint8_t *Bimg;      // [k_tiles][TILE_BYTES]
+    const float *cmax;        // max ||c||^2
+    int *idx;                 // [n_vectors]
+    int *list;                // vectors that need the full scan
+    int *count;               // entries of the list
+    int *status;
+    long long n_vectors;
+    int k_tiles;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred P1;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+                 "selp.b32 %0, 1, 0, P1;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when it was abandoned (time limit here, or the abort flag raised elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, VPTQ_E_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// K-major operand with 32-byte rows and the 32-byte swizzle: 8-row groups of 256 bytes
+__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                              // leading-dimension offset: unused for one swizzle row
+    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;         // stride between 8-row groups
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                              // 32-byte swizzle
+    return d;
+}
+// kind::f16: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
+constexpr uint32_t SCAN_IDESC = (1u << 4) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+__device__ __forceinline__ void umma_fresh(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(SCAN_IDESC) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 32 consecutive accumulator columns of this lane's row: the load is only issued here ...
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+}
+// ... and its registers may be read after this wait (they are operands of the wait so that no use moves above it)
+__device__ __forceinline__ void tmem_ld32_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+// smallest of 32 values
+__device__ __forceinline__ float min32(const uint32_t (&d)[32])
+{
+    float m[16];
+#pragma unroll
+    for (int j = 0; j < 16; j++) m[j] = fminf(__uint_as_float(d[j]), __uint_as_float(d[j + 16]));
+#pragma unroll
+    for (int w = 8; w > 0; w >>= 1)
+#pragma unroll
+        for (int j = 0; j < w; j++) m[j] = fminf(m[j], m[j + w]);
+    return m[0];
+}
+
+// byte offset of 16-byte chunk c (0 or 1) of row r in a tile image (32-byte swizzle: bit 4 ^= bit 7)
+__device__ __forceinline__ int image_offset(int r, int c) { return r * ROW_BYTES + ((c ^ ((r >> 2) & 1)) << 4); }
+
+// ---- preparation: the centroid tiles as shared-memory images, and max ||c||^2 ---------------------------
+__global__ void __launch_bounds__(256)
+assign_prepare_kernel(const __half *__restrict__ C, int k, int v, uint8_t *__restrict__ Bimg, float *cmax,
+                      int *count, int *status, int k_tiles)
+{
+    const int i = blockIdx.x * 256 + threadIdx.x;          // centroid (or padding row of the last tile)
+    if (i == 0) { *count = 0; *status = 0; }
+    if (i >= k_tiles * KT) return;
+    __half row[16];
+#pragma unroll
+    for (int j = 0; j < 16; j++) row[j] = __float2half_rn(0.f);
+    float norm = PAD_NORM;
+    if (i < k) {
+        norm = 0.f;
+        for (int j = 0; j < v; j++) {
+            const float c = __half2float(__ldg(C + (long long)i * v + j));
+            norm = __fmaf_rn(c, c, norm);
+            row[j] = __float2half_rn(-2.f * c);             // exact (a power of two), overflow apart
+        }
+        atomicMax(reinterpret_cast<int *>(cmax), __float_as_int(norm));      // norm >= 0: integer order = float order
+    }
+    const __half hi = __float2half_rn(norm);
+    row[14] = hi;
+    row[15] = __float2half_rn(norm - __half2float(hi));
+    uint8_t *tile = Bimg + (long long)(i / KT) * TILE_BYTES;
+    const uint4 *src = reinterpret_cast<const uint4 *>(row);
+    *reinterpret_cast<uint4 *>(tile + image_offset(i % KT, 0)) = src[0];
+    *reinterpret_cast<uint4 *>(tile + image_offset(i % KT, 1)) = src[1];
+}
+
+// ---- the scan ---------------------------------------------------------------------------------------------
+template <int VMAX>
+__global__ void __launch_bounds__(SCAN_THREADS, 1)
+assign_scan_kernel(ScanParams P)
+{
+    __shared__ __align__(1024) uint8_t sA[2 * TILE_BYTES];
+    __shared__ __align__(1024) uint8_t sB[B_STAGES * TILE_BYTES];
+    __shared__ __align__(8) uint64_t bars[2 * B_STAGES + 5];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_word;
+    volatile int *abort_flag = &abort_word;
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar_fullB = [&](int s) { return bar0 + 8u * s; };
+    auto bar_emptyB = [&](int s) { return bar0 + 8u * (B_STAGES + s); };
+    auto bar_accFull = [&](int b) { return bar0 + 8u * (2 * B_STAGES + b); };
+    auto bar_accEmpty = [&](int b) { return bar0 + 8u * (2 * B_STAGES + 2 + b); };
+    const uint32_t bar_aFull = bar0 + 8u * (2 * B_STAGES + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < B_STAGES; s++) { mbar_init(bar_fullB(s), 1); mbar_init(bar_emptyB(s), 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(bar_accFull(b), 1); mbar_init(bar_accEmpty(b), EPI_WARPS); }
+        mbar_init(bar_aFull, EPI_WARPS);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    const long long n_steps = (P.n_vectors + STEP_VECTORS - 1) / STEP_VECTORS;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ================= centroid tiles: linear bulk copies into the ring =================
+        if (lane == 0) {
+            long long it = 0;
+            for (long long step = blockIdx.x; step < n_steps && ok; step += gridDim.x)
+                for (int kt = 0; kt < P.k_tiles; kt++, it++) {
+                    const int s = (int)(it % B_STAGES);
+                    if (!(ok = mbar_wait(bar_emptyB(s), (uint32_t)((it / B_STAGES) & 1) ^ 1u, abort_flag, P.status))) break;
+                    mbar_expect_tx(bar_fullB(s), TILE_BYTES);
+                    bulk_load(smem_u32(sB) + s * TILE_BYTES, P.Bimg + (long long)kt * TILE_BYTES, TILE_BYTES, bar_fullB(s));
+                }
+            if (!ok) {
+                // abandoned: give copies still in flight a bounded time to land before the CTA exits
+                const long long first = it > B_STAGES ? it - B_STAGES : 0;
+                for (long long j = first; j < it; j++) {
+                    const long long t0c = clock64();
+                    while (!mbar_try(bar_fullB((int)(j % B_STAGES)), (uint32_t)((j / B_STAGES) & 1)) &&
+                           clock64() - t0c < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issue =================
+        if (lane == 0) {
+            const uint64_t adesc0 = operand_desc(smem_u32(sA));
+            const uint64_t bdesc0 = operand_desc(smem_u32(sB));
+            long long it = 0, step_no = 0;
+            for (long long step = blockIdx.x; step < n_steps && ok; step += gridDim.x, step_no++) {
+                if (!(ok = mbar_wait(bar_aFull, (uint32_t)(step_no & 1), abort_flag, P.status))) break;
+                for (int kt = 0; kt < P.k_tiles; kt++, it++) {
+                    const int s = (int)(it % B_STAGES), b = (int)(it & 1);
+                    if (!(ok = mbar_wait(bar_fullB(s), (uint32_t)((it / B_STAGES) & 1), abort_flag, P.status))) break;
+                    if (!(ok = mbar_wait(bar_accEmpty(b), (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag, P.status))) break;
+                    tc_fence_after();
+                    const uint64_t bd = bdesc0 + (uint64_t)((s * TILE_BYTES) >> 4);
+                    umma_fresh(tmem_base + (uint32_t)((b * 2 + 0) * KT), adesc0, bd);
+                    umma_fresh(tmem_base + (uint32_t)((b * 2 + 1) * KT), adesc0 + (uint64_t)(TILE_BYTES >> 4), bd);
+                    umma_commit(bar_emptyB(s));
+                    umma_commit(bar_accFull(b));
+                }
+            }
+        }
+    } else {
+        // ================= A tiles, then the running minima; a lane owns one vector of the step =================
+        const int ew = warp - 2;
+        const int q = warp & 3;                      // TMEM lane quarter this warp may read
+        const int a = ew >> 2;                       // A tile
+        const int row = 32 * q + lane;               // row of the A tile = TMEM lane
+        const float cmax = __ldg(P.cmax);
+        long long it = 0;
+        for (long long step = blockIdx.x; step < n_steps && ok; step += gridDim.x) {
+            const long long g = step * STEP_VECTORS + a * 128 + row;
+            const bool valid = g < P.n_vectors;
+            const int r = valid ? (int)(g / P.N) : 0, n = valid ? (int)(g % P.N) : 0;
+            float x[VMAX];
+            float xn = 0.f;
+#pragma unroll
+            for (int j = 0; j < VMAX; j++) {
+                x[j] = (valid && j < P.v) ? __half2float(__ldg(P.W + (long long)(r * P.v + j) * P.N + n)) : 0.f;
+                xn = __fmaf_rn(x[j], x[j], xn);
+            }
+            // the A tile of this step may be overwritten: its MMAs completed before the last accFull of the previous step
+            {
+                __half rowv[16];
+#pragma unroll
+                for (int j = 0; j < 14; j++) rowv[j] = __float2half_rn(j < VMAX ? x[j < VMAX ? j : 0] : 0.f);   // exact: x came from FP16
+                rowv[14] = __float2half_rn(1.f);         // times hi
+                rowv[15] = __float2half_rn(1.f);         // times lo
+                const uint4 *src = reinterpret_cast<const uint4 *>(rowv);
+                uint8_t *tile = sA + a * TILE_BYTES;
+                *reinterpret_cast<uint4 *>(tile + image_offset(row, 0)) = src[0];
+                *reinterpret_cast<uint4 *>(tile + image_offset(row, 1)) = src[1];
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_aFull);
+            }
+            float b1 = __int_as_float(0x7f800000), b2 = b1;
+            int g1 = 0;
+            for (int kt = 0; kt < P.k_tiles; kt++, it++) {
+                const int b = (int)(it & 1);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_accFull(b), (uint32_t)((it >> 1) & 1), abort_flag, P.status));
+                if (!ok) break;
+                tc_fence_after();
+                // the load of the next group of 32 distances is in flight while this one is reduced
+                const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)((b * 2 + a) * KT);
+                uint32_t d0[32], d1[32];
+                tmem_ld32_issue(t_row, d0);
+#pragma unroll
+                for (int grp = 0; grp < KT / GROUP; grp += 2) {
+                    tmem_ld32_wait(d0);
+                    tmem_ld32_issue(t_row + (uint32_t)((grp + 1) * GROUP), d1);
+                    float gm = min32(d0);
+                    if (gm < b1) { b2 = b1; b1 = gm; g1 = kt * (KT / GROUP) + grp; }
+                    else if (gm < b2) b2 = gm;
+                    tmem_ld32_wait(d1);
+                    if (grp + 2 < KT / GROUP) tmem_ld32_issue(t_row + (uint32_t)((grp + 2) * GROUP), d0);
+                    gm = min32(d1);
+                    if (gm < b1) { b2 = b1; b1 = gm; g1 = kt * (KT / GROUP) + grp + 1; }
+                    else if (gm < b2) b2 = gm;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_accEmpty(b));
+            }
+            if (!ok) break;
+            if (valid) {
+                // the group of the smallest filter value, with the arithmetic that defines the result
+                int best = 0;
+                float best_d = __int_as_float(0x7f800000);
+                const int i0 = g1 * GROUP, i1 = min(P.k, i0 + GROUP);
+                for (int i = i0; i < i1; i++) {
+                    float dd = 0.f;
+#pragma unroll
+                    for (int j = 0; j < VMAX; j++) {
+                        const float c = j < P.v ? __half2float(__ldg(P.C + (long long)i * P.v + j)) : 0.f;
+                        const float t = __fsub_rn(x[j], c);
+                        dd = __fmaf_rn(t, t, dd);
+                    }
+                    if (dd < best_d) { best_d = dd; best = i; }
+                }
+                P.idx[g] = best;
+                // not clearly the only candidate group: the full scan decides
+                const float eps = MARGIN * (xn + cmax);
+                // (norms beyond the FP16 range make the filter meaningless: then every vector is listed)
+                if (!(b2 - b1 > eps) || !(fabsf(b1) < 3.0e38f) || !(cmax < PAD_NORM)) P.list[atomicAdd(P.count, 1)] = (int)g;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncwarp();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+int scan_sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+        else return 148;
+    }
+    return n;
+}
+
+struct ScanLayout {
+    long long off_cmax, off_count, off_bimg, off_list, bytes;
+    int k_tiles;
+};
+
+ScanLayout scan_layout(long long n_vectors, int k)
+{
+    ScanLayout l;
+    l.k_tiles = ceil_div(k, KT);
+    l.off_cmax = 16;                    // status word at byte 0
+    l.off_count = 32;
+    l.off_bimg = 256;
+    l.off_list = l.off_bimg + (long long)l.k_tiles * TILE_BYTES;
+    l.bytes = l.off_list + (n_vectors * 4 + 255) / 256 * 256;
+    return l;
+}
+
+}  // namespace
+
+// vectors of at most 14 components (two of the 16 K columns carry the norm), whole vector rows, enough
+// centroids for the filter to pay, vector numbers that fit an int
+bool assign_tcgen05_supported(int M, int N, int v, int k)
+{
+    if (v < 1 || v > 14 || k < 1024 || k > 65536 || M % v != 0) return false;
+    return (long long)(M / v) * N < 0x7fffffffLL && (long long)(M / v) * N >= 4096;
+}
+
+long long assign_tcgen05_workspace_bytes(int M, int N, int v, int k)
+{
+    return scan_layout((long long)ceil_div(M, v) * N, k).bytes;
+}
+
+cudaError_t launch_assign_tcgen05(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, void *ws,
+                                  cudaStream_t st)
+{
+    const long long n_vectors = (long long)(M / v) * N;
+    const ScanLayout l = scan_layout(n_vectors, k);
+    uint8_t *w8 = reinterpret_cast<uint8_t *>(ws);
+    ScanParams P;
+    P.W = W; P.M = M; P.N = N; P.v = v; P.k = k; P.C = C;
+    P.Bimg = w8 + l.off_bimg;
+    P.cmax = reinterpret_cast<const float *>(w8 + l.off_cmax);
+    P.idx = idx;
+    P.list = reinterpret_cast<int *>(w8 + l.off_list);
+    P.count = reinterpret_cast<int *>(w8 + l.off_count);
+    P.status = reinterpret_cast<int *>(w8);
+    P.n_vectors = n_vectors;
+    P.k_tiles = l.k_tiles;
+    cudaError_t e = cudaMemsetAsync(w8 + l.off_cmax, 0, 4, st);
+    if (e != cudaSuccess) return e;
+    assign_prepare_kernel<<<ceil_div(l.k_tiles * KT, 256), 256, 0, st>>>(C, k, v, w8 + l.off_bimg,
+                                                                         reinterpret_cast<float *>(w8 + l.off_cmax),
+                                                                         P.count, P.status, l.k_tiles);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long n_steps = (n_vectors + STEP_VECTORS - 1) / STEP_VECTORS;
+    const int grid = (int)(n_steps < scan_sm_count() ? n_steps : scan_sm_count());
+    if (v <= 8) assign_scan_kernel<8><<<grid, SCAN_THREADS, 0, st>>>(P);
+    else assign_scan_kernel<14><<<grid, SCAN_THREADS, 0, st>>>(P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // the vectors whose candidate group was not clearly the only one: all centroids, FP32
+    return launch_assign_listed(W, M, N, v, C, k, idx, P.list, P.count, n_vectors, st);
+}
+
+}  // namespace vptq

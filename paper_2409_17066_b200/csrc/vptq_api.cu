@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "paths.cuh"
+#include "assign.cuh"
 
 using namespace vptq;
 
@@ -184,18 +185,46 @@ int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, void *W_
     return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 
-int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
-                int32_t *idx, void *stream)
+static bool assign_uses_tensor_cores(int32_t M, int32_t N, int32_t v, int32_t k, int32_t flags)
+{
+    return !(flags & VPTQ_FLAG_FORCE_GENERIC) && assign_tcgen05_supported(M, N, v, k);
+}
+
+const char *vptq_assign_path(int32_t M, int32_t N, int32_t v, int32_t k, int32_t flags)
+{
+    if (M < 0 || N < 0 || v < 1 || k < 1 || k > 65536 || !assign_supported(v, k)) return "invalid";
+    return assign_uses_tensor_cores(M, N, v, k, flags) ? "assign_tcgen05" : "assign_fp32";
+}
+
+int64_t vptq_assign_workspace_bytes(int32_t M, int32_t N, int32_t v, int32_t k, int32_t flags)
 {
     if (M < 0 || N < 0 || v < 1 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
     if (!assign_supported(v, k)) return VPTQ_E_UNSUPPORTED;
+    return assign_uses_tensor_cores(M, N, v, k, flags) ? assign_tcgen05_workspace_bytes(M, N, v, k) : 0;
+}
+
+int vptq_assign(const void *W, int32_t M, int32_t N, int32_t v, const void *codebook, int32_t k,
+                int32_t *idx, int32_t flags, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (M < 0 || N < 0 || v < 1 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (!assign_supported(v, k)) return VPTQ_E_UNSUPPORTED;
+    if (flags & ~VPTQ_FLAG_FORCE_GENERIC) return VPTQ_E_UNSUPPORTED;
     if (M == 0 || N == 0) return VPTQ_OK;
     if (W == nullptr || codebook == nullptr || idx == nullptr) return VPTQ_E_NULL;
     if ((reinterpret_cast<uintptr_t>(W) & 1u) || (reinterpret_cast<uintptr_t>(codebook) & 1u) ||
         (reinterpret_cast<uintptr_t>(idx) & 3u)) return VPTQ_E_ALIGN;
-    cudaError_t e = launch_assign(reinterpret_cast<const __half *>(W), M, N, v,
-                                  reinterpret_cast<const __half *>(codebook), k, idx,
-                                  reinterpret_cast<cudaStream_t>(stream));
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (assign_uses_tensor_cores(M, N, v, k, flags)) {
+        if (workspace == nullptr || (long long)workspace_bytes < assign_tcgen05_workspace_bytes(M, N, v, k))
+            return VPTQ_E_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return VPTQ_E_ALIGN;
+        e = launch_assign_tcgen05(reinterpret_cast<const __half *>(W), M, N, v,
+                                  reinterpret_cast<const __half *>(codebook), k, idx, workspace, st);
+    } else {
+        e = launch_assign(reinterpret_cast<const __half *>(W), M, N, v,
+                          reinterpret_cast<const __half *>(codebook), k, idx, st);
+    }
     return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 

@@ -118,3 +118,19 @@ def test_fused_call_argument_errors_and_path_names(binding):
     assert b.vptq_linear_fused_workspace_bytes([q, kv], 64) == max(b.vptq_linear_workspace_bytes(q, 64),
                                                                   b.vptq_linear_workspace_bytes(kv, 64))
 
+
+def test_assign_path_and_workspace_queries(binding):
+    b = binding
+    assert b.vptq_assign_path(4096, 4096, 8, 65536) == "assign_tcgen05"
+    assert b.vptq_assign_path(4096, 4096, 8, 65536, b.FLAG_FORCE_GENERIC) == "assign_fp32"
+    assert b.vptq_assign_path(4100, 4096, 8, 65536) == "assign_fp32"        # v does not divide M
+    assert b.vptq_assign_path(4096, 4096, 16, 65536) == "assign_fp32"       # two of 16 K columns carry the norm
+    assert b.vptq_assign_path(4096, 4096, 8, 256) == "assign_fp32"          # small tables do not pay
+    assert b.vptq_assign_path(4096, 4096, 40, 256) == "invalid"
+    assert b.lib.vptq_assign_workspace_bytes(4096, 4096, 8, 256, 0) == 0
+    need = b.lib.vptq_assign_workspace_bytes(4096, 4096, 8, 65536, 0)
+    assert need >= 65536 * 32 + 4 * 512 * 4096
+    assert b.lib.vptq_assign(0x1000, 4096, 4096, 8, 0x1000, 65536, 0x1000, 0, None, 0, None) == b.E_WORKSPACE
+    assert b.lib.vptq_assign(None, 4096, 4096, 8, 0x1000, 65536, 0x1000, 0, None, 0, None) == b.E_NULL
+    assert b.lib.vptq_assign(0x1000, 4096, 4096, 8, 0x1000, 70000, 0x1000, 0, None, 0, None) == b.E_SHAPE
+

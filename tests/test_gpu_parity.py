@@ -270,8 +270,46 @@ def test_assign_is_bit_identical_to_the_oracle(b, M, N, v, k):
     rng = np.random.default_rng(1000 * v + k)
     W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
     Cb = rng.normal(0, 0.02, (k, v)).astype(np.float16)
-    idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda()).cpu().numpy()
+    idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda(), b.FLAG_FORCE_GENERIC).cpu().numpy()
     assert np.array_equal(idx, oracle.assign(W, v, Cb))
+
+
+@pytest.mark.parametrize("M,N,v,k,sigma", [
+    (136, 520, 8, 4096, 0.02),     # 35 steps of 256 vectors (the last one ragged), 32 centroid tiles
+    (132, 400, 6, 4096, 0.02),     # v = 6
+    (120, 500, 12, 2000, 0.02),    # v = 12, a padded last centroid tile
+    (64, 600, 8, 65536, 0.02),     # the largest table
+    (136, 520, 8, 4096, 30.0),     # large values: norms of about 7000
+    (72, 520, 1, 1024, 1.0),       # v = 1
+])
+def test_assign_on_tensor_cores_gives_the_same_indices(b, M, N, v, k, sigma):
+    rng = np.random.default_rng(77 * v + k)
+    W = rng.normal(0, sigma, (M, N)).astype(np.float16)
+    Cb = rng.normal(0, sigma, (k, v)).astype(np.float16)
+    assert b.vptq_assign_path(M, N, v, k) == "assign_tcgen05"
+    assert b.vptq_assign_path(M, N, v, k, b.FLAG_FORCE_GENERIC) == "assign_fp32"
+    Wd, Cd = torch.from_numpy(W).cuda(), torch.from_numpy(Cb).cuda()
+    idx = b.vptq_assign(Wd, v, Cd).cpu().numpy()
+    assert np.array_equal(idx, oracle.assign(W, v, Cb))
+
+
+def test_assign_on_tensor_cores_with_ties_everywhere(b):
+    # every centroid occurs 16 times, 128 apart: equal distances in different candidate groups; the lowest index
+    # wins, which only the full FP32 scan of the listed vectors can know
+    rng = np.random.default_rng(5)
+    M, N, v = 64, 600, 8
+    base = rng.normal(0, 0.02, (128, v)).astype(np.float16)
+    Cb = np.tile(base, (16, 1))
+    W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
+    assert b.vptq_assign_path(M, N, v, Cb.shape[0]) == "assign_tcgen05"
+    idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda()).cpu().numpy()
+    assert idx.max() < 128
+    assert np.array_equal(idx, oracle.assign(W, v, Cb))
+    # norms beyond the FP16 range: the filter is meaningless, every vector goes through the full scan
+    big = (rng.normal(0, 150.0, (2048, v))).astype(np.float16)
+    Wb = rng.normal(0, 150.0, (M, N)).astype(np.float16)
+    idx = b.vptq_assign(torch.from_numpy(Wb).cuda(), v, torch.from_numpy(big).cuda()).cpu().numpy()
+    assert np.array_equal(idx, oracle.assign(Wb, v, big))
 
 
 def test_assign_then_pack_and_dequant_reproduce_the_matrix(b):
