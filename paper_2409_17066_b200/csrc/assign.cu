@@ -25,20 +25,12 @@ constexpr int CHUNK_FLOATS = 4096;        // 16 KB of shared memory: CHUNK_FLOAT
 template <int VMAX>
 __global__ void __launch_bounds__(ASSIGN_THREADS)
 assign_kernel(const __half *__restrict__ W, int M, int N, int v, const __half *__restrict__ C, int k,
-              int *__restrict__ idx, long long n_vectors, const int *__restrict__ list, const int *__restrict__ count)
+              int *__restrict__ idx, long long n_vectors)
 {
     constexpr int CHUNK = CHUNK_FLOATS / VMAX;
     __shared__ __align__(16) float cb[CHUNK_FLOATS];
-    // all vectors, or (list != nullptr) the vectors list[0 .. *count) only
-    const long long slot = (long long)blockIdx.x * ASSIGN_THREADS + threadIdx.x;
-    long long g = slot;
-    bool valid = slot < n_vectors;
-    if (list != nullptr) {
-        const int cnt = __ldg(count);
-        if ((long long)blockIdx.x * ASSIGN_THREADS >= cnt) return;       // the whole block has nothing to do
-        valid = slot < cnt;
-        g = valid ? __ldg(list + slot) : 0;
-    }
+    const long long g = (long long)blockIdx.x * ASSIGN_THREADS + threadIdx.x;
+    const bool valid = g < n_vectors;
     const int r = valid ? (int)(g / N) : 0, n = valid ? (int)(g % N) : 0;
     const int vlen = min(v, M - r * v);              // components of this vector that exist
     float x[VMAX];
@@ -84,28 +76,102 @@ assign_kernel(const __half *__restrict__ W, int M, int N, int v, const __half *_
     if (valid) idx[g] = best;
 }
 
+// ---- the same decision for a short list of vectors: one warp per vector, its lanes share out the centroids ----
+constexpr int LISTED_WARPS = 16;
+
+template <int VMAX>
+__global__ void __launch_bounds__(LISTED_WARPS * 32)
+assign_listed_kernel(const __half *__restrict__ W, int M, int N, int v, const __half *__restrict__ C, int k,
+                     int *__restrict__ idx, const int *__restrict__ list, const int *__restrict__ count)
+{
+    constexpr int CHUNK = CHUNK_FLOATS / VMAX;
+    __shared__ __align__(16) float cb[CHUNK_FLOATS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cnt = __ldg(count);
+    for (long long first = (long long)blockIdx.x * LISTED_WARPS; first < cnt; first += (long long)gridDim.x * LISTED_WARPS) {
+        const bool valid = first + warp < cnt;
+        const long long g = valid ? __ldg(list + first + warp) : 0;
+        const int r = (int)(g / N), n = (int)(g % N);
+        const int vlen = min(v, M - r * v);
+        float x[VMAX];
+#pragma unroll
+        for (int j = 0; j < VMAX; j++)
+            x[j] = (valid && j < vlen) ? __half2float(__ldg(W + (long long)(r * v + j) * N + n)) : 0.f;
+        float best_d = __int_as_float(0x7f800000);
+        int best = 0x7fffffff;                         // no finite distance seen yet
+        for (int c0 = 0; c0 < k; c0 += CHUNK) {
+            const int cn = min(CHUNK, k - c0);
+            __syncthreads();
+            // component-major in shared memory: the lanes of a warp read consecutive centroids, consecutive banks
+            for (int e = threadIdx.x; e < cn * VMAX; e += LISTED_WARPS * 32) {
+                const int i = e / VMAX, j = e % VMAX;
+                cb[j * CHUNK + i] = j < v ? __half2float(__ldg(C + (long long)(c0 + i) * v + j)) : 0.f;
+            }
+            __syncthreads();
+            if (!valid) continue;
+            // (ascending within a lane: the first of equal distances stays)
+            if (vlen == v) {
+#pragma unroll 2
+                for (int i = lane; i < cn; i += 32) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int j = 0; j < VMAX; j++) {
+                        const float t = __fsub_rn(x[j], cb[j * CHUNK + i]);
+                        d = __fmaf_rn(t, t, d);
+                    }
+                    if (d < best_d) { best_d = d; best = c0 + i; }
+                }
+            } else {
+                for (int i = lane; i < cn; i += 32) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int j = 0; j < VMAX; j++) {
+                        const float t = j < vlen ? __fsub_rn(x[j], cb[j * CHUNK + i]) : 0.f;
+                        d = __fmaf_rn(t, t, d);
+                    }
+                    if (d < best_d) { best_d = d; best = c0 + i; }
+                }
+            }
+        }
+        // across the lanes: the smallest distance, and of equal distances the lowest index
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float od = __shfl_xor_sync(0xffffffffu, best_d, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, best, o);
+            if (od < best_d || (od == best_d && oi < best)) { best_d = od; best = oi; }
+        }
+        if (valid && lane == 0) idx[g] = best == 0x7fffffff ? 0 : best;
+    }
+}
+
 }  // namespace
 
 bool assign_supported(int v, int k) { return v >= 1 && v <= 32 && k >= 1 && k <= 65536; }
 
-cudaError_t launch_assign_listed(const __half *W, int M, int N, int v, const __half *C, int k, int *idx,
-                                 const int *list, const int *count, long long n_vectors, cudaStream_t st)
+cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st)
 {
+    const long long n_vectors = (long long)ceil_div(M, v) * N;
     if (n_vectors == 0) return cudaSuccess;
-    // (with a list the grid is sized for the worst case, every vector listed; blocks beyond the count return at once)
     const long long blocks = (n_vectors + ASSIGN_THREADS - 1) / ASSIGN_THREADS;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
     const dim3 grid((unsigned)blocks);
-    if (v <= 4) assign_kernel<4><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
-    else if (v <= 8) assign_kernel<8><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
-    else if (v <= 16) assign_kernel<16><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
-    else assign_kernel<32><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors, list, count);
+    if (v <= 4) assign_kernel<4><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
+    else if (v <= 8) assign_kernel<8><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
+    else if (v <= 16) assign_kernel<16><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
+    else assign_kernel<32><<<grid, ASSIGN_THREADS, 0, st>>>(W, M, N, v, C, k, idx, n_vectors);
     return cudaGetLastError();
 }
 
-cudaError_t launch_assign(const __half *W, int M, int N, int v, const __half *C, int k, int *idx, cudaStream_t st)
+cudaError_t launch_assign_listed(const __half *W, int M, int N, int v, const __half *C, int k, int *idx,
+                                 const int *list, const int *count, int sm_count, cudaStream_t st)
 {
-    return launch_assign_listed(W, M, N, v, C, k, idx, nullptr, nullptr, (long long)ceil_div(M, v) * N, st);
+    // a fixed grid (the count is on the device): every block takes 16 listed vectors at a time
+    const dim3 grid((unsigned)(4 * sm_count));
+    if (v <= 4) assign_listed_kernel<4><<<grid, LISTED_WARPS * 32, 0, st>>>(W, M, N, v, C, k, idx, list, count);
+    else if (v <= 8) assign_listed_kernel<8><<<grid, LISTED_WARPS * 32, 0, st>>>(W, M, N, v, C, k, idx, list, count);
+    else if (v <= 16) assign_listed_kernel<16><<<grid, LISTED_WARPS * 32, 0, st>>>(W, M, N, v, C, k, idx, list, count);
+    else assign_listed_kernel<32><<<grid, LISTED_WARPS * 32, 0, st>>>(W, M, N, v, C, k, idx, list, count);
+    return cudaGetLastError();
 }
 
 }  // namespace vptq

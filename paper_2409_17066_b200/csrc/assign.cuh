@@ -4,9 +4,9 @@
 
 namespace vptq {
 
-// the plain FP32 kernel for the vectors list[0 .. *count) only (both on the device)
+// the FP32 definition for the vectors list[0 .. *count) only (both on the device): one warp per vector
 cudaError_t launch_assign_listed(const __half *W, int M, int N, int v, const __half *C, int k, int *idx,
-                                 const int *list, const int *count, long long n_vectors, cudaStream_t st);
+                                 const int *list, const int *count, int sm_count, cudaStream_t st);
 
 // tensor-core filter + FP32 decision: same indices as the plain kernel
 bool assign_tcgen05_supported(int M, int N, int v, int k);

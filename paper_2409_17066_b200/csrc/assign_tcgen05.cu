@@ -2,14 +2,15 @@
 //
 // The squared distance is ||c||^2 - 2 x.c + ||x||^2, and the first two terms are a contraction over the
 // vector's components: D[vector][centroid] = A * B^T with
-//   A row (a vector):   x_0 .. x_{v-1}, 0 .., 1, 1          (16 FP16 values, K = 16)
-//   B row (a centroid): -2c_0 .. -2c_{v-1}, 0 .., hi, lo     hi + lo = ||c||^2 split into two FP16 values
+//   A row (a vector):   x_0 .. x_{v-1}, 0 .., 1, 2^-11            (16 FP16 values, K = 16)
+//   B row (a centroid): -2c_0 .. -2c_{v-1}, 0 .., hi, 2^11 lo     hi + lo = ||c||^2 split into two FP16 values
+//                                                                (lo scaled so that it does not underflow)
 // One tcgen05.mma (M = 128 vectors, N = 128 centroids, K = 16) gives 16 K approximate distances.  They
 // only FILTER: per vector the kernel keeps the smallest and the second smallest minimum over groups of
 // 32 centroids and the group of the smallest.  Then the 32 centroids of that group are evaluated with
 // the arithmetic that defines the result (FP32 fma chain, lowest index wins: the same code as the plain
 // kernel), and a vector whose two group minima are closer than a bound on the filter's error is put on
-// a list; the plain kernel scans all centroids for the vectors on the list.  The indices are therefore
+// a list; a second kernel scans all centroids for the vectors on the list (one warp per vector).  The indices are therefore
 // those of the FP32 definition, bit for bit, whatever the tensor core's summation order.
 //   bound: |filter - (definition - ||x||^2)| <= 2^-18 (||x||^2 + max ||c||^2) (FP16 split of the norm,
 //   FP32 accumulation of 10 products, rounding of the fma chain); the margin tested is 2^-14 of it.
@@ -185,7 +186,7 @@ assign_prepare_kernel(const __half *__restrict__ C, int k, int v, uint8_t *__res
     }
     const __half hi = __float2half_rn(norm);
     row[14] = hi;
-    row[15] = __float2half_rn(norm - __half2float(hi));
+    row[15] = __float2half_rn((norm - __half2float(hi)) * 2048.f);     // the A row multiplies it by 2^-11
     uint8_t *tile = Bimg + (long long)(i / KT) * TILE_BYTES;
     const uint4 *src = reinterpret_cast<const uint4 *>(row);
     *reinterpret_cast<uint4 *>(tile + image_offset(i % KT, 0)) = src[0];
@@ -298,7 +299,7 @@ assign_scan_kernel(ScanParams P)
 #pragma unroll
                 for (int j = 0; j < 14; j++) rowv[j] = __float2half_rn(j < VMAX ? x[j < VMAX ? j : 0] : 0.f);   // exact: x came from FP16
                 rowv[14] = __float2half_rn(1.f);         // times hi
-                rowv[15] = __float2half_rn(1.f);         // times lo
+                rowv[15] = __float2half_rn(1.f / 2048.f);    // times 2^11 lo
                 const uint4 *src = reinterpret_cast<const uint4 *>(rowv);
                 uint8_t *tile = sA + a * TILE_BYTES;
                 *reinterpret_cast<uint4 *>(tile + image_offset(row, 0)) = src[0];
@@ -444,7 +445,7 @@ cudaError_t launch_assign_tcgen05(const __half *W, int M, int N, int v, const __
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     // the vectors whose candidate group was not clearly the only one: all centroids, FP32
-    return launch_assign_listed(W, M, N, v, C, k, idx, P.list, P.count, n_vectors, st);
+    return launch_assign_listed(W, M, N, v, C, k, idx, P.list, P.count, scan_sm_count(), st);
 }
 
 }  // namespace vptq
