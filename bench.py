@@ -497,32 +497,50 @@ def extra_configs(vb, synth, peaks):
 
 def encoder_assign(vb, synth):
     """The quantizer's assignment step (Eq. 2) on a matrix of the size of config 1's layer: every one of the
-    2.1 M vectors against all 65536 centroids.  Bound by the FP32 pipes: one subtract and one fma per
-    component and centroid; peak = SMs x 128 FP32 lanes x SM clock instructions per second."""
+    2.1 M vectors against all 65536 centroids, by the tensor-core filter + FP32 decision (the default) and by
+    the plain FP32 kernel (same indices).  The FP32 kernel is bound by the FP32 pipes: one subtract and one
+    fma per component and centroid; peak = SMs x 128 FP32 lanes x SM clock instructions per second."""
     import numpy as np
     import torch
     M, N, v, k = 4096, 4096, 8, 65536
     rng = np.random.default_rng(synth.BASE_SEED + 77)
     W = torch.from_numpy(rng.normal(0, 0.02, (M, N)).astype(np.float16)).cuda()
     Cb = torch.from_numpy(rng.normal(0, 0.02, (k, v)).astype(np.float16)).cuda()
-    vb.vptq_assign(W, v, Cb)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(3):
-        vb.vptq_assign(W, v, Cb)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 3
-    props = torch.cuda.get_device_properties(0)
-    pairs = (M // v) * N * k * v                                   # (subtract, fma) pairs
-    peak = props.multi_processor_count * 128 * 1.965e9             # FP32 instructions per second at the maximum SM clock
-    return {"encoder_assign_4096x4096_v8_k65536": {
-        "ms": ms, "G_distances_per_s": (M // v) * N * k / (ms * 1e-3) / 1e9,
-        "roofline": {"bound": "alu", "achieved": 2 * pairs / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
-                     "unit": "T FP32 instructions/s (one subtract and one fma per component)",
-                     "frac": 2 * pairs / (ms * 1e-3) / peak,
-                     "peak_source": "148 SMs x 128 FP32 lanes x 1.965 GHz (unit counts and maximum clock)"}}}
+    idx = torch.empty((M // v, N), dtype=torch.int32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    out = {}
+    for flags in (0, vb.FLAG_FORCE_GENERIC):
+        need = vb.lib.vptq_assign_workspace_bytes(M, N, v, k, flags)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+
+        def call():
+            rc = vb.lib.vptq_assign(W.data_ptr(), M, N, v, Cb.data_ptr(), k, idx.data_ptr(), flags,
+                                    ws.data_ptr() if need else None, need, st)
+            assert rc == vb.OK, rc
+        call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 3
+        path = vb.vptq_assign_path(M, N, v, k, flags)
+        r = {"ms": ms, "G_distances_per_s": (M // v) * N * k / (ms * 1e-3) / 1e9}
+        if flags == 0:
+            assert vb.vptq_workspace_status(ws) == vb.OK
+            r["vectors_sent_to_the_full_fp32_scan"] = int(ws[32:36].view(torch.int32).item()) / ((M // v) * N)
+        else:
+            props = torch.cuda.get_device_properties(0)
+            pairs = (M // v) * N * k * v                               # (subtract, fma) pairs
+            peak = props.multi_processor_count * 128 * 1.965e9         # FP32 instructions per second at the maximum SM clock
+            r["roofline"] = {"bound": "alu", "achieved": 2 * pairs / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
+                             "unit": "T FP32 instructions/s (one subtract and one fma per component)",
+                             "frac": 2 * pairs / (ms * 1e-3) / peak,
+                             "peak_source": "148 SMs x 128 FP32 lanes x 1.965 GHz (unit counts and maximum clock)"}
+        out[f"encoder_{path}_4096x4096_v8_k65536"] = r
+    return out
 
 
 def main():
