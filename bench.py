@@ -552,6 +552,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-fuse", action="store_true", help="one vptq_linear call per layer (no vptq_linear_fused)")
+    ap.add_argument("--encoder", action="store_true",
+                    help="only the quantizer's assignment step (Eq. 2) at full size (profiling case)")
     ap.add_argument("--cfg", type=int, default=WORKLOAD_CFG,
                     help="workload number (default: the headline workload); others are profiling cases")
     ap.add_argument("--layers", default="", help="comma-separated layer names to keep (profiling cases)")
@@ -559,6 +561,16 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.encoder:
+        import torch
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+        from paper_2409_17066_b200 import build as vbuild
+        from paper_2409_17066_b200 import synth
+        vbuild.build()
+        from paper_2409_17066_b200 import binding as vb
+        print(json.dumps(encoder_assign(vb, synth)))
+        return 0
     return run_ours(args)
 
 

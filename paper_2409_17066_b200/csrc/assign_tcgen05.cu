@@ -19,8 +19,9 @@
 // centroid tiles (4 KB, shared-memory image with the 32-byte swizzle applied by the preparation kernel)
 // with linear bulk copies into a ring; warp 1 issues the MMAs (two per centroid tile, fresh accumulators
 // in one of two TMEM buffers); warps 2-9 write the A tiles of a step, then drain the accumulators: a lane
-// owns one vector, reads 32 distances per tcgen05.ld and keeps its two running minima (35 instructions
-// per 32 distances: the epilogue, not the tensor core, bounds the kernel).
+// owns one vector, reads 32 distances per tcgen05.ld and keeps its two running minima (about 40 instructions
+// per 32 distances, nearly all of them min/compare/select on the ALU pipe: that pipe, not the tensor core,
+// bounds the kernel; the three-input min.f32 was tried and changes nothing).
 // Every mbarrier wait is bounded; a wait that gives up sets the status word of the workspace.
 #include "common.cuh"
 #include "assign.cuh"
