@@ -25,10 +25,13 @@
 // Every mbarrier wait is bounded; a wait that gives up sets the status word of the workspace.
 #include "common.cuh"
 #include "assign.cuh"
+#include "tcgen05_ptx.cuh"
 
 namespace vptq {
 
 namespace {
+
+using namespace tc;
 
 constexpr int KT = 128;                       // centroids per tile (N of the MMA)
 constexpr int ROW_BYTES = 32;                 // K = 16 FP16 values
@@ -38,7 +41,6 @@ constexpr int EPI_WARPS = 8;
 constexpr int SCAN_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int STEP_VECTORS = 256;             // two A tiles
 constexpr int GROUP = 32;                     // centroids per candidate group (one tcgen05.ld)
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
 constexpr float PAD_NORM = 60000.f;           // norm of the padding rows of the last centroid tile: never the minimum
 constexpr float MARGIN = 1.0f / 16384.0f;     // 2^-14
 
@@ -56,62 +58,8 @@ struct ScanParams {
     int k_tiles;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred P1;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
-                 "selp.b32 %0, 1, 0, P1;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when it was abandoned (time limit here, or the abort flag raised elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
-{
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    unsigned spins = 0;
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if ((++spins & 255u) == 0) {
-            if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicExch(status, VPTQ_E_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 // K-major operand with 32-byte rows and the 32-byte swizzle: 8-row groups of 256 bytes
-__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)1 << 16;                              // leading-dimension offset: unused for one swizzle row
-    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;         // stride between 8-row groups
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)6 << 61;                              // 32-byte swizzle
-    return d;
-}
+__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr) { return make_smem_desc(saddr, 16, 8 * ROW_BYTES, LAYOUT_SW32); }
 // kind::f16: FP16 x FP16 -> FP32, both operands K-major, M = 128, N = 128
 constexpr uint32_t SCAN_IDESC = (1u << 4) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 __device__ __forceinline__ void umma_fresh(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc)
@@ -120,12 +68,6 @@ __device__ __forceinline__ void umma_fresh(uint32_t d_tmem, uint64_t a_desc, uin
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(SCAN_IDESC) : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // 32 consecutive accumulator columns of this lane's row: the load is only issued here ...
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -206,7 +148,7 @@ assign_scan_kernel(ScanParams P)
     __shared__ int abort_word;
     volatile int *abort_flag = &abort_word;
 
-    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t bar0 = smem_addr(bars);
     auto bar_fullB = [&](int s) { return bar0 + 8u * s; };
     auto bar_emptyB = [&](int s) { return bar0 + 8u * (B_STAGES + s); };
     auto bar_accFull = [&](int b) { return bar0 + 8u * (2 * B_STAGES + b); };
@@ -222,7 +164,7 @@ assign_scan_kernel(ScanParams P)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_slot)), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -242,7 +184,7 @@ assign_scan_kernel(ScanParams P)
                     const int s = (int)(it % B_STAGES);
                     if (!(ok = mbar_wait(bar_emptyB(s), (uint32_t)((it / B_STAGES) & 1) ^ 1u, abort_flag, P.status))) break;
                     mbar_expect_tx(bar_fullB(s), TILE_BYTES);
-                    bulk_load(smem_u32(sB) + s * TILE_BYTES, P.Bimg + (long long)kt * TILE_BYTES, TILE_BYTES, bar_fullB(s));
+                    bulk_load(smem_addr(sB) + s * TILE_BYTES, P.Bimg + (long long)kt * TILE_BYTES, TILE_BYTES, bar_fullB(s));
                 }
             if (!ok) {
                 // abandoned: give copies still in flight a bounded time to land before the CTA exits
@@ -257,8 +199,8 @@ assign_scan_kernel(ScanParams P)
     } else if (warp == 1) {
         // ================= MMA issue =================
         if (lane == 0) {
-            const uint64_t adesc0 = operand_desc(smem_u32(sA));
-            const uint64_t bdesc0 = operand_desc(smem_u32(sB));
+            const uint64_t adesc0 = operand_desc(smem_addr(sA));
+            const uint64_t bdesc0 = operand_desc(smem_addr(sB));
             long long it = 0, step_no = 0;
             for (long long step = blockIdx.x; step < n_steps && ok; step += gridDim.x, step_no++) {
                 if (!(ok = mbar_wait(bar_aFull, (uint32_t)(step_no & 1), abort_flag, P.status))) break;

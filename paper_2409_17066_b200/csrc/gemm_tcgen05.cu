@@ -44,10 +44,13 @@
 
 #include "common.cuh"
 #include "gemm.cuh"
+#include "tcgen05_ptx.cuh"
 
 namespace vptq {
 
 namespace {
+
+using namespace tc;
 
 constexpr int TILE_M = 128;
 constexpr int TILE_K = 32;
@@ -69,7 +72,6 @@ constexpr int GEMM_THREADS = 32 * (2 + PRODUCER_WARPS + EPI_WARPS);   // 640
 constexpr int A_SBO = 2048;   // bytes between consecutive 8-column groups of the A stage
 constexpr int A_LBO = 1024;   // bytes between the two 64-row blocks of the A stage
 constexpr int B_SBO = 512;    // bytes between consecutive 8-token groups of the B stage (8 x 64 B)
-constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;
 
 constexpr int WS_STATUS_BYTES = 256;
 constexpr int FLAG_ORDER_MIN_SHARE = 24;
@@ -92,52 +94,6 @@ struct GemmParams {
 };
 
 // ---- PTX wrappers ----------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred P1;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
-                 "selp.b32 %0, 1, 0, P1;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Wait until the preceding kernel of the stream (the pre-pass) has completed and its writes are visible.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-// Bounded wait.  Returns false when the wait was abandoned (timeout here or abort raised elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
-{
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    unsigned spins = 0;
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if ((++spins & 255u) == 0) {
-            if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                grid_dependency_wait();                  // the pre-pass clears the status word
-                atomicExch(status, VPTQ_E_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-
 // Bounded wait until *flag >= target (set by another CTA of this grid; all CTAs of the grid are resident).
 __device__ __forceinline__ bool flag_wait(const int *flag, int target, volatile int *abort_flag, int *status)
 {
@@ -159,25 +115,6 @@ __device__ __forceinline__ bool flag_wait(const int *flag, int target, volatile 
         __nanosleep(64);
     }
 }
-
-// linear bulk copy global -> shared memory (16-byte aligned addresses, size a multiple of 16)
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);            // start address, 16-byte units
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;   // leading-dimension byte offset
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;   // stride-dimension byte offset
-    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
-    d |= (uint64_t)layout << 61;                         // swizzle mode
-    return d;
-}
-constexpr uint32_t LAYOUT_SW128 = 2, LAYOUT_SW64 = 4;
 
 // kind::f16, FP16 x FP16 -> FP32, A MN-major, B K-major, M = 128, N = 256
 constexpr uint32_t IDESC = (1u << 4) | (0u << 7) | (0u << 10) | (1u << 15) | (0u << 16) |
@@ -202,14 +139,6 @@ __device__ __forceinline__ void umma_kblock(uint32_t d_tmem, uint64_t ad, uint64
     umma_f16(d_tmem, ad1, bd1, 1u);
     if (two_halves) umma_f16(d_tmem + MMA_N, ad1, bd1 + bh, 1u);
 }
-// Arrive on the barrier once all MMAs issued so far have completed.
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
