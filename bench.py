@@ -311,7 +311,7 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     value = whole_job_gbps(step_bytes, world, ms_step)
 
-    # per-launch durations of the dominant kernel (all seven calls run the same kernel family)
+    # per-launch durations of the dominant kernel (all calls of the step run the same kernel family)
     call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call if pc is not None]
     n_ev = len(call_ms)
     layer_ms = [statistics.mean(call_ms[i][ci] for i in range(n_ev)) for ci in range(len(calls))]
