@@ -56,7 +56,8 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
 
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
                    "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel",
-                   "fused_decode_l2_fma": "decode_l2_fma_kernel"}
+                   "fused_decode_l2_fma": "decode_l2_fma_kernel", "fused_decode_smem_fma": "decode_smem_fma_kernel",
+                   "fused_decode_gl_fma": "decode_gl_fma_kernel"}
 # projections of a decoder layer that read the same activations
 FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
 
@@ -254,7 +255,7 @@ def run_ours(args):
     while li < len(layers):
         group = next((g for g in FUSE_GROUPS if tuple(names[li:li + len(g)]) == g), None)
         if group is not None and not args.no_fuse and \
-                vb.vptq_linear_fused_path([layers[j][0].desc for j in range(li, li + len(group))], B) == "fused_decode_l2_fma":
+                vb.vptq_linear_fused_path([layers[j][0].desc for j in range(li, li + len(group))], B).startswith("fused_"):
             idx = list(range(li, li + len(group)))
             calls.append((idx, [vb.FusedLayers([layers[j][c] for j in idx]) for c in range(copies)]))
         else:

@@ -8,6 +8,8 @@ namespace vptq {
 bool smem_fma_supported(const LayerView &L, int B);
 int smem_fma_launches(const LayerView &L, int B);
 cudaError_t launch_decode_smem_fma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
+bool smem_fma_fused_supported(const LayerView *Ls, int n, int B);
+cudaError_t launch_decode_smem_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st);
 
 // codebooks in shared memory, ldmatrix gathers + mma.sync (per-output-row scale, all-outlier layers)
 bool smem_mma_supported(const LayerView &L, int B);
@@ -27,5 +29,7 @@ cudaError_t launch_decode_l2_fma_fused(const LayerView *Ls, int n, const void *x
 bool gl_fma_supported(const LayerView &L, int B);
 int gl_fma_launches(const LayerView &L, int B);
 cudaError_t launch_decode_gl_fma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
+bool gl_fma_fused_supported(const LayerView *Ls, int n, int B);
+cudaError_t launch_decode_gl_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st);
 
 }  // namespace vptq

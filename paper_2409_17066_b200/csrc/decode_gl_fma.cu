@@ -13,6 +13,7 @@
 // sums meet in shared memory; the epilogue adds the bias term and converts (a7).  No scratch.
 #include "common.cuh"
 #include "decode.cuh"
+#include "fused_split.cuh"
 
 namespace vptq {
 
@@ -23,9 +24,11 @@ constexpr int PART_BUDGET = 32 * 1024;      // bytes of per-row partial sums per
 constexpr int GL_WARPS = 16;
 
 struct GlFmaParams {
-    LayerView L;
+    LayerView L[MAX_FUSED];        // a fused launch: layer l is the work of CTAs [cta_begin[l], cta_begin[l + 1])
+    void *out[MAX_FUSED];
+    int cta_begin[MAX_FUSED + 1];
+    int n_layers;
     const void *x;
-    void *out;
     int B;                 // tokens in this launch (<= TB)
     int slab_cols;         // main columns per slab (multiple of 256)
     int n_slabs;
@@ -133,13 +136,20 @@ __device__ __forceinline__ void load_row_words(const __half *__restrict__ tab, l
     }
 }
 
-template <int TB, int VV, bool RES>
+template <int TB, int VV, bool RES, bool FUSED>
 __global__ void __launch_bounds__(GL_WARPS * 32, 1)
-decode_gl_fma_kernel(GlFmaParams P)
+decode_gl_fma_kernel(const __grid_constant__ GlFmaParams P)
 {
     constexpr int WARPS = GL_WARPS, THREADS = WARPS * 32, VW = VV / 2;
     extern __shared__ __align__(16) uint8_t smem[];
-    const LayerView &L = P.L;
+    // the layer this CTA works on, and its place among that layer's CTAs
+    int li = 0;
+    if (FUSED)
+        while (li + 1 < P.n_layers && (int)blockIdx.x >= P.cta_begin[li + 1]) li++;
+    const LayerView &L = P.L[FUSED ? li : 0];
+    void *const out = P.out[FUSED ? li : 0];
+    const int bid = FUSED ? (int)blockIdx.x - P.cta_begin[li] : (int)blockIdx.x;
+    const int gdim = FUSED ? P.cta_begin[li + 1] - P.cta_begin[li] : (int)gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     __half *xs_out = reinterpret_cast<__half *>(smem);                                       // [TB][n_out_pad]
@@ -149,8 +159,8 @@ decode_gl_fma_kernel(GlFmaParams P)
     float *red = bterm + 8;                                                                  // [WARPS][8]
 
     // vector rows of this CTA, and the output rows they cover
-    const int r0 = (int)((long long)L.R * blockIdx.x / gridDim.x);
-    const int r1 = (int)((long long)L.R * (blockIdx.x + 1) / gridDim.x);
+    const int r0 = (int)((long long)L.R * bid / gdim);
+    const int r1 = (int)((long long)L.R * (bid + 1) / gdim);
     const int m_lo = r0 * L.v;
     const int m_hi = min(L.M, r1 * L.v);
     const int vw = L.v >> 1;
@@ -394,7 +404,7 @@ decode_gl_fma_kernel(GlFmaParams P)
         const int m = m_lo + ml;
         const int rr = m / L.v, jj = m - rr * L.v;
         const float y = part[((rr - r0) * TB + t) * 16 + jj] + bterm[t];
-        store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
+        store_out(out, (long long)t * L.M + m, y, L.out_dtype);
     }
 }
 
@@ -402,6 +412,7 @@ struct GlFmaPlan {
     int slab_cols, n_slabs, grid, part_floats, n_out_pad;
     size_t smem;
     bool ok;
+    int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
 int gl_num_sms()
@@ -437,20 +448,22 @@ GlFmaPlan plan_gl_fma(const LayerView &L, int TB)
     return p;
 }
 
+template <int TB, int VV, bool RES, bool FUSED>
+cudaError_t launch_kernel(const GlFmaParams &P, const GlFmaPlan &pl, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(decode_gl_fma_kernel<TB, VV, RES, FUSED>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    decode_gl_fma_kernel<TB, VV, RES, FUSED><<<pl.grid, GL_WARPS * 32, pl.smem, st>>>(P);
+    return cudaGetLastError();
+}
+
 template <int TB, int VV>
 cudaError_t launch_one(const GlFmaParams &P, const GlFmaPlan &pl, bool res, cudaStream_t st)
 {
-    cudaError_t e;
-    if (res) {
-        e = cudaFuncSetAttribute(decode_gl_fma_kernel<TB, VV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-        if (e != cudaSuccess) return e;
-        decode_gl_fma_kernel<TB, VV, true><<<pl.grid, GL_WARPS * 32, pl.smem, st>>>(P);
-    } else {
-        e = cudaFuncSetAttribute(decode_gl_fma_kernel<TB, VV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-        if (e != cudaSuccess) return e;
-        decode_gl_fma_kernel<TB, VV, false><<<pl.grid, GL_WARPS * 32, pl.smem, st>>>(P);
-    }
-    return cudaGetLastError();
+    const bool fused = P.n_layers > 1;
+    if (res) return fused ? launch_kernel<TB, VV, true, true>(P, pl, st) : launch_kernel<TB, VV, true, false>(P, pl, st);
+    return fused ? launch_kernel<TB, VV, false, true>(P, pl, st) : launch_kernel<TB, VV, false, false>(P, pl, st);
 }
 
 template <int TB>
@@ -459,6 +472,26 @@ cudaError_t launch_vv(const GlFmaParams &P, const GlFmaPlan &pl, int v, bool res
     if (v <= 8) return launch_one<TB, 8>(P, pl, res, st);
     if (v <= 12) return launch_one<TB, 12>(P, pl, res, st);
     return launch_one<TB, 16>(P, pl, res, st);
+}
+
+// several layers of the same format (apart from M) in one grid
+bool plan_gl_fma_fused(const LayerView *Ls, int n, int TB, GlFmaPlan *out)
+{
+    if (n < 2 || n > MAX_FUSED) return false;
+    for (int l = 1; l < n; l++)
+        if (!same_geometry(Ls[0], Ls[l])) return false;
+    GlFmaPlan p = plan_gl_fma(Ls[0], TB);
+    if (!p.ok) return false;
+    int R[MAX_FUSED], rows_cta = 0;
+    for (int l = 0; l < n; l++) R[l] = Ls[l].R;
+    if (!split_ctas(R, n, gl_num_sms(), p.cta_begin, &rows_cta)) return false;
+    p.grid = gl_num_sms();
+    p.smem -= (size_t)p.part_floats * 4;
+    p.part_floats = rows_cta * TB * 16;
+    p.smem += (size_t)p.part_floats * 4;
+    if ((long long)p.part_floats * 4 > PART_BUDGET || p.smem > 200 * 1024) return false;
+    *out = p;
+    return true;
 }
 
 }  // namespace
@@ -487,15 +520,53 @@ cudaError_t launch_decode_gl_fma(const LayerView &L, const void *x, int B, void 
     const bool res = L.k2 > 0;
     for (int t0 = 0; t0 < B; t0 += TB) {
         GlFmaParams P;
-        P.L = L; P.B = (B - t0 < TB) ? (B - t0) : TB;
+        memset(&P, 0, sizeof(P));
+        P.L[0] = L; P.n_layers = 1; P.cta_begin[1] = pl.grid;
+        P.B = (B - t0 < TB) ? (B - t0) : TB;
         P.x = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * xe;
-        P.out = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
+        P.out[0] = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
         P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs;
         P.n_out_pad = pl.n_out_pad; P.part_floats = pl.part_floats;
         cudaError_t e;
         if (TB == 4) e = launch_vv<4>(P, pl, L.v, res, st);
         else if (TB == 2) e = launch_vv<2>(P, pl, L.v, res, st);
         else e = launch_vv<1>(P, pl, L.v, res, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+bool gl_fma_fused_supported(const LayerView *Ls, int n, int B)
+{
+    for (int l = 0; l < n; l++)
+        if (!gl_fma_supported(Ls[l], B)) return false;
+    GlFmaPlan pl;
+    return plan_gl_fma_fused(Ls, n, gl_token_group(B), &pl);
+}
+
+cudaError_t launch_decode_gl_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st)
+{
+    const int TB = gl_token_group(B);
+    GlFmaPlan pl;
+    if (!plan_gl_fma_fused(Ls, n, TB, &pl)) return cudaErrorInvalidValue;
+    const bool res = Ls[0].k2 > 0;
+    for (int t0 = 0; t0 < B; t0 += TB) {
+        GlFmaParams P;
+        memset(&P, 0, sizeof(P));
+        for (int l = 0; l < n; l++) {
+            P.L[l] = Ls[l];
+            P.out[l] = reinterpret_cast<uint8_t *>(outs[l]) + (size_t)t0 * Ls[l].M * (Ls[l].out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
+        }
+        for (int l = 0; l <= n; l++) P.cta_begin[l] = pl.cta_begin[l];
+        P.n_layers = n;
+        P.B = (B - t0 < TB) ? (B - t0) : TB;
+        P.x = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * Ls[0].N * 2;
+        P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs;
+        P.n_out_pad = pl.n_out_pad; P.part_floats = pl.part_floats;
+        cudaError_t e;
+        if (TB == 4) e = launch_vv<4>(P, pl, Ls[0].v, res, st);
+        else if (TB == 2) e = launch_vv<2>(P, pl, Ls[0].v, res, st);
+        else e = launch_vv<1>(P, pl, Ls[0].v, res, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

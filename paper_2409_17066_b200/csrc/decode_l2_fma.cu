@@ -27,6 +27,7 @@
 // a prologue and a ragged tail each.
 #include "common.cuh"
 #include "decode.cuh"
+#include "fused_split.cuh"
 
 namespace vptq {
 
@@ -36,7 +37,6 @@ constexpr int RB_ROWS = 16;                 // vector rows per completion counte
 constexpr int XS_BUDGET = 64 * 1024;        // bytes of staged activations per CTA
 constexpr int PART_BUDGET = 32 * 1024;      // bytes of per-row partial sums per CTA (OWNER mode)
 constexpr int WARPS_TB4 = 16;               // 4 tokens per launch need 128 registers per thread
-constexpr int MAX_FUSED = 4;                // layers of one fused launch
 
 struct L2FmaParams {
     LayerView L[MAX_FUSED];
@@ -448,30 +448,10 @@ bool plan_l2_fused(const LayerView *Ls, int n, int TB, L2Plan *out)
         if (Ls[l].N != Ls[0].N || Ls[l].x_bf16 != Ls[0].x_bf16 || Ls[l].k2 != Ls[0].k2) return false;
     L2Plan p = plan_l2(Ls[0], TB);          // slab geometry, warps, residual table: functions of N, k2, TB
     const int G = l2_num_sms();
+    int R[MAX_FUSED], rows_cta = 0;
     long long rows = 0;
-    for (int l = 0; l < n; l++) rows += Ls[l].R;
-    if (rows < G) return false;
-    int ctas[MAX_FUSED], used = 0;
-    for (int l = 0; l < n; l++) {
-        ctas[l] = (int)((long long)G * Ls[l].R / rows);
-        if (ctas[l] < 1) ctas[l] = 1;
-        used += ctas[l];
-    }
-    if (used > G) return false;
-    for (; used < G; used++) {
-        int best = 0;
-        for (int l = 1; l < n; l++)
-            if ((long long)ceil_div(Ls[l].R, ctas[l]) * ctas[best] > (long long)ceil_div(Ls[best].R, ctas[best]) * ctas[l] ||
-                ceil_div(Ls[l].R, ctas[l]) > ceil_div(Ls[best].R, ctas[best]))
-                best = l;
-        ctas[best]++;
-    }
-    int rows_cta = 0;
-    p.cta_begin[0] = 0;
-    for (int l = 0; l < n; l++) {
-        rows_cta = rows_cta > ceil_div(Ls[l].R, ctas[l]) ? rows_cta : ceil_div(Ls[l].R, ctas[l]);
-        p.cta_begin[l + 1] = p.cta_begin[l] + ctas[l];
-    }
+    for (int l = 0; l < n; l++) { R[l] = Ls[l].R; rows += Ls[l].R; }
+    if (!split_ctas(R, n, G, p.cta_begin, &rows_cta)) return false;
     const double eff_cta = (double)rows / ((double)G * rows_cta);
     const long long t_cta = (long long)rows_cta * (p.slab_cols / 256);
     const double eff_warp = (double)t_cta / ((double)p.warps * (double)((t_cta + p.warps - 1) / p.warps));

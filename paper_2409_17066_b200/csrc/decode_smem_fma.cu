@@ -19,6 +19,7 @@
 // sums meet in shared memory; the epilogue adds the bias term and converts (a7).  No scratch.
 #include "common.cuh"
 #include "decode.cuh"
+#include "fused_split.cuh"
 
 namespace vptq {
 
@@ -29,9 +30,11 @@ constexpr int PART_BUDGET = 16 * 1024;      // bytes of per-row partial sums per
 constexpr int SMEM_FMA_MAX_B = 4;
 
 struct SmemFmaParams {
-    LayerView L;
+    LayerView L[MAX_FUSED];        // a fused launch: layer l is the work of CTAs [cta_begin[l], cta_begin[l + 1])
+    void *out[MAX_FUSED];
+    int cta_begin[MAX_FUSED + 1];
+    int n_layers;
     const void *x;
-    void *out;
     int B;                 // tokens in this launch (<= TB)
     int slab_cols;         // main columns per slab (multiple of 256)
     int n_slabs;
@@ -119,13 +122,20 @@ __device__ __forceinline__ uint4 load_centroid_row(const __half *__restrict__ ta
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int TB, int VV, bool RES, int WARPS>
+template <int TB, int VV, bool RES, int WARPS, bool FUSED>
 __global__ void __launch_bounds__(WARPS * 32, 1)
-decode_smem_fma_kernel(SmemFmaParams P)
+decode_smem_fma_kernel(const __grid_constant__ SmemFmaParams P)
 {
     constexpr int THREADS = WARPS * 32;
     extern __shared__ __align__(16) uint8_t smem[];
-    const LayerView &L = P.L;
+    // the layer this CTA works on, and its place among that layer's CTAs
+    int li = 0;
+    if (FUSED)
+        while (li + 1 < P.n_layers && (int)blockIdx.x >= P.cta_begin[li + 1]) li++;
+    const LayerView &L = P.L[FUSED ? li : 0];
+    void *const out = P.out[FUSED ? li : 0];
+    const int bid = FUSED ? (int)blockIdx.x - P.cta_begin[li] : (int)blockIdx.x;
+    const int gdim = FUSED ? P.cta_begin[li + 1] - P.cta_begin[li] : (int)gridDim.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     uint4 *cb1 = reinterpret_cast<uint4 *>(smem);                                            // [k1]
@@ -137,8 +147,8 @@ decode_smem_fma_kernel(SmemFmaParams P)
     float *red = bterm + 8;                                                                  // [WARPS][8]
 
     // vector rows of this CTA, and the output rows they cover
-    const int r0 = (int)((long long)L.R * blockIdx.x / gridDim.x);
-    const int r1 = (int)((long long)L.R * (blockIdx.x + 1) / gridDim.x);
+    const int r0 = (int)((long long)L.R * bid / gdim);
+    const int r1 = (int)((long long)L.R * (bid + 1) / gdim);
     const int m_lo = r0 * L.v;
     const int m_hi = min(L.M, r1 * L.v);
 
@@ -400,7 +410,7 @@ decode_smem_fma_kernel(SmemFmaParams P)
         const int m = m_lo + ml;
         const int rr = m / L.v, jj = m - rr * L.v;
         const float y = part[((rr - r0) * TB + t) * 8 + jj] + bterm[t];
-        store_out(P.out, (long long)t * L.M + m, y, L.out_dtype);
+        store_out(out, (long long)t * L.M + m, y, L.out_dtype);
     }
 }
 
@@ -408,6 +418,7 @@ struct SmemFmaPlan {
     int slab_cols, n_slabs, cb2_rep, grid, part_floats, n_out_pad, warps;
     size_t smem;
     bool ok;
+    int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
 int fma_num_sms()
@@ -445,20 +456,42 @@ SmemFmaPlan plan_smem_fma(const LayerView &L, int TB)
     return p;
 }
 
+template <int TB, int VV, bool RES, int WARPS, bool FUSED>
+cudaError_t launch_kernel(const SmemFmaParams &P, const SmemFmaPlan &pl, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    if (e != cudaSuccess) return e;
+    decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
+    return cudaGetLastError();
+}
+
 template <int TB, int VV, int WARPS>
 cudaError_t launch_one(const SmemFmaParams &P, const SmemFmaPlan &pl, bool res, cudaStream_t st)
 {
-    cudaError_t e;
-    if (res) {
-        e = cudaFuncSetAttribute(decode_smem_fma_kernel<TB, VV, true, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-        if (e != cudaSuccess) return e;
-        decode_smem_fma_kernel<TB, VV, true, WARPS><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
-    } else {
-        e = cudaFuncSetAttribute(decode_smem_fma_kernel<TB, VV, false, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
-        if (e != cudaSuccess) return e;
-        decode_smem_fma_kernel<TB, VV, false, WARPS><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
-    }
-    return cudaGetLastError();
+    const bool fused = P.n_layers > 1;
+    if (res) return fused ? launch_kernel<TB, VV, true, WARPS, true>(P, pl, st) : launch_kernel<TB, VV, true, WARPS, false>(P, pl, st);
+    return fused ? launch_kernel<TB, VV, false, WARPS, true>(P, pl, st) : launch_kernel<TB, VV, false, WARPS, false>(P, pl, st);
+}
+
+// several layers of the same format (apart from M) in one grid
+bool plan_smem_fma_fused(const LayerView *Ls, int n, int TB, SmemFmaPlan *out)
+{
+    if (n < 2 || n > MAX_FUSED) return false;
+    for (int l = 1; l < n; l++)
+        if (!same_geometry(Ls[0], Ls[l])) return false;
+    SmemFmaPlan p = plan_smem_fma(Ls[0], TB);
+    if (!p.ok) return false;
+    int R[MAX_FUSED], rows_cta = 0;
+    for (int l = 0; l < n; l++) R[l] = Ls[l].R;
+    if (!split_ctas(R, n, fma_num_sms(), p.cta_begin, &rows_cta)) return false;
+    p.grid = fma_num_sms();
+    p.smem -= (size_t)p.part_floats * 4;
+    p.part_floats = rows_cta * TB * 8;
+    p.smem += (size_t)p.part_floats * 4;
+    if ((long long)p.part_floats * 4 > PART_BUDGET || p.smem > 224 * 1024) return false;
+    *out = p;
+    return true;
 }
 
 template <int TB, int WARPS>
@@ -498,9 +531,11 @@ cudaError_t launch_decode_smem_fma(const LayerView &L, const void *x, int B, voi
     const bool res = L.k2 > 0;
     for (int t0 = 0; t0 < B; t0 += TB) {
         SmemFmaParams P;
-        P.L = L; P.B = (B - t0 < TB) ? (B - t0) : TB;
+        memset(&P, 0, sizeof(P));
+        P.L[0] = L; P.n_layers = 1; P.cta_begin[1] = pl.grid;
+        P.B = (B - t0 < TB) ? (B - t0) : TB;
         P.x = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * xe;
-        P.out = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
+        P.out[0] = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
         P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.cb2_replicated = pl.cb2_rep;
         P.n_out_pad = pl.n_out_pad; P.part_floats = pl.part_floats;
         cudaError_t e;
@@ -508,6 +543,43 @@ cudaError_t launch_decode_smem_fma(const LayerView &L, const void *x, int B, voi
         else if (TB == 4) e = launch_vv<4, 16>(P, pl, L.v, res, st);
         else if (TB == 2) e = launch_vv<2, 32>(P, pl, L.v, res, st);
         else e = launch_vv<1, 32>(P, pl, L.v, res, st);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+bool smem_fma_fused_supported(const LayerView *Ls, int n, int B)
+{
+    for (int l = 0; l < n; l++)
+        if (!smem_fma_supported(Ls[l], B)) return false;
+    SmemFmaPlan pl;
+    return plan_smem_fma_fused(Ls, n, fma_token_group(B), &pl);
+}
+
+cudaError_t launch_decode_smem_fma_fused(const LayerView *Ls, int n, const void *x, int B, void *const *outs, cudaStream_t st)
+{
+    const int TB = fma_token_group(B);
+    SmemFmaPlan pl;
+    if (!plan_smem_fma_fused(Ls, n, TB, &pl)) return cudaErrorInvalidValue;
+    const bool res = Ls[0].k2 > 0;
+    for (int t0 = 0; t0 < B; t0 += TB) {
+        SmemFmaParams P;
+        memset(&P, 0, sizeof(P));
+        for (int l = 0; l < n; l++) {
+            P.L[l] = Ls[l];
+            P.out[l] = reinterpret_cast<uint8_t *>(outs[l]) + (size_t)t0 * Ls[l].M * (Ls[l].out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
+        }
+        for (int l = 0; l <= n; l++) P.cta_begin[l] = pl.cta_begin[l];
+        P.n_layers = n;
+        P.B = (B - t0 < TB) ? (B - t0) : TB;
+        P.x = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * Ls[0].N * 2;
+        P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.cb2_replicated = pl.cb2_rep;
+        P.n_out_pad = pl.n_out_pad; P.part_floats = pl.part_floats;
+        cudaError_t e;
+        if (TB == 8) e = launch_vv<8, 16>(P, pl, Ls[0].v, res, st);
+        else if (TB == 4) e = launch_vv<4, 16>(P, pl, Ls[0].v, res, st);
+        else if (TB == 2) e = launch_vv<2, 32>(P, pl, Ls[0].v, res, st);
+        else e = launch_vv<1, 32>(P, pl, Ls[0].v, res, st);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

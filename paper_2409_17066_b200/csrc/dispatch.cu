@@ -91,17 +91,32 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
 
 // ---- several layers that read the same activations ---------------------------------------------------
 
-bool fused_path_available(const LayerView *Ls, const int *flags, int n, int B)
+// The kernel family that serves all n layers with one launch per token group, or PATH_GENERIC when there is none.
+LinearPath fused_path(const LayerView *Ls, const int *flags, int n, int B)
 {
-    if (n < 2 || B > DECODE_MAX_B) return false;
-    for (int l = 0; l < n; l++)
-        if (choose_path(Ls[l], B, flags[l]) != PATH_DECODE_L2_FMA) return false;
-    return l2_fma_fused_supported(Ls, n, B);
+    if (n < 2 || B > DECODE_MAX_B) return PATH_GENERIC;
+    const LinearPath path = choose_path(Ls[0], B, flags[0]);
+    for (int l = 1; l < n; l++)
+        if (choose_path(Ls[l], B, flags[l]) != path) return PATH_GENERIC;
+    if (path == PATH_DECODE_L2_FMA && l2_fma_fused_supported(Ls, n, B)) return path;
+    if (path == PATH_DECODE_SMEM_FMA && smem_fma_fused_supported(Ls, n, B)) return path;
+    if (path == PATH_DECODE_GL_FMA && gl_fma_fused_supported(Ls, n, B)) return path;
+    return PATH_GENERIC;
+}
+
+const char *linear_fused_path_name(const LayerView *Ls, const int *flags, int n, int B)
+{
+    switch (fused_path(Ls, flags, n, B)) {
+    case PATH_DECODE_L2_FMA: return "fused_decode_l2_fma";
+    case PATH_DECODE_SMEM_FMA: return "fused_decode_smem_fma";
+    case PATH_DECODE_GL_FMA: return "fused_decode_gl_fma";
+    default: return "one_by_one";
+    }
 }
 
 long long linear_fused_workspace_bytes(const LayerView *Ls, const int *flags, int n, int B)
 {
-    if (fused_path_available(Ls, flags, n, B)) return 0;
+    if (fused_path(Ls, flags, n, B) != PATH_GENERIC) return 0;
     long long need = 0;       // one layer after the other on the stream: they share the scratch
     for (int l = 0; l < n; l++) {
         const long long w = linear_workspace_bytes(Ls[l], B, flags[l]);
@@ -112,7 +127,10 @@ long long linear_fused_workspace_bytes(const LayerView *Ls, const int *flags, in
 
 int linear_fused_launches(const LayerView *Ls, const int *flags, int n, int B)
 {
-    if (fused_path_available(Ls, flags, n, B)) return l2_fma_fused_launches(B);
+    const LinearPath path = fused_path(Ls, flags, n, B);
+    if (path == PATH_DECODE_L2_FMA) return l2_fma_fused_launches(B);
+    if (path == PATH_DECODE_SMEM_FMA) return smem_fma_launches(Ls[0], B);      // one launch per token group
+    if (path == PATH_DECODE_GL_FMA) return gl_fma_launches(Ls[0], B);
     int total = 0;
     for (int l = 0; l < n; l++) total += linear_launches(Ls[l], B, flags[l]);
     return total;
@@ -121,8 +139,11 @@ int linear_fused_launches(const LayerView *Ls, const int *flags, int n, int B)
 int linear_fused_dispatch(const LayerView *Ls, const int *flags, int n, const void *x, int B, void *const *outs,
                           void *ws, cudaStream_t st, cudaError_t *cuda_err)
 {
-    if (fused_path_available(Ls, flags, n, B)) {
-        *cuda_err = launch_decode_l2_fma_fused(Ls, n, x, B, outs, st);
+    const LinearPath path = fused_path(Ls, flags, n, B);
+    if (path != PATH_GENERIC) {
+        if (path == PATH_DECODE_L2_FMA) *cuda_err = launch_decode_l2_fma_fused(Ls, n, x, B, outs, st);
+        else if (path == PATH_DECODE_SMEM_FMA) *cuda_err = launch_decode_smem_fma_fused(Ls, n, x, B, outs, st);
+        else *cuda_err = launch_decode_gl_fma_fused(Ls, n, x, B, outs, st);
         return *cuda_err == cudaSuccess ? VPTQ_OK : VPTQ_E_CUDA;
     }
     for (int l = 0; l < n; l++) {

@@ -352,7 +352,7 @@ const char *vptq_linear_fused_path(const vptq_layer_desc *descs, int32_t n_layer
     LayerView Ls[VPTQ_MAX_FUSED_LAYERS];
     int flags[VPTQ_MAX_FUSED_LAYERS];
     if (fused_views(descs, nullptr, n_layers, B, Ls, flags) != VPTQ_OK) return "invalid";
-    return fused_path_available(Ls, flags, n_layers, B) ? "fused_decode_l2_fma" : "one_by_one";
+    return linear_fused_path_name(Ls, flags, n_layers, B);
 }
 
 int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,

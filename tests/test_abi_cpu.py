@@ -108,10 +108,16 @@ def test_fused_call_argument_errors_and_path_names(binding):
     assert b.vptq_linear_fused_workspace_bytes([q, kv, kv], 1) == 0
     assert b.vptq_linear_fused_launches([q, kv, kv], 1) == 1
     assert b.vptq_linear_fused_launches([q, kv, kv], 6) == 2          # token groups of 4
-    # layers that take another kernel family run one after the other and share the scratch
+    # layers of one format (apart from M) with their codebooks in shared memory are fused as well ...
     small = b.make_desc(11008, 4096, 6, 4096, 256, n_outlier=41, v0=4, k0=4096)
-    assert b.vptq_linear_fused_path([small, small], 1) == "one_by_one"
-    assert b.vptq_linear_fused_launches([small, small], 1) == 2 * b.vptq_linear_launches(small, 1)
+    assert b.vptq_linear_fused_path([small, small], 1) == "fused_decode_smem_fma"
+    assert b.vptq_linear_fused_launches([small, small], 1) == 1
+    # ... layers of different formats, or of different kernel families, run one after the other and share the scratch
+    other = b.make_desc(11008, 4096, 6, 4096, 256, n_outlier=40, v0=4, k0=4096)
+    assert b.vptq_linear_fused_path([small, other], 1) == "one_by_one"
+    assert b.vptq_linear_fused_launches([small, other], 1) == 2 * b.vptq_linear_launches(small, 1)
+    assert b.vptq_linear_fused_path([small, q], 1) == "invalid"            # different N
+    assert b.vptq_linear_fused_path([small, small], 8) == "one_by_one"      # 8 tokens: the mma kernel, not fused
     # a single layer, or many tokens, is not fused either
     assert b.vptq_linear_fused_path([q], 1) == "one_by_one"
     assert b.vptq_linear_fused_path([q, kv], 64) == "one_by_one"

@@ -244,6 +244,24 @@ def test_linear_fused_matches_oracle_and_single_calls(b, Ms, N, k2, B, out_dtype
         assert rel_err(y, y1.astype(np.float64)) <= 1e-3 * TOL + (4e-3 if dl.desc.out_dtype != b.DTYPE_FP32 else 0)
 
 
+@pytest.mark.parametrize("family,Ms,kw,B", [
+    ("fused_decode_smem_fma", (1200, 1176), dict(N=700, v=6, k1=4096, k2=256, n_out=7, v0=4, k0=4096), 1),
+    ("fused_decode_smem_fma", (1200, 900, 1500), dict(N=700, v=6, k1=4096, k2=256, n_out=7, v0=4, k0=4096), 3),
+    ("fused_decode_smem_fma", (1600, 1360), dict(N=520, v=8, k1=256), 4),
+    ("fused_decode_gl_fma", (1200, 1800), dict(N=134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4), 1),
+    ("fused_decode_gl_fma", (1200, 1800), dict(N=134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4, permuted=True), 2),
+])
+def test_linear_fused_other_kernel_families(b, family, Ms, kw, B):
+    specs = [synth.LayerSpec("f%d" % i, M, **kw) for i, M in enumerate(Ms)]
+    ds, dls, x, outs = _fused_case(b, specs, B, 411)
+    assert b.vptq_linear_fused_path([dl.desc for dl in dls], B) == family
+    assert b.vptq_linear_fused_workspace_bytes([dl.desc for dl in dls], B) == 0
+    for d, dl, y in zip(ds, dls, outs):
+        y = y.float().cpu().numpy()
+        assert np.isfinite(y).all()
+        assert rel_err(y, oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+
+
 def test_linear_fused_runs_other_kernel_families_one_by_one(b):
     spec = {sp.name: sp for sp in synth.small_specs()}["s_v6_full"]
     specs = [spec, spec]
