@@ -492,7 +492,46 @@ def extra_configs(vb, synth, peaks):
                 res[key] = r
             del variants, base, d
             torch.cuda.empty_cache()
+    res.update(extra_fused(vb, synth, peaks))
     res.update(encoder_assign(vb, synth))
+    return res
+
+
+def extra_fused(vb, synth, peaks):
+    """Projections that read the same activations through one vptq_linear_fused call, against one call per layer
+    (device time per call from CUDA-graph replays over > 2 x L2 of weight copies), for the workloads whose decode
+    kernels keep the codebooks in shared memory (config 2) or per group in global memory (the published 2.26-bit
+    setting); the k/v projections of those models have the shape of q."""
+    import torch
+    res = {}
+    for cfg, names, B in ((2, ("gate_proj", "up_proj"), 1), (5, ("q_proj", "q_proj", "q_proj"), 1),
+                          (5, ("gate_proj", "gate_proj"), 1)):
+        by_name = {s.name: (li, s) for li, s in enumerate(synth.CONFIGS[cfg]["layers"])}
+        ds = []
+        for i, nm in enumerate(names):
+            li, sp = by_name[nm]
+            ds.append(synth.make_layer(sp, cfg, li + 10 * i, B))       # weights of its own per projection
+        for d in ds[1:]:
+            d["x"] = ds[0]["x"]
+        base = [vb.DeviceLayer(d) for d in ds]
+        wb = sum(dl.weight_bytes() for dl in base)
+        n = max(2, min(32, int(2 * 130e6 / wb) + 1))
+        copies = [[dl] + [dl.clone_streams() for _ in range(n - 1)] for dl in base]
+        fused = [vb.FusedLayers([copies[l][c] for l in range(len(base))]) for c in range(n)]
+        x = base[0].upload_x(ds[0]["x"][:B])
+        outs = [torch.empty((B, dl.spec.M), dtype=vb._TORCH_DT[dl.desc.out_dtype], device="cuda") for dl in base]
+        g, _, _ = time_calls(lambda i: fused[i].linear(x, outs), n)
+
+        def one_by_one(i):
+            for l in range(len(base)):
+                copies[l][i].linear(x, outs[l])
+        gs, _, _ = time_calls(one_by_one, n)
+        label = "+".join(names) if len(set(names)) > 1 else f"{len(names)}x{names[0]}"
+        res[f"cfg{cfg}_fused_{label}_B{B}"] = {
+            "us": 1e3 * g, "us_one_call_per_layer": 1e3 * gs, "GBps": wb / (g * 1e-3) / 1e9,
+            "frac_hbm": wb / (g * 1e-3) / 1e9 / peaks["hbm"], "path": fused[0].path(B), "weight_copies": n}
+        del fused, copies, base, ds
+        torch.cuda.empty_cache()
     return res
 
 
