@@ -332,6 +332,25 @@ def test_assign_on_tensor_cores_with_ties_everywhere(b):
     assert np.array_equal(idx, oracle.assign(Wb, v, big))
 
 
+@pytest.mark.parametrize("flags", [0, 4], ids=["tensor_cores", "fp32"])
+def test_assign_with_values_that_are_not_numbers(b, flags):
+    # NaN and infinite components: such distances never win (oracle rule); the tensor-core filter cannot rank
+    # them and sends the vectors (all of them, when the codebook has such an entry) through the full FP32 scan
+    rng = np.random.default_rng(31)
+    M, N, v, k = 64, 600, 8, 2048
+    W = rng.normal(0, 0.02, (M, N)).astype(np.float16)
+    W[3, 5] = np.nan
+    W[17, 100] = np.inf
+    W[40, 7] = -np.inf
+    Cb = rng.normal(0, 0.02, (k, v)).astype(np.float16)
+    for bad_codebook in (False, True):
+        if bad_codebook:
+            Cb[77, 2] = np.nan
+            Cb[900, 0] = np.inf
+        idx = b.vptq_assign(torch.from_numpy(W).cuda(), v, torch.from_numpy(Cb).cuda(), flags).cpu().numpy()
+        assert np.array_equal(idx, oracle.assign(W, v, Cb))
+
+
 def test_assign_then_pack_and_dequant_reproduce_the_matrix(b):
     # a matrix built from centroids goes through assign -> pack -> dequant unchanged
     spec = synth.LayerSpec("enc", 264, 300, v=8, k1=4096, has_scale=False)

@@ -558,3 +558,11 @@ def test_a_kmeans_step_never_increases_the_weighted_distortion():
     idx_r = oracle.assign(Wr, v, C)
     Cr = oracle.kmeans_update(Wr, v, idx_r, C, h)
     assert oracle.distortion(Wr, v, idx_r, Cr, h) <= oracle.distortion(Wr, v, idx_r, C, h) * (1 + 2e-3)
+
+
+def test_assign_distances_that_are_not_numbers_never_win():
+    # a centroid with a NaN component is never chosen; a vector with a NaN or infinite component gets index 0
+    C = np.array([[np.nan, 0.0], [1.0, 1.0], [5.0, 5.0]], np.float16)
+    W = np.array([[1.0, 5.0, np.nan, np.inf], [1.25, 4.0, 0.0, 0.0]], np.float16)
+    assert oracle.assign(W, 2, C).tolist() == [[1, 2, 0, 0]]
+
