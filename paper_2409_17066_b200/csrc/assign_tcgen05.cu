@@ -4,7 +4,9 @@
 // vector's components: D[vector][centroid] = A * B^T with
 //   A row (a vector):   x_0 .. x_{v-1}, 0 .., 1, 2^-11            (16 FP16 values, K = 16)
 //   B row (a centroid): -2c_0 .. -2c_{v-1}, 0 .., hi, 2^11 lo     hi + lo = ||c||^2 split into two FP16 values
-//                                                                (lo scaled so that it does not underflow)
+// with x and c first multiplied by a power of two 2^s that brings max ||c||^2 to about 2^8: FP16 keeps its
+// 11 bits only for normal numbers, and small weights (1e-4) and their squared norms are far below them.
+// The scaling is exact for values that stay in range and leaves the order of the distances unchanged.
 // One tcgen05.mma (M = 128 vectors, N = 128 centroids, K = 16) gives 16 K approximate distances.  They
 // only FILTER: per vector the kernel keeps the smallest and the second smallest minimum over groups of
 // 32 centroids and the group of the smallest.  Then the 32 centroids of that group are evaluated with
@@ -13,7 +15,8 @@
 // a list; a second kernel scans all centroids for the vectors on the list (one warp per vector).  The indices are therefore
 // those of the FP32 definition, bit for bit, whatever the tensor core's summation order.
 //   bound: |filter - (definition - ||x||^2)| <= 2^-18 (||x||^2 + max ||c||^2) (FP16 split of the norm,
-//   FP32 accumulation of 10 products, rounding of the fma chain); the margin tested is 2^-14 of it.
+//   FP32 accumulation of 10 products, rounding of the fma chain); the margin tested is 2^-15 of that sum,
+//   four times what two such errors can add up to.
 //
 // Persistent grid, one CTA per SM, 256 vectors (two A tiles) per step.  Warp 0 streams the prepared
 // centroid tiles (4 KB, shared-memory image with the 32-byte swizzle applied by the preparation kernel)
@@ -42,7 +45,7 @@ constexpr int SCAN_THREADS = 32 * (2 + EPI_WARPS);
 constexpr int STEP_VECTORS = 256;             // two A tiles
 constexpr int GROUP = 32;                     // centroids per candidate group (one tcgen05.ld)
 constexpr float PAD_NORM = 60000.f;           // norm of the padding rows of the last centroid tile: never the minimum
-constexpr float MARGIN = 1.0f / 16384.0f;     // 2^-14
+constexpr float MARGIN = 1.0f / 32768.0f;     // 2^-15
 
 struct ScanParams {
     const __half *W;
@@ -106,14 +109,37 @@ __device__ __forceinline__ float min32(const uint32_t (&d)[32])
 // byte offset of 16-byte chunk c (0 or 1) of row r in a tile image (32-byte swizzle: bit 4 ^= bit 7)
 __device__ __forceinline__ int image_offset(int r, int c) { return r * ROW_BYTES + ((c ^ ((r >> 2) & 1)) << 4); }
 
-// ---- preparation: the centroid tiles as shared-memory images, and max ||c||^2 ---------------------------
+// The power of two that brings max ||c||^2 to [2^8, 2^10): 2^s multiplies vectors and centroids.
+__device__ __forceinline__ int scale_exponent(float cmax)
+{
+    if (!(cmax > 0.f) || !(cmax < 3.0e38f)) return 0;
+    int s = (8 - ilogbf(cmax) + 1) / 2;                 // ilogbf: floor(log2)
+    return s < -12 ? -12 : (s > 24 ? 24 : s);
+}
+
+// ---- preparation, first pass: max ||c||^2; clears the list count and the status word -------------------------
 __global__ void __launch_bounds__(256)
-assign_prepare_kernel(const __half *__restrict__ C, int k, int v, uint8_t *__restrict__ Bimg, float *cmax,
-                      int *count, int *status, int k_tiles)
+assign_norms_kernel(const __half *__restrict__ C, int k, int v, float *cmax, int *count, int *status)
+{
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i == 0) { *count = 0; *status = 0; }
+    if (i >= k) return;
+    float norm = 0.f;
+    for (int j = 0; j < v; j++) {
+        const float c = __half2float(__ldg(C + (long long)i * v + j));
+        norm = __fmaf_rn(c, c, norm);
+    }
+    // norm >= 0: integer order = float order; a NaN norm has the largest bit pattern and so becomes the maximum
+    atomicMax(reinterpret_cast<int *>(cmax), __float_as_int(norm));
+}
+
+// ---- preparation, second pass: the scaled centroid tiles as shared-memory images -----------------------------
+__global__ void __launch_bounds__(256)
+assign_prepare_kernel(const __half *__restrict__ C, int k, int v, uint8_t *__restrict__ Bimg, const float *cmax, int k_tiles)
 {
     const int i = blockIdx.x * 256 + threadIdx.x;          // centroid (or padding row of the last tile)
-    if (i == 0) { *count = 0; *status = 0; }
     if (i >= k_tiles * KT) return;
+    const float scale = exp2f((float)scale_exponent(*cmax));
     __half row[16];
 #pragma unroll
     for (int j = 0; j < 16; j++) row[j] = __float2half_rn(0.f);
@@ -121,11 +147,10 @@ assign_prepare_kernel(const __half *__restrict__ C, int k, int v, uint8_t *__res
     if (i < k) {
         norm = 0.f;
         for (int j = 0; j < v; j++) {
-            const float c = __half2float(__ldg(C + (long long)i * v + j));
+            const float c = __half2float(__ldg(C + (long long)i * v + j)) * scale;
             norm = __fmaf_rn(c, c, norm);
-            row[j] = __float2half_rn(-2.f * c);             // exact (a power of two), overflow apart
+            row[j] = __float2half_rn(-2.f * c);             // exact while in range
         }
-        atomicMax(reinterpret_cast<int *>(cmax), __float_as_int(norm));      // norm >= 0: integer order = float order
     }
     const __half hi = __float2half_rn(norm);
     row[14] = hi;
@@ -223,7 +248,8 @@ assign_scan_kernel(ScanParams P)
         const int q = warp & 3;                      // TMEM lane quarter this warp may read
         const int a = ew >> 2;                       // A tile
         const int row = 32 * q + lane;               // row of the A tile = TMEM lane
-        const float cmax = __ldg(P.cmax);
+        const float scale = exp2f((float)scale_exponent(__ldg(P.cmax)));
+        const float cmax = __ldg(P.cmax) * scale * scale;      // in the filter's units
         long long it = 0;
         for (long long step = blockIdx.x; step < n_steps && ok; step += gridDim.x) {
             const long long g = step * STEP_VECTORS + a * 128 + row;
@@ -234,13 +260,13 @@ assign_scan_kernel(ScanParams P)
 #pragma unroll
             for (int j = 0; j < VMAX; j++) {
                 x[j] = (valid && j < P.v) ? __half2float(__ldg(P.W + (long long)(r * P.v + j) * P.N + n)) : 0.f;
-                xn = __fmaf_rn(x[j], x[j], xn);
+                xn = __fmaf_rn(x[j] * scale, x[j] * scale, xn);
             }
             // the A tile of this step may be overwritten: its MMAs completed before the last accFull of the previous step
             {
                 __half rowv[16];
 #pragma unroll
-                for (int j = 0; j < 14; j++) rowv[j] = __float2half_rn(j < VMAX ? x[j < VMAX ? j : 0] : 0.f);   // exact: x came from FP16
+                for (int j = 0; j < 14; j++) rowv[j] = __float2half_rn(j < VMAX ? x[j < VMAX ? j : 0] * scale : 0.f);   // exact while in range
                 rowv[14] = __float2half_rn(1.f);         // times hi
                 rowv[15] = __float2half_rn(1.f / 2048.f);    // times 2^11 lo
                 const uint4 *src = reinterpret_cast<const uint4 *>(rowv);
@@ -298,8 +324,10 @@ assign_scan_kernel(ScanParams P)
                 P.idx[g] = best;
                 // not clearly the only candidate group: the full scan decides
                 const float eps = MARGIN * (xn + cmax);
-                // (norms beyond the FP16 range make the filter meaningless: then every vector is listed)
-                if (!(b2 - b1 > eps) || !(fabsf(b1) < 3.0e38f) || !(cmax < PAD_NORM)) P.list[atomicAdd(P.count, 1)] = (int)g;
+                // (a vector or a table that leaves the FP16 range even after scaling makes the filter meaningless:
+                //  such vectors, or then all of them, are listed)
+                if (!(b2 - b1 > eps) || !(fabsf(b1) < 3.0e38f) || !(xn < 3.0e9f) || !(cmax < PAD_NORM))
+                    P.list[atomicAdd(P.count, 1)] = (int)g;
             }
         }
     }
@@ -376,9 +404,11 @@ cudaError_t launch_assign_tcgen05(const __half *W, int M, int N, int v, const __
     P.k_tiles = l.k_tiles;
     cudaError_t e = cudaMemsetAsync(w8 + l.off_cmax, 0, 4, st);
     if (e != cudaSuccess) return e;
-    assign_prepare_kernel<<<ceil_div(l.k_tiles * KT, 256), 256, 0, st>>>(C, k, v, w8 + l.off_bimg,
-                                                                         reinterpret_cast<float *>(w8 + l.off_cmax),
-                                                                         P.count, P.status, l.k_tiles);
+    assign_norms_kernel<<<ceil_div(k, 256), 256, 0, st>>>(C, k, v, reinterpret_cast<float *>(w8 + l.off_cmax),
+                                                          P.count, P.status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    assign_prepare_kernel<<<ceil_div(l.k_tiles * KT, 256), 256, 0, st>>>(C, k, v, w8 + l.off_bimg, P.cmax, l.k_tiles);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long n_steps = (n_vectors + STEP_VECTORS - 1) / STEP_VECTORS;

@@ -301,6 +301,8 @@ def test_assign_is_bit_identical_to_the_oracle(b, M, N, v, k):
     (72, 520, 1, 1024, 1.0),       # v = 1
     (136, 520, 8, 4096, 1e-3),     # small values: norms of about 1e-5 (the low half of the FP16 split must not underflow)
     (136, 520, 8, 4096, 1e-4),     # FP16 subnormals throughout
+    (136, 520, 8, 4096, 3e-6),     # a few FP16 subnormal steps: many equal vectors and centroids
+    (136, 520, 8, 4096, 3000.0),   # near the top of the FP16 range
 ])
 def test_assign_on_tensor_cores_gives_the_same_indices(b, M, N, v, k, sigma):
     rng = np.random.default_rng(77 * v + k)
