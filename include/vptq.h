@@ -175,12 +175,15 @@ int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
  *   descs, ptrs  host arrays of n_layers descriptors / pointer sets; all layers have the same N and
  *                x_dtype (else VPTQ_E_SHAPE); M, codebooks, scale/bias and out_dtype are per layer
  *   outs         host array of n_layers DEVICE pointers, outs[l] = [B][M_l] row-major
- * When every layer takes the "decode_l2_fma" path (B <= 16) and whole vector rows of the layers spread
- * evenly over the SMs, one kernel per token group serves all layers (no launch, prologue and ragged
- * tail per layer; no scratch); otherwise the layers run one after the other on `stream`, sharing the
- * workspace.  vptq_linear_fused_path() names which: "fused_decode_l2_fma" or "one_by_one".  Each
- * layer's result is the one vptq_linear gives for it (same arithmetic, same summation order within a
- * vector row).  Errors as for vptq_linear; nothing is launched when an argument is rejected. */
+ * When every layer takes the same one of the decode paths "decode_l2_fma" (B <= 16), "decode_smem_fma"
+ * or "decode_gl_fma" (B <= 4; for these two the layers must also share their format apart from M: v,
+ * codebook sizes, outlier columns, groups, scale flag) and whole vector rows of the layers spread evenly
+ * over the SMs, one kernel per token group serves all layers (no launch, prologue and ragged tail per
+ * layer; no scratch); otherwise the layers run one after the other on `stream`, sharing the workspace.
+ * vptq_linear_fused_path() names which: "fused_decode_l2_fma", "fused_decode_smem_fma",
+ * "fused_decode_gl_fma" or "one_by_one" ("invalid" for arguments the call would reject).  Each layer's
+ * result is the one vptq_linear gives for it (same arithmetic, same summation order within a vector
+ * row).  Errors as for vptq_linear; nothing is launched when an argument is rejected. */
 #define VPTQ_MAX_FUSED_LAYERS 4
 int64_t vptq_linear_fused_workspace_bytes(const vptq_layer_desc *descs, int32_t n_layers, int32_t B);
 int vptq_linear_fused(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
