@@ -262,6 +262,24 @@ def test_linear_fused_other_kernel_families(b, family, Ms, kw, B):
         assert rel_err(y, oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
 
 
+def test_linear_fused_host_io_matches_the_device_call(b):
+    specs = [synth.LayerSpec("h%d" % i, M, 4096, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype=od)
+             for i, (M, od) in enumerate(((4096, "fp16"), (1024, "fp32"), (1024, "fp16")))]
+    B = 2
+    ds, dls, x, outs = _fused_case(b, specs, B, 511)
+    fused = b.FusedLayers(dls)
+    assert fused.path(B) == "fused_decode_l2_fma"
+    x_host = torch.from_numpy(np.ascontiguousarray(ds[0]["x"])).view(torch.bfloat16).pin_memory()
+    outs_host = [torch.empty_like(o, device="cpu").pin_memory() for o in outs]
+    x_dev = torch.empty_like(x)
+    outs_dev = [torch.empty_like(o) for o in outs]
+    fused.linear_host_io(x_host, outs_host, x_dev, outs_dev)
+    torch.cuda.synchronize()
+    for d, oh, o in zip(ds, outs_host, outs):
+        assert rel_err(oh.float().numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+        assert rel_err(oh.float().numpy(), o.float().cpu().numpy().astype(np.float64)) <= 4e-3
+
+
 def test_linear_fused_runs_other_kernel_families_one_by_one(b):
     spec = {sp.name: sp for sp in synth.small_specs()}["s_v6_full"]
     specs = [spec, spec]
