@@ -262,6 +262,22 @@ def test_linear_fused_other_kernel_families(b, family, Ms, kw, B):
         assert rel_err(y, oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
 
 
+@pytest.mark.parametrize("B", [1, 40])
+def test_linear_host_io_matches_the_device_call(b, B):
+    # host activations in, host result out (pinned memory), the weights resident: the decode and the batched path
+    spec = synth.LayerSpec("hio", 264, 1030, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32")
+    d = synth.make_layer(spec, 79, 2, B)
+    dl = b.DeviceLayer(d)
+    x_host = torch.from_numpy(np.ascontiguousarray(d["x"])).view(torch.bfloat16).pin_memory()
+    out_host = torch.empty((B, spec.M), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty((B, spec.N), dtype=torch.bfloat16, device="cuda")
+    out_dev = torch.empty((B, spec.M), dtype=torch.float32, device="cuda")
+    b.vptq_linear_host_io(dl.desc, x_host, dl.ptrs, out_host, x_dev, out_dev, dl.workspace(B))
+    torch.cuda.synchronize()
+    assert rel_err(out_host.numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+    assert torch.equal(out_host, out_dev.cpu())
+
+
 def test_linear_fused_host_io_matches_the_device_call(b):
     specs = [synth.LayerSpec("h%d" % i, M, 4096, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype=od)
              for i, (M, od) in enumerate(((4096, "fp16"), (1024, "fp32"), (1024, "fp16")))]
