@@ -36,7 +36,12 @@
  * their FP32 operation order, the bit-packed index stream, "the first n_out
  * STORED columns are the outlier columns", and the form of the column order
  * (an explicit list of N input-feature numbers; scale and bias follow the
- * stored order).
+ * stored order), and the arithmetic of the assignment step (Eq. 2 names the
+ * Euclidean distance, not its precision, summation order or tie rule: FP32, fused
+ * multiply-add, components ascending, lowest index wins).
+ *
+ * Every function has a pin in tests/test_oracle_pins.py that is not itself: none is
+ * "parity unpinned" except in the sense above (choices the paper does not make).
  *
  * Arithmetic: lookup sum, scale and bias in FP32 with three separately rounded
  * operations (build with -ffp-contract=off), result rounded to FP16
