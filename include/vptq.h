@@ -26,7 +26,10 @@
  * Conventions, unless an entry point says otherwise:
  *   - every data pointer is a DEVICE pointer owned by the caller and must be 16-byte
  *     aligned; the library allocates nothing and keeps no state between calls;
- *   - `stream` is a cudaStream_t passed as void*; calls are asynchronous on it;
+ *   - `stream` is a cudaStream_t passed as void*; calls are asynchronous on it.  It must belong to
+ *     the CURRENT device, and so must every pointer: launch plans (grid sizes, row splits, scratch
+ *     needs and so the answers of the *_workspace_bytes queries) follow the current device's SM count,
+ *     and vptq_linear_noalloc takes the current device's copy of its built-in scratch;
  *   - the return value is 0 (VPTQ_OK) or a negative VPTQ_E_* code; nothing throws,
  *     aborts or traps.  vptq_status_string() names a code; vptq_last_cuda_error()
  *     gives the CUDA runtime's text for the last VPTQ_E_CUDA on this thread.
@@ -136,6 +139,15 @@ int vptq_pack(const int32_t *idx, int32_t n_rows, int32_t n_cols, int32_t k,
 int vptq_unpack(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k,
                 int32_t *idx, void *stream);
 
+/* The same two steps on HOST memory, for callers that prepare or inspect a checkpoint on the CPU (the
+ * paper does not describe a stream format; this is the format statement at the top of this file applied
+ * by plain host code, no CUDA call, synchronous).  idx and packed are host pointers of any alignment.
+ * vptq_pack_host writes every byte of `packed` (padding included), stores 0 for an index outside [0,k)
+ * and then returns VPTQ_E_INDEX_RANGE; vptq_unpack_host never reads past a row's ceil(cols*b/8) bytes.
+ * Byte for byte the streams of vptq_pack / vptq_unpack. */
+int vptq_pack_host(const int32_t *idx, int32_t n_rows, int32_t n_cols, int32_t k, uint8_t *packed);
+int vptq_unpack_host(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k, int32_t *idx);
+
 /* ---- dequantisation (Sec. 2.2 "dequantizes the weight matrix from the lookup table by
  *      index and centroid"; Sec. 3.2.2 decode; Sec. 3.2.3; App. D.2 "restore to FP16") -- */
 
@@ -231,8 +243,8 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *
  * Limits and errors: layers of another geometry return VPTQ_E_UNSUPPORTED.  The kernel
  * needs scratch only when the layer's vector rows do not divide well over the SMs (it then
- * deals the work out regardless of rows and adds partial sums up in scratch): 4 * min(B,4) * M
- * bytes plus a few KB of counters.  A layer whose need exceeds the array returns
+ * deals the work out regardless of rows and adds partial sums up in scratch): 4 * g * M bytes, g the
+ * tokens per launch (4 for B >= 4, 2 for B = 2 or 3, else 1), plus a few KB of counters.  A layer whose need exceeds the array returns
  * VPTQ_E_SCRATCH_LIMIT (M up to about 65000 fits at any B); nothing is launched in either
  * case.  vptq_linear_workspace_bytes() tells the need of a given layer and B.
  *
@@ -254,7 +266,7 @@ int vptq_linear_noalloc(const vptq_layer_desc *desc, const void *x, int32_t B,
  * weight matrix (v consecutive rows of one column: Sec. 3.1, Algorithm 1), i.e. the index matrix that
  * vptq_pack packs and vptq_dequant looks up again.  (With a Hessian-weighted objective the weight of a
  * vector's column is common to all its distances and does not change the argmin: Sec. 3.2.1 moves the
- * weights into the k-means centroid update, which this library does not have.)
+ * weights into the k-means centroid update: vptq_kmeans_update below.)
  *   W        fp16 [M][N] row-major (device)      codebook  fp16 [k][v] (device)
  *   idx      int32 [ceil(M/v)][N] (device, written)
  * Arithmetic, fixed because it decides an integer: FP32, components in ascending order,
@@ -294,10 +306,11 @@ int vptq_kmeans_update(const void *W, int32_t M, int32_t N, int32_t v, const int
 
 const char *vptq_status_string(int code);
 const char *vptq_last_cuda_error(void);
-/* Only meaningful after a vptq_linear call that took the "gemm_tcgen05" path: that path keeps an
- * int32 status word at byte 0 of its workspace.  This call synchronises `stream`, reads the word
- * and returns VPTQ_E_TIMEOUT if a bounded device-side wait gave up during the call (the output
- * is then invalid; the context stays usable), else VPTQ_OK.  A null workspace returns VPTQ_OK. */
+/* The two tensor-core paths — vptq_linear on "gemm_tcgen05" and vptq_assign on "assign_tcgen05" — keep an
+ * int32 status word at byte 0 of their workspace; after any other call the workspace holds no status and
+ * this call has no meaning.  It synchronises `stream`, reads the word and returns VPTQ_E_TIMEOUT if a
+ * bounded device-side wait gave up during the call (the output is then invalid; the context stays
+ * usable), else VPTQ_OK.  A null workspace returns VPTQ_OK. */
 int vptq_workspace_status(const void *workspace, void *stream);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_fma",
  * "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05".  For tests and benchmark logs. */

@@ -58,6 +58,8 @@ EXPORTS = {
     "vptq_layer_weight_bytes": (C.c_int64, [C.POINTER(LayerDesc)]),
     "vptq_pack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
+    "vptq_pack_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
+    "vptq_unpack_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
     "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
                               C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -157,6 +159,23 @@ def vptq_unpack(packed: torch.Tensor, rows: int, cols: int, k: int) -> torch.Ten
     assert packed.numel() == lib.vptq_packed_bytes(rows, cols, k)
     idx = torch.empty((rows, cols), dtype=torch.int32, device=packed.device)
     _check(lib.vptq_unpack(_ptr(packed), rows, cols, k, _ptr(idx), _stream()))
+    return idx
+
+
+def vptq_pack_host(idx: np.ndarray, k: int) -> np.ndarray:
+    """Host int32 [rows][cols] -> host uint8 [rows][row_bytes] (no CUDA call)."""
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    rows, cols = idx.shape
+    packed = np.empty((rows, max(0, lib.vptq_packed_row_bytes(cols, k))), dtype=np.uint8)
+    _check(lib.vptq_pack_host(idx.ctypes.data, rows, cols, k, packed.ctypes.data))
+    return packed
+
+
+def vptq_unpack_host(packed: np.ndarray, rows: int, cols: int, k: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    assert packed.size == lib.vptq_packed_bytes(rows, cols, k)
+    idx = np.empty((rows, cols), dtype=np.int32)
+    _check(lib.vptq_unpack_host(packed.ctypes.data, rows, cols, k, idx.ctypes.data))
     return idx
 
 

@@ -342,18 +342,6 @@ assign_scan_kernel(ScanParams P)
     }
 }
 
-int scan_sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 struct ScanLayout {
     long long off_cmax, off_count, off_bimg, off_list, bytes;
     int k_tiles;
@@ -412,13 +400,13 @@ cudaError_t launch_assign_tcgen05(const __half *W, int M, int N, int v, const __
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const long long n_steps = (n_vectors + STEP_VECTORS - 1) / STEP_VECTORS;
-    const int grid = (int)(n_steps < scan_sm_count() ? n_steps : scan_sm_count());
+    const int grid = (int)(n_steps < device_sm_count() ? n_steps : device_sm_count());
     if (v <= 8) assign_scan_kernel<8><<<grid, SCAN_THREADS, 0, st>>>(P);
     else assign_scan_kernel<14><<<grid, SCAN_THREADS, 0, st>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     // the vectors whose candidate group was not clearly the only one: all centroids, FP32
-    return launch_assign_listed(W, M, N, v, C, k, idx, P.list, P.count, scan_sm_count(), st);
+    return launch_assign_listed(W, M, N, v, C, k, idx, P.list, P.count, device_sm_count(), st);
 }
 
 }  // namespace vptq

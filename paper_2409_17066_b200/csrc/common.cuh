@@ -98,11 +98,17 @@ __device__ __forceinline__ void store_out(void *out, long long i, float val, int
 }
 #endif
 
+// streaming multiprocessors of the current device, cached per device ordinal (device_info.cu)
+int device_sm_count();
+
 // ---- launchers implemented in the kernel files -------------------------------------------
 cudaError_t launch_pack(const int32_t *idx, int rows, int cols, int k, uint8_t *packed,
                         int32_t *bad_count, cudaStream_t st);
 cudaError_t launch_unpack(const uint8_t *packed, int rows, int cols, int k, int32_t *idx,
                           cudaStream_t st);
+// the same two steps on host memory (pack_host.cu); pack_host returns the number of indices outside [0,k)
+long long pack_host(const int32_t *idx, int rows, int cols, int k, uint8_t *packed);
+void unpack_host(const uint8_t *packed, int rows, int cols, int k, int32_t *idx);
 cudaError_t launch_dequant(const LayerView &L, __half *W, cudaStream_t st);
 // assignment step of the quantizer (Eq. 2): idx [ceil(M/v)][N]
 bool assign_supported(int v, int k);

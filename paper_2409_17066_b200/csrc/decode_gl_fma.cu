@@ -415,24 +415,12 @@ struct GlFmaPlan {
     int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
-int gl_num_sms()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 int gl_token_group(int B) { return B >= 4 ? 4 : (B >= 2 ? 2 : 1); }
 
 GlFmaPlan plan_gl_fma(const LayerView &L, int TB)
 {
     GlFmaPlan p;
-    const int G = gl_num_sms();
+    const int G = device_sm_count();
     p.grid = L.R < G ? L.R : G;
     const int rows_cta = ceil_div(L.R, p.grid);
     p.part_floats = rows_cta * TB * 16;
@@ -484,8 +472,8 @@ bool plan_gl_fma_fused(const LayerView *Ls, int n, int TB, GlFmaPlan *out)
     if (!p.ok) return false;
     int R[MAX_FUSED], rows_cta = 0;
     for (int l = 0; l < n; l++) R[l] = Ls[l].R;
-    if (!split_ctas(R, n, gl_num_sms(), p.cta_begin, &rows_cta)) return false;
-    p.grid = gl_num_sms();
+    if (!split_ctas(R, n, device_sm_count(), p.cta_begin, &rows_cta)) return false;
+    p.grid = device_sm_count();
     p.smem -= (size_t)p.part_floats * 4;
     p.part_floats = rows_cta * TB * 16;
     p.smem += (size_t)p.part_floats * 4;

@@ -392,18 +392,6 @@ struct L2Plan {
     int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
-int l2_num_sms()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 L2Plan plan_l2(const LayerView &L, int TB)
 {
     L2Plan p;
@@ -414,7 +402,7 @@ L2Plan plan_l2(const LayerView &L, int TB)
     p.slab_cols = slab;
     p.n_slabs = (n_pad + slab - 1) / slab;
     p.chunks_total = n_pad / 256;
-    const int G = l2_num_sms();
+    const int G = device_sm_count();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
     // OWNER mode when whole rows divide well over the SMs (and over the warps of a CTA)
     const int rows_cta = ceil_div(L.R, G);
@@ -447,7 +435,7 @@ bool plan_l2_fused(const LayerView *Ls, int n, int TB, L2Plan *out)
     for (int l = 1; l < n; l++)
         if (Ls[l].N != Ls[0].N || Ls[l].x_bf16 != Ls[0].x_bf16 || Ls[l].k2 != Ls[0].k2) return false;
     L2Plan p = plan_l2(Ls[0], TB);          // slab geometry, warps, residual table: functions of N, k2, TB
-    const int G = l2_num_sms();
+    const int G = device_sm_count();
     int R[MAX_FUSED], rows_cta = 0;
     long long rows = 0;
     for (int l = 0; l < n; l++) { R[l] = Ls[l].R; rows += Ls[l].R; }

@@ -421,25 +421,13 @@ struct SmemFmaPlan {
     int cta_begin[MAX_FUSED + 1];   // fused launches only
 };
 
-int fma_num_sms()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 int fma_token_group(int B) { return B >= 8 ? 8 : (B >= 4 ? 4 : (B >= 2 ? 2 : 1)); }
 
 SmemFmaPlan plan_smem_fma(const LayerView &L, int TB)
 {
     SmemFmaPlan p;
     p.warps = TB >= 4 ? 16 : 32;
-    const int G = fma_num_sms();
+    const int G = device_sm_count();
     p.grid = L.R < G ? L.R : G;
     const int rows_cta = ceil_div(L.R, p.grid);
     p.part_floats = rows_cta * TB * 8;
@@ -484,8 +472,8 @@ bool plan_smem_fma_fused(const LayerView *Ls, int n, int TB, SmemFmaPlan *out)
     if (!p.ok) return false;
     int R[MAX_FUSED], rows_cta = 0;
     for (int l = 0; l < n; l++) R[l] = Ls[l].R;
-    if (!split_ctas(R, n, fma_num_sms(), p.cta_begin, &rows_cta)) return false;
-    p.grid = fma_num_sms();
+    if (!split_ctas(R, n, device_sm_count(), p.cta_begin, &rows_cta)) return false;
+    p.grid = device_sm_count();
     p.smem -= (size_t)p.part_floats * 4;
     p.part_floats = rows_cta * TB * 8;
     p.smem += (size_t)p.part_floats * 4;

@@ -475,21 +475,6 @@ bool smem_mma_supported(const LayerView &L, int B)
     return true;
 }
 
-static int g_num_sms = 0;
-
-static int num_sms()
-{
-    if (g_num_sms == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            g_num_sms = n;
-        else
-            return 148;
-    }
-    return g_num_sms;
-}
-
 namespace {
 template <int NT>
 cudaError_t launch_variant(const SmemMmaParams &P, bool perm, int grid, size_t smem, cudaStream_t st)
@@ -516,7 +501,7 @@ cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, voi
     const int TP = 8 * NT;
     P.cb1_bytes = L.Nc > 0 ? pad16(L.k1 * 16) : 0;
     P.cb2_bytes = L.k2 ? pad16(L.k2 * 16) : 0;
-    const int sms = num_sms();
+    const int sms = device_sm_count();
     P.rows_per_cta = ceil_div(L.R, sms);
     const int budget = 220 * 1024 - P.cb1_bytes - P.cb2_bytes - (TP + WARPS * TP) * 4;
     const int per_row = (WARPS * TP * 8 + 8 * TP) * 4;

@@ -673,18 +673,6 @@ struct GemmPlan {
     long long ws_bytes, off_flags, off_bterm, off_xs;
 };
 
-int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-        else return 148;
-    }
-    return n;
-}
-
 size_t gemm_smem_bytes(int cb2_bytes)
 {
     return 1024 + (size_t)A_STAGES * A_STAGE_BYTES + (size_t)B_STAGES * B_STAGE_BYTES + cb2_bytes +
@@ -694,7 +682,7 @@ size_t gemm_smem_bytes(int cb2_bytes)
 GemmPlan plan_gemm(const LayerView &L, int B)
 {
     GemmPlan p;
-    int workers = sm_count();
+    int workers = device_sm_count();
     p.cb2_rep = (L.k2 > 0 && L.k2 <= 256) ? 1 : 0;
     p.cb2_bytes = L.k2 ? L.k2 * 16 * (p.cb2_rep ? CB2_REPLICAS : 1) : 0;
     p.tiles_m = ceil_div(L.M, TILE_M);

@@ -172,6 +172,23 @@ int vptq_unpack(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k
     return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 
+int vptq_pack_host(const int32_t *idx, int32_t n_rows, int32_t n_cols, int32_t k, uint8_t *packed)
+{
+    if (n_rows < 0 || n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (n_rows == 0 || n_cols == 0) return VPTQ_OK;
+    if (idx == nullptr || packed == nullptr) return VPTQ_E_NULL;
+    return pack_host(idx, n_rows, n_cols, k, packed) == 0 ? VPTQ_OK : VPTQ_E_INDEX_RANGE;
+}
+
+int vptq_unpack_host(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int32_t k, int32_t *idx)
+{
+    if (n_rows < 0 || n_cols < 0 || k < 1 || k > 65536) return VPTQ_E_SHAPE;
+    if (n_rows == 0 || n_cols == 0) return VPTQ_OK;
+    if (idx == nullptr || packed == nullptr) return VPTQ_E_NULL;
+    unpack_host(packed, n_rows, n_cols, k, idx);
+    return VPTQ_OK;
+}
+
 int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, void *W_out, void *stream)
 {
     int rc = check_desc(desc);

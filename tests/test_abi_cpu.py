@@ -140,3 +140,32 @@ def test_assign_path_and_workspace_queries(binding):
     assert b.lib.vptq_assign(None, 4096, 4096, 8, 0x1000, 65536, 0x1000, 0, None, 0, None) == b.E_NULL
     assert b.lib.vptq_assign(0x1000, 4096, 4096, 8, 0x1000, 70000, 0x1000, 0, None, 0, None) == b.E_SHAPE
 
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 5, 16, 100, 256, 257, 4096, 5000, 8192, 40000, 65536])
+def test_host_pack_and_unpack_write_the_oracle_bytes(binding, k):
+    # vptq_pack_host / vptq_unpack_host: plain host code, no CUDA call; byte for byte the oracle's stream
+    b = binding
+    rng = np.random.default_rng(k)
+    for shape in [(1, 1), (3, 7), (5, 41), (4, 257), (2, 4055), (9, 4096)]:
+        for idx in (rng.integers(0, k, size=shape, dtype=np.int32), np.full(shape, k - 1, np.int32),
+                    np.zeros(shape, np.int32)):
+            ref = oracle.pack(idx, k)
+            got = b.vptq_pack_host(idx, k)
+            assert got.shape == ref.shape and np.array_equal(got, ref)
+            # unpack what the ORACLE packed
+            assert np.array_equal(b.vptq_unpack_host(ref, shape[0], shape[1], k), idx)
+
+
+def test_host_pack_argument_errors(binding):
+    b = binding
+    idx = np.array([[0, 1, 5, 2], [7, 0, -1, 3]], np.int32)
+    out = np.full((2, 16), 0xAA, np.uint8)
+    assert b.lib.vptq_pack_host(idx.ctypes.data, 2, 4, 5, out.ctypes.data) == b.E_INDEX_RANGE
+    # the stream is complete all the same, with 0 stored for the three bad entries
+    assert np.array_equal(b.vptq_unpack_host(out, 2, 4, 5), np.array([[0, 1, 0, 2], [0, 0, 0, 3]], np.int32))
+    assert b.lib.vptq_pack_host(None, 2, 4, 5, out.ctypes.data) == b.E_NULL
+    assert b.lib.vptq_pack_host(idx.ctypes.data, 2, 4, 0, out.ctypes.data) == b.E_SHAPE
+    assert b.lib.vptq_pack_host(None, 0, 4, 5, None) == b.OK
+    assert b.lib.vptq_unpack_host(out.ctypes.data, 2, 4, 70000, idx.ctypes.data) == b.E_SHAPE
+    assert b.lib.vptq_unpack_host(None, 2, 4, 5, idx.ctypes.data) == b.E_NULL
