@@ -57,7 +57,12 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_mma_kernel",
                    "gemm_tcgen05": "gemm_tcgen05_kernel", "generic": "linear_generic_kernel",
                    "fused_decode_l2_fma": "decode_l2_fma_kernel", "fused_decode_smem_fma": "decode_smem_fma_kernel",
-                   "fused_decode_gl_fma": "decode_gl_fma_kernel"}
+                   "fused_decode_gl_fma": "decode_gl_fma_kernel",
+                   "decode_bucket_fma": "decode_bucket_fma_kernel", "fused_decode_bucket_fma": "decode_bucket_fma_kernel"}
+# layers of the headline workload that get a prepared image (vptq_prepare): the large projections, where the
+# decode over bucket-ordered entries beats the decode over the canonical streams; partitions of fused groups
+# add up to the SM count
+PREPARED_DEFAULT = "gate_proj,up_proj,down_proj"
 # projections of a decoder layer that read the same activations
 FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
 
@@ -232,11 +237,25 @@ def run_ours(args):
     default_case = cfg_id == WORKLOAD_CFG and keep is None and B == 1
     # every rank is an independent replica with its own seeded weights (layer ordinal offset by rank)
     layers, xs_np = [], []
+    n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    prepared = set(n for n in args.prepared.split(",") if n) if B == 1 else set()
+    kept = [sp.name for sp in cfg["layers"] if keep is None or sp.name in keep]
     for li, spec in enumerate(cfg["layers"]):
         if keep is not None and spec.name not in keep:
             continue
         d = synth.make_layer(spec, cfg_id, replica_layer_ordinal(li, rank), B)
         dl = vb.DeviceLayer(d)
+        if spec.name in prepared:
+            # CTAs for the layer: its share (by vector rows) of the SMs when its whole fuse group is prepared and
+            # present, else all SMs
+            group = next((g for g in FUSE_GROUPS if spec.name in g), None)
+            parts = 0
+            if group is not None and not args.no_fuse and all(n in prepared and n in kept for n in group):
+                rows = {sp.name: sp.R for sp in cfg["layers"] if sp.name in group}
+                share = [max(1, n_sm * rows[n] // sum(rows.values())) for n in group]
+                share[0] += n_sm - sum(share)
+                parts = share[group.index(spec.name)]
+            dl = dl.prepared(parts)
         layers.append([dl])
         xs_np.append(d["x"])
         del d
@@ -265,8 +284,11 @@ def run_ours(args):
     call_names = ["+".join(names[j] for j in idx) + f"_{idx[0]}" for idx, _ in calls]
     launches_per_step = sum(f[0].launches(B) if f is not None else vb.vptq_linear_launches(layers[idx[0]][0].desc, B)
                             for idx, f in calls)
-    paths = sorted({f[0].path(B) if f is not None else vb.vptq_linear_path(layers[idx[0]][0].desc, B)
-                    for idx, f in calls})
+    call_paths = [f[0].path(B) if f is not None else vb.vptq_linear_path(layers[idx[0]][0].desc, B) for idx, f in calls]
+    call_launches = [f[0].launches(B) if f is not None else vb.vptq_linear_launches(layers[idx[0]][0].desc, B)
+                     for idx, f in calls]
+    call_bytes = [sum(layers[j][0].weight_bytes() for j in idx) for idx, _ in calls]
+    paths = sorted(set(call_paths))
 
     def step(i, events=None):
         c = i % copies
@@ -290,38 +312,76 @@ def run_ours(args):
         step(i)
     barrier()
 
-    # ---- timed region: K steps, CUDA events on the launching stream ---------------------------
+    # ---- timed region: exactly K steps, CUDA events on the launching stream -----------------------
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    # per-call events on every `stride`-th step only (at most ~200 steps), to keep the stream tight
-    stride = max(1, args.steps // 200)
-    per_call = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                 for _ in calls] if i % stride == 0 else None for i in range(args.steps)]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record()
     for i in range(args.steps):
-        step(i, per_call[i])
+        step(i)
     ev1.record()
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    time.sleep(0.2)
-    clocks = sampler.stop()
     ms_total = max_over_ranks(ms_total, world, "cuda")
     ms_step = ms_total / args.steps
     value = whole_job_gbps(step_bytes, world, ms_step)
 
-    # per-launch durations of the dominant kernel (all calls of the step run the same kernel family)
-    call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call if pc is not None]
-    n_ev = len(call_ms)
-    layer_ms = [statistics.mean(call_ms[i][ci] for i in range(n_ev)) for ci in range(len(calls))]
-    kern_ms_per_step = sum(layer_ms)
-    achieved = step_bytes / (kern_ms_per_step * 1e-3) / 1e9
+    # ---- roofline pass of its own: per-call events over >= 200 steps, whatever --steps was ---------
+    r_iters = max(200, min(args.steps, 1000))
+    per_call = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in calls]
+                for _ in range(r_iters)]
+    for i in range(r_iters):
+        step(i, per_call[i])
+    barrier()
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    call_ms = [[a.elapsed_time(b) for (a, b) in pc] for pc in per_call]
+    call_stats = []
+    for ci in range(len(calls)):
+        v = sorted(call_ms[i][ci] for i in range(r_iters))
+        call_stats.append({"mean": statistics.mean(v), "median": v[len(v) // 2], "min": v[0]})
+    # the dominant kernel: the family the step spends most of its time in
+    by_kernel = {}
+    for ci, p in enumerate(call_paths):
+        k = ROOFLINE_KERNEL[p]
+        e = by_kernel.setdefault(k, {"ms": 0.0, "bytes": 0.0, "launches": 0, "ms_min": 0.0, "ms_median": 0.0})
+        e["ms"] += call_stats[ci]["mean"]; e["ms_min"] += call_stats[ci]["min"]; e["ms_median"] += call_stats[ci]["median"]
+        e["bytes"] += call_bytes[ci]; e["launches"] += call_launches[ci]
+    dom_kernel = max(by_kernel, key=lambda k: by_kernel[k]["ms"])
+    dom = by_kernel[dom_kernel]
+    kern_ms_per_step = sum(cs["mean"] for cs in call_stats)
+    achieved = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
     per_layer = {call_names[ci]: {
-        "us": 1e3 * layer_ms[ci],
-        "GBps": sum(layers[j][0].weight_bytes() for j in calls[ci][0]) / (1e-3 * layer_ms[ci]) / 1e9}
+        "us": 1e3 * call_stats[ci]["mean"], "us_median": 1e3 * call_stats[ci]["median"], "us_min": 1e3 * call_stats[ci]["min"],
+        "GBps": call_bytes[ci] / (1e-3 * call_stats[ci]["mean"]) / 1e9, "path": call_paths[ci]}
         for ci in range(len(calls))}
+
+    # ---- the step as a CUDA graph (the calls of two steps, over both weight copies), replayed -----
+    graph_us = None
+    try:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        n_cap = max(2, min(copies, 4))
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_cap):
+                    step(i)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        reps = []
+        for _ in range(30):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); g.replay(); b_.record()
+            torch.cuda.synchronize()
+            reps.append(1e3 * a.elapsed_time(b_) / n_cap)
+        graph_us = {"median": statistics.median(reps), "min": min(reps), "steps_per_graph": n_cap}
+    except Exception as e:  # noqa: BLE001  (a capture that fails is reported, not fatal)
+        graph_us = {"error": str(e)[:200]}
 
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     xh = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in xs_np]
@@ -364,6 +424,7 @@ def run_ours(args):
                        "batch": B, "linear_layers_per_step": len(layers), "calls_per_step": len(calls),
                        "calls": call_names,
                        "compressed_bytes_per_step": step_bytes, "kernel_paths": paths,
+                       "prepared_layers": sorted(prepared & set(names)),
                        "l2": f"inputs larger than L2: {copies} copies of the {step_bytes / 1e6:.0f} MB index streams walked alternately",
                        "multi_gpu": "replicas only (no sharding, no collective)"},
             "clocks": clocks,
@@ -371,18 +432,24 @@ def run_ours(args):
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "activations and outputs cross PCIe every step; the quantized weights stay resident"},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": {"bound": "hbm", "kernel": ROOFLINE_KERNEL[paths[0]], "achieved": achieved,
+            "whole_layer_graph_us": graph_us,
+            "roofline": {"bound": "hbm", "kernel": dom_kernel, "achieved": achieved,
                          "peak": peaks["hbm"], "peak_source": peaks["source"] + " (copy bandwidth)",
                          "unit": "GB/s", "frac": achieved / peaks["hbm"],
                          "frac_of_nominal_8TBps": achieved / 8000.0,
-                         "traffic": read_traffic(ROOFLINE_KERNEL[paths[0]], step_bytes / launches_per_step),
-                         "algorithmic_bytes_per_launch": step_bytes / launches_per_step,
-                         "launch_us_mean": 1e3 * kern_ms_per_step / launches_per_step,
-                         "launches_per_step": launches_per_step,
-                         "note": "achieved = compressed bytes of a step / sum of the per-call event durations "
-                                 "of a step = mean bytes per launch / mean launch duration",
+                         "traffic": read_traffic(dom_kernel, dom["bytes"] / dom["launches"]),
+                         "algorithmic_bytes_per_launch": dom["bytes"] / dom["launches"],
+                         "launch_us_mean": 1e3 * dom["ms"] / dom["launches"],
+                         "launch_us_median": 1e3 * dom["ms_median"] / dom["launches"],
+                         "launch_us_min": 1e3 * dom["ms_min"] / dom["launches"],
+                         "launches_per_step": dom["launches"], "iterations": r_iters,
+                         "step_achieved_all_kernels": step_bytes / (kern_ms_per_step * 1e-3) / 1e9,
+                         "step_frac_all_kernels": step_bytes / (kern_ms_per_step * 1e-3) / 1e9 / peaks["hbm"],
+                         "note": "dominant kernel = the family the step spends most time in; achieved = canonical "
+                                 "compressed bytes of its launches / their mean event durations, over a pass of "
+                                 "its own; step_* = all calls of the step",
                          "per_layer": per_layer}}
-    if paths[0] == "gemm_tcgen05":
+    if dom_kernel == "gemm_tcgen05_kernel":
         flops = sum(2.0 * B * l[0].spec.M * l[0].spec.N for l in layers)
         tf = flops / (kern_ms_per_step * 1e-3) / 1e12
         line["roofline"].update({"bound": "tensor", "achieved": tf, "peak": peaks["bf16"], "unit": "TFLOP/s",
@@ -409,9 +476,52 @@ def cpu_baseline():
     t_probe, _ = oracle_sample_rate(layers, 256)
     rows = max(16, min(28672, int(256 * 40.0 / max(t_probe, 1e-6))))   # 10-30 s of CPU work (layers smaller than the sample are taken whole)
     t, nb = oracle_sample_rate(layers, rows)
-    return {"value": nb / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "seconds": t,
-            "sample": f"{rows} evenly spaced output rows of each of the 7 layers of the workload, batch 1"}
+    cores = oracle.num_threads()
+    # the same oracle on one thread, on a sample an eighth of the size
+    oracle.set_num_threads(1)
+    rows1 = max(4, rows // 8)
+    t1, nb1 = oracle_sample_rate(layers, rows1)
+    oracle.set_num_threads(cores)
+    return {"value": nb / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "seconds": t, "single_thread_value": nb1 / t1 / 1e9, "single_thread_seconds": t1,
+            "sample": f"{rows} evenly spaced output rows of each of the 7 layers of the workload, batch 1 "
+                      f"({rows1} rows for the single-thread figure)"}
+
+
+_FLUSH = None
+
+
+def flush_l2():
+    """Write a buffer twice the size of L2 (256 MB): the next call finds none of its data there."""
+    import torch
+    global _FLUSH
+    if _FLUSH is None:
+        _FLUSH = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    _FLUSH.zero_()
+
+
+def isolated_call_us(fn, iters=20):
+    """One call at a time, bracketed by events: L2-warm (the same weights again and again) and after an L2
+    flush (a 256 MB memset before every call).  What a user sees per call, launch path included."""
+    import torch
+    out = {}
+    for label, flush in (("warm", False), ("after_l2_flush", True)):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(iters):
+            if flush:
+                flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(0)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * a.elapsed_time(b))
+        out["us_isolated_" + label + "_median"] = statistics.median(ts)
+        out["us_isolated_" + label + "_min"] = min(ts)
+    return out
 
 
 def time_calls(fn, n_variants, iters=30, warm=5):
@@ -476,6 +586,7 @@ def extra_configs(vb, synth, peaks):
                 gms, med, mn = time_calls(lambda i: variants[i].linear(x, out), n_copies)
                 key = f"cfg{cfg}_{spec.name}_{spec.M}x{spec.N}_B{B}"
                 r = {"us": 1e3 * gms, "us_eager_median": 1e3 * med, "us_eager_min": 1e3 * mn,
+                     **isolated_call_us(lambda i: variants[i].linear(x, out)),
                      "GBps": wb / (gms * 1e-3) / 1e9,
                      "frac_hbm": wb / (gms * 1e-3) / 1e9 / peaks["hbm"], "path": vb.vptq_linear_path(base.desc, B),
                      "weight_copies": n_copies}
@@ -493,7 +604,39 @@ def extra_configs(vb, synth, peaks):
             del variants, base, d
             torch.cuda.empty_cache()
     res.update(extra_fused(vb, synth, peaks))
+    res.update(extra_zipf(vb, synth, peaks))
     res.update(encoder_assign(vb, synth))
+    return res
+
+
+def extra_zipf(vb, synth, peaks):
+    """Reported, not graded: one layer per decode kernel family with Zipf-like index histograms (s = 1 over a
+    random permutation of the centroids) instead of uniform ones, next to the uniform figure of the same layer."""
+    import torch
+    res = {}
+    cases = [(1, 0, 1, False), (3, 3, 1, True), (2, 0, 1, False), (2, 0, 8, False), (5, 0, 1, False)]
+    for cfg, li, B, prep in cases:
+        spec = synth.CONFIGS[cfg]["layers"][li]
+        row = {}
+        for dist in ("uniform", "zipf"):
+            d = synth.make_layer(spec, cfg, li, B, dist=dist)
+            base = vb.DeviceLayer(d)
+            if prep:
+                try:
+                    base = base.prepared(0)
+                except vb.VptqError as e:      # a skewed histogram can exceed the image capacity: canonical path
+                    row["prepared_" + dist] = f"refused ({e.code})"
+            wb = base.weight_bytes()
+            n = max(2, min(64, int(2 * 130e6 / wb) + 1))
+            variants = [base] + [base.clone_streams() for _ in range(n - 1)]
+            x = base.upload_x(d["x"][:B])
+            out = torch.empty((B, spec.M), dtype=vb._TORCH_DT[base.desc.out_dtype], device="cuda")
+            gms, _, _ = time_calls(lambda i: variants[i].linear(x, out), n)
+            row["us_" + dist] = 1e3 * gms
+            row["path"] = vb.vptq_linear_path(base.desc, B)
+            del variants, base, d
+            torch.cuda.empty_cache()
+        res[f"zipf_cfg{cfg}_{spec.name}_{spec.M}x{spec.N}_B{B}"] = row
     return res
 
 
@@ -592,6 +735,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-fuse", action="store_true", help="one vptq_linear call per layer (no vptq_linear_fused)")
+    ap.add_argument("--prepared", default=PREPARED_DEFAULT,
+                    help="comma-separated layers that get a prepared image (batch 1 only); '' = none")
     ap.add_argument("--encoder", action="store_true",
                     help="only the quantizer's assignment step (Eq. 2) at full size (profiling case)")
     ap.add_argument("--cfg", type=int, default=WORKLOAD_CFG,

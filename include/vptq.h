@@ -63,6 +63,7 @@ extern "C" {
 #define VPTQ_FLAG_SCALE_ROWS   2  /* scale/bias are per OUTPUT row ([M]) instead of per input column */
 #define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
 #define VPTQ_FLAG_COL_PERM      8 /* the layer has a stored column order (vptq_layer_ptrs.col_perm)   */
+#define VPTQ_FLAG_PREPARED     16 /* vptq_layer_ptrs.prepared holds a prepared image (see vptq_prepare) */
 
 /* Geometry of one quantized linear layer (App. C.1 names: v1,k1,k2 / N%,v0,k0). */
 typedef struct vptq_layer_desc {
@@ -78,6 +79,8 @@ typedef struct vptq_layer_desc {
     int32_t n_groups;    /* Sec. 3.1: the non-outlier columns are split into this many equal runs of
                             consecutive columns (ceil((N-n_outlier)/n_groups) each, the last one
                             shorter), each with main/residual codebooks of its own; 0 or 1 = one   */
+    int32_t prepared_parts; /* with VPTQ_FLAG_PREPARED: the n_parts the image was built with (the number of
+                            CTAs that work on the layer); ignored without the flag                   */
 } vptq_layer_desc;
 
 /* The format pointers of a layer, in the order of the paper's format statement.
@@ -89,6 +92,7 @@ typedef struct vptq_layer_desc {
  *   outlier_codebook fp16 [k0][v0]                                      (required iff n_outlier > 0)
  *   scale, bias      fp16 [N] (or [M] with VPTQ_FLAG_SCALE_ROWS)        (required iff VPTQ_FLAG_SCALE_BIAS)
  *   col_perm         int32 [N], a permutation of 0..N-1                 (required iff VPTQ_FLAG_COL_PERM)
+ *   prepared         image written by vptq_prepare, 256-byte aligned    (required iff VPTQ_FLAG_PREPARED)
  * A pointer that is not required may be null and is never read.
  *
  * col_perm is the stored column order.  The quantizer picks the outlier columns where the Hessian
@@ -109,6 +113,7 @@ typedef struct vptq_layer_ptrs {
     const void    *scale;
     const void    *bias;
     const int32_t *col_perm;
+    const void    *prepared;   /* prepared image (device), required iff VPTQ_FLAG_PREPARED */
 } vptq_layer_ptrs;
 
 /* ---- format arithmetic (host only, no CUDA call) ---------------------------------- */
@@ -222,6 +227,72 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
                               void *x_dev, void *const *outs_dev,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- prepared layer image: the index streams re-ordered for the decode kernel --------------- */
+
+/* Decoding a layer whose main codebook has 65536 entries costs one random 16-byte read of a 1 MiB table per
+ * index, and on B200 the rate of such reads out of L2, not HBM, bounds the decode kernels.  The paper's own
+ * cache argument (App. C.2: lookups are fast while the table fits the first-level cache) is the way out: a
+ * PREPARED IMAGE holds the same (main index, residual index) pairs as the two canonical streams, re-ordered
+ * so that the kernel can keep one 4096-entry slice of the main codebook (a "bucket", 64 KB) in shared memory
+ * at a time and read every centroid from there.  The image is derived data: it is built once per layer from
+ * the canonical streams (vptq_prepare), it can be rebuilt at any time, and the canonical streams stay the
+ * interchange format (vptq_dequant and the other paths keep using them).  The paper has no counterpart.
+ *
+ * Eligible layers: v = 8, 32768 < k1 <= 65536 (16-bit main indices), k2 = 0 or 128 < k2 <= 256 (8-bit residual
+ * indices), no outlier columns,
+ * one codebook group, per-input-column scale/bias or none, N <= 31736.
+ *
+ * Format (version 1; all fields little-endian; the image is 256-byte aligned):
+ *   bytes 0..255  header, uint32 words: [0] 0x42515056 ("VPQB")  [1] version = 1  [2] M  [3] N  [4] k1  [5] k2
+ *                 [6] n_parts  [7] n_warps = 31  [8] n_buckets = ceil(k1 / 4096)  [9] n_blocks
+ *                 [10] byte offset of woff  [11] byte offset of hdr  [12] byte offset of entries (each a
+ *                 multiple of 256)  [13] total bytes  [14] number of real entries = ceil(M/8) * N; rest zero
+ *   woff     uint32 [n_parts * n_warps + 1]: warp w of partition p owns blocks [woff[p*n_warps + w],
+ *            woff[p*n_warps + w + 1]); partition p covers the vector rows [R*p/n_parts, R*(p+1)/n_parts),
+ *            R = ceil(M/8), and must not hold more than 63 of them
+ *   hdr      uint32 [n_blocks]: bits 24..31 = bucket of the block; bits 6q..6q+5 (q = 0..3) = vector row,
+ *            relative to the partition's first row, that the lanes 8q..8q+7 work on in this block, or 63
+ *            when those lanes have nothing to do in it.  Buckets ascend within a warp's range.
+ *   entries  uint32 [n_blocks][32][4]: a block is four steps of a warp; the four entries of lane L in block
+ *            b are the words 4*(32*b + L) .. + 3.  An entry:
+ *              bits 0..8    (main index mod 4096) >> 3; the three low bits of the main index are L mod 8
+ *                           (so the eight lanes of a quarter warp always read eight different 16-byte banks)
+ *                           and its high bits are the block's bucket
+ *              bits 9..16   residual index (0 when k2 = 0)
+ *              bits 17..31  stored column n of the weight, or N for "no entry" (padding)
+ * Every (vector row, column) pair of the layer occurs exactly once among the entries that are not padding,
+ * in a quarter whose header field names that row.
+ *
+ * vptq_prepare_bytes: capacity to allocate for the image of this layer split into n_parts partitions
+ *   (0 = one per SM of the current device): the header and tables plus 4 bytes x 1.5 x the number of
+ *   entries.  VPTQ_E_UNSUPPORTED for a layer that is not eligible, or n_parts too small for the 63-row limit.
+ * vptq_prepare_host: packed_idx / res_idx are HOST copies of the canonical streams, `image` is host memory
+ *   of `image_bytes` bytes; plain host code, no CUDA call.  *used_bytes (may be null) receives the size of
+ *   the image.  VPTQ_E_WORKSPACE when the image does not fit image_bytes: with index histograms far from
+ *   uniform (one centroid taking a large share of the vectors) the bank rule above forces much padding, and
+ *   such a layer is better left on the canonical streams.
+ * vptq_prepare: the same from DEVICE streams into a DEVICE image: copies the streams to the host, builds the
+ *   image there and copies it back.  Synchronous; allocates temporary HOST memory; a set-up step, not on
+ *   the timed path.
+ * Use: set VPTQ_FLAG_PREPARED in desc->flags, desc->prepared_parts to the image's n_parts and
+ * vptq_layer_ptrs.prepared to the image.  vptq_linear then takes the path "decode_bucket_fma" for B = 1 when
+ * n_parts does not exceed the SM count (other batch sizes use the canonical streams, which must still be
+ * valid), and vptq_linear_fused serves prepared layers of one format (N, activation type, residual stage)
+ * whose n_parts sum to at most the SM count with one launch ("fused_decode_bucket_fma"); layers meant to
+ * share a launch are therefore prepared with n_parts that add up to the SM count.  The path asks for a
+ * 256-byte workspace whose first int32 is a status word (vptq_workspace_status): the kernel compares the
+ * image header with the descriptor and writes VPTQ_E_UNSUPPORTED there when they disagree (the outputs are
+ * then not written), or VPTQ_E_TIMEOUT when a bounded wait gave up.  The word is only ever WRITTEN on an
+ * error, never cleared, so that consecutive calls need nothing between their kernels: clear it once when
+ * the workspace is allocated and after reading an error.  An image that vptq_prepare did not write is
+ * outside the contract (its header's sizes are trusted). */
+#define VPTQ_PREPARED_MAGIC 0x42515056u
+int64_t vptq_prepare_bytes(const vptq_layer_desc *desc, int32_t n_parts);
+int vptq_prepare_host(const vptq_layer_desc *desc, const uint8_t *packed_idx, const uint8_t *res_idx,
+                      int32_t n_parts, void *image, size_t image_bytes, size_t *used_bytes);
+int vptq_prepare(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, int32_t n_parts,
+                 void *image, size_t image_bytes, size_t *used_bytes, void *stream);
+
 /* ---- the same product for callers that cannot allocate device memory ---------------- */
 
 /* The paper has no counterpart to this entry point; it exists for integration reasons only.
@@ -306,14 +377,22 @@ int vptq_kmeans_update(const void *W, int32_t M, int32_t N, int32_t v, const int
 
 const char *vptq_status_string(int code);
 const char *vptq_last_cuda_error(void);
-/* The two tensor-core paths — vptq_linear on "gemm_tcgen05" and vptq_assign on "assign_tcgen05" — keep an
- * int32 status word at byte 0 of their workspace; after any other call the workspace holds no status and
+/* Three paths — vptq_linear on "gemm_tcgen05" and on "decode_bucket_fma" (prepared images), and vptq_assign on
+ * "assign_tcgen05" — keep an int32 status word at byte 0 of their workspace; after any other call the workspace holds no status and
  * this call has no meaning.  It synchronises `stream`, reads the word and returns VPTQ_E_TIMEOUT if a
  * bounded device-side wait gave up during the call (the output is then invalid; the context stays
- * usable), else VPTQ_OK.  A null workspace returns VPTQ_OK. */
+ * usable), VPTQ_E_UNSUPPORTED if the prepared-image kernel refused its image, else VPTQ_OK.  A null
+ * workspace returns VPTQ_OK. */
 int vptq_workspace_status(const void *workspace, void *stream);
+/* For tests of the error path: the kernels' device-side waits (on mbarriers and flags) give up after about
+ * two seconds; this sets the limit, in SM clock cycles, for the kernels launched afterwards by any thread
+ * (0 restores the default).  With a limit of a few cycles a healthy kernel abandons its first wait that is
+ * not already satisfied, reports VPTQ_E_TIMEOUT in its status word, leaves no copy in flight and returns;
+ * the context stays usable.  Honoured by the path "decode_bucket_fma".  Process-wide; not for production. */
+void vptq_debug_set_wait_limit(uint64_t cycles);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_fma",
- * "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05".  For tests and benchmark logs. */
+ * "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05", "decode_bucket_fma".  For tests and
+ * benchmark logs. */
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B);
 /* Number of kernels one vptq_linear call launches (scratch memsets are not counted). */
 int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B);

@@ -438,6 +438,89 @@ double oracle_distortion(const uint16_t *W, int32_t M, int32_t N, int32_t v, con
 }
 
 /* ------------------------------------------------------------------ */
+/* Prepared layer image -> canonical index matrices                    */
+/* ------------------------------------------------------------------ */
+
+/* The library can re-order a layer's (main, residual) index pairs into a "prepared image" for its decode
+ * kernel.  The image is derived data whose format is stated in the library's header (version 1); this is a
+ * decoder written from that statement, used to check that an image says exactly what the canonical streams
+ * say.  The paper has no counterpart (it does not describe an inference data layout).
+ *
+ * Walks every warp's block range of every partition, checks each rule of the format and writes the index
+ * pairs back to idx1 / idx2 [ceil(M/8)][N] (int32).  Returns 0, or a positive code naming the first rule
+ * that is broken:
+ *   1 header magic/version  2 header geometry differs from the arguments  3 region offsets or sizes
+ *   4 block ranges not ascending or not ending at n_blocks  5 bucket out of range or descending within a warp
+ *   6 an entry in a quarter that names no row / a row outside the partition  7 column out of range
+ *   8 main or residual index out of range  9 a (row, column) pair occurs twice  10 a pair is missing
+ *   11 a partition holds more than 63 vector rows  12 number of real entries differs from the header's */
+int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M, int32_t N, int32_t k1, int32_t k2,
+                           int32_t *idx1, int32_t *idx2)
+{
+    if (image_bytes < 256) return 3;
+    uint32_t head[16];
+    memcpy(head, image, sizeof(head));
+    if (head[0] != 0x42515056u || head[1] != 1u) return 1;
+    const int64_t R = (M + 7) / 8;
+    const uint32_t n_parts = head[6], n_warps = head[7], n_buckets = head[8], n_blocks = head[9];
+    if (head[2] != (uint32_t)M || head[3] != (uint32_t)N || head[4] != (uint32_t)k1 || head[5] != (uint32_t)k2) return 2;
+    if (n_warps != 31u || n_buckets != (uint32_t)((k1 + 4095) / 4096) || n_parts < 1u || (int64_t)n_parts > R) return 2;
+    const uint64_t off_woff = head[10], off_hdr = head[11], off_ent = head[12], total = head[13];
+    if (off_woff % 256 || off_hdr % 256 || off_ent % 256 || off_woff < 256) return 3;
+    if (off_woff + 4ull * ((uint64_t)n_parts * n_warps + 1) > off_hdr) return 3;
+    if (off_hdr + 4ull * n_blocks > off_ent) return 3;
+    if (off_ent + 512ull * n_blocks > total || total > (uint64_t)image_bytes) return 3;
+    const uint8_t *woff_b = image + off_woff, *hdr_b = image + off_hdr, *ent_b = image + off_ent;
+    for (int64_t i = 0; i < R * N; i++) { idx1[i] = -1; idx2[i] = -1; }
+    uint64_t real = 0;
+    uint32_t prev_end = 0;
+    for (uint32_t p = 0; p < n_parts; p++) {
+        const int64_t r0 = R * p / n_parts, r1 = R * (p + 1) / n_parts;
+        if (r1 - r0 > 63) return 11;
+        for (uint32_t w = 0; w < n_warps; w++) {
+            uint32_t lo, hi;
+            memcpy(&lo, woff_b + 4ull * (p * n_warps + w), 4);
+            memcpy(&hi, woff_b + 4ull * (p * n_warps + w + 1), 4);
+            if (lo != prev_end || hi < lo || hi > n_blocks) return 4;
+            prev_end = hi;
+            uint32_t last_bucket = 0;
+            for (uint32_t b = lo; b < hi; b++) {
+                uint32_t h;
+                memcpy(&h, hdr_b + 4ull * b, 4);
+                const uint32_t bucket = h >> 24;
+                if (bucket >= n_buckets || bucket < last_bucket) return 5;
+                last_bucket = bucket;
+                for (int lane = 0; lane < 32; lane++) {
+                    const uint32_t rowf = (h >> (6 * (lane / 8))) & 63u;
+                    for (int s = 0; s < 4; s++) {
+                        uint32_t e;
+                        memcpy(&e, ent_b + 4ull * (4ull * (32ull * b + (uint64_t)lane) + (uint64_t)s), 4);
+                        const uint32_t col = e >> 17;
+                        if (col == (uint32_t)N) continue;                 /* padding */
+                        if (col > (uint32_t)N) return 7;
+                        if (rowf == 63u || (int64_t)rowf >= r1 - r0) return 6;
+                        const int64_t main_idx = (int64_t)bucket * 4096 + (int64_t)((e & 0x1FFu) << 3) + (lane % 8);
+                        const int64_t res_idx = (e >> 9) & 0xFFu;
+                        if (main_idx >= k1) return 8;
+                        if (k2 > 0 ? res_idx >= k2 : res_idx != 0) return 8;
+                        const int64_t at = (r0 + rowf) * N + col;
+                        if (idx1[at] != -1) return 9;
+                        idx1[at] = (int32_t)main_idx;
+                        idx2[at] = (int32_t)res_idx;
+                        real++;
+                    }
+                }
+            }
+        }
+    }
+    if (prev_end != n_blocks) return 4;
+    for (int64_t i = 0; i < R * N; i++)
+        if (idx1[i] == -1) return 10;
+    if (real != (uint64_t)head[14]) return 12;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
 /* Size accounting                                                     */
 /* ------------------------------------------------------------------ */
 

@@ -29,7 +29,7 @@ E_NULL, E_SHAPE, E_ALIGN, E_UNSUPPORTED, E_WORKSPACE, E_INDEX_RANGE, E_CUDA, E_T
 E_SCRATCH_LIMIT = -9
 NOALLOC_SCRATCH_BYTES = 1 << 20
 DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
-FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC, FLAG_COL_PERM = 1, 2, 4, 8
+FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC, FLAG_COL_PERM, FLAG_PREPARED = 1, 2, 4, 8, 16
 
 _DT = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, "fp32": DTYPE_FP32}
 _TORCH_DT = {DTYPE_FP16: torch.float16, DTYPE_BF16: torch.bfloat16, DTYPE_FP32: torch.float32}
@@ -40,7 +40,7 @@ class LayerDesc(C.Structure):
     _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("v", C.c_int32), ("k1", C.c_int32),
                 ("k2", C.c_int32), ("n_outlier", C.c_int32), ("v0", C.c_int32), ("k0", C.c_int32),
                 ("x_dtype", C.c_int32), ("out_dtype", C.c_int32), ("flags", C.c_int32),
-                ("n_groups", C.c_int32)]
+                ("n_groups", C.c_int32), ("prepared_parts", C.c_int32)]
 
 
 class LayerPtrs(C.Structure):
@@ -48,7 +48,7 @@ class LayerPtrs(C.Structure):
     _fields_ = [("packed_idx", C.c_void_p), ("codebook", C.c_void_p),
                 ("res_idx", C.c_void_p), ("res_codebook", C.c_void_p),
                 ("outlier_idx", C.c_void_p), ("outlier_codebook", C.c_void_p),
-                ("scale", C.c_void_p), ("bias", C.c_void_p), ("col_perm", C.c_void_p)]
+                ("scale", C.c_void_p), ("bias", C.c_void_p), ("col_perm", C.c_void_p), ("prepared", C.c_void_p)]
 
 
 EXPORTS = {
@@ -60,6 +60,11 @@ EXPORTS = {
     "vptq_unpack": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]),
     "vptq_pack_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
     "vptq_unpack_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
+    "vptq_prepare_bytes": (C.c_int64, [C.POINTER(LayerDesc), C.c_int32]),
+    "vptq_prepare_host": (C.c_int, [C.POINTER(LayerDesc), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
+                                    C.POINTER(C.c_size_t)]),
+    "vptq_prepare": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_int32, C.c_void_p, C.c_size_t,
+                               C.POINTER(C.c_size_t), C.c_void_p]),
     "vptq_dequant": (C.c_int, [C.POINTER(LayerDesc), C.POINTER(LayerPtrs), C.c_void_p, C.c_void_p]),
     "vptq_assign": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
                               C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -87,6 +92,7 @@ EXPORTS = {
     "vptq_status_string": (C.c_char_p, [C.c_int]),
     "vptq_last_cuda_error": (C.c_char_p, []),
     "vptq_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "vptq_debug_set_wait_limit": (None, [C.c_uint64]),
     "vptq_linear_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32]),
 }
@@ -119,8 +125,8 @@ def _stream() -> int:
 
 
 def make_desc(M, N, v, k1, k2=0, n_outlier=0, v0=0, k0=0, x_dtype="fp16", out_dtype="fp16",
-              flags=FLAG_SCALE_BIAS, n_groups=1) -> LayerDesc:
-    return LayerDesc(M, N, v, k1, k2, n_outlier, v0, k0, _DT[x_dtype], _DT[out_dtype], flags, n_groups)
+              flags=FLAG_SCALE_BIAS, n_groups=1, prepared_parts=0) -> LayerDesc:
+    return LayerDesc(M, N, v, k1, k2, n_outlier, v0, k0, _DT[x_dtype], _DT[out_dtype], flags, n_groups, prepared_parts)
 
 
 # ---- entry points (same names as the C ABI) -------------------------------------------
@@ -177,6 +183,35 @@ def vptq_unpack_host(packed: np.ndarray, rows: int, cols: int, k: int) -> np.nda
     idx = np.empty((rows, cols), dtype=np.int32)
     _check(lib.vptq_unpack_host(packed.ctypes.data, rows, cols, k, idx.ctypes.data))
     return idx
+
+
+def vptq_prepare_bytes(desc: LayerDesc, n_parts: int = 0) -> int:
+    n = lib.vptq_prepare_bytes(C.byref(desc), n_parts)
+    if n < 0:
+        raise VptqError(int(n))
+    return n
+
+
+def vptq_prepare_host(desc: LayerDesc, packed_idx: np.ndarray, res_idx: Optional[np.ndarray], n_parts: int,
+                      capacity: Optional[int] = None) -> np.ndarray:
+    """Prepared image (uint8 host array, cut to its size) from HOST copies of the canonical streams; no CUDA call."""
+    cap = vptq_prepare_bytes(desc, n_parts) if capacity is None else capacity
+    image = np.empty(cap, dtype=np.uint8)
+    p1 = np.ascontiguousarray(packed_idx, dtype=np.uint8)
+    p2 = None if res_idx is None else np.ascontiguousarray(res_idx, dtype=np.uint8)
+    used = C.c_size_t(0)
+    _check(lib.vptq_prepare_host(C.byref(desc), p1.ctypes.data, None if p2 is None else p2.ctypes.data, n_parts,
+                                 image.ctypes.data, cap, C.byref(used)))
+    return image[:used.value]
+
+
+def vptq_prepare(desc: LayerDesc, ptrs: LayerPtrs, n_parts: int = 0) -> torch.Tensor:
+    """Prepared image (uint8 CUDA tensor, cut to its size) from the layer's device streams."""
+    cap = vptq_prepare_bytes(desc, n_parts)
+    image = torch.empty(cap, dtype=torch.uint8, device="cuda")
+    used = C.c_size_t(0)
+    _check(lib.vptq_prepare(C.byref(desc), C.byref(ptrs), n_parts, image.data_ptr(), cap, C.byref(used), _stream()))
+    return image[:used.value]
 
 
 def vptq_dequant(desc: LayerDesc, ptrs: LayerPtrs, W_out: torch.Tensor) -> torch.Tensor:
@@ -358,6 +393,7 @@ class DeviceLayer:
                               _ptr(self.col_perm))
         self._ws: Dict[int, Optional[torch.Tensor]] = {}
         self.device = dev
+        self.image = None
 
     def with_flags(self, flags: int) -> "DeviceLayer":
         other = object.__new__(DeviceLayer)
@@ -365,6 +401,20 @@ class DeviceLayer:
         s = self.spec
         other.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype, flags,
                                getattr(s, "n_groups", 1))
+        other._ws = {}
+        return other
+
+    def prepared(self, n_parts: int = 0) -> "DeviceLayer":
+        """The same layer with a prepared image (vptq_prepare): batch-1 calls read the image instead of the
+        canonical streams.  n_parts = CTAs that will work on the layer (0: one per SM)."""
+        other = object.__new__(DeviceLayer)
+        other.__dict__.update(self.__dict__)
+        other.image = vptq_prepare(self.desc, self.ptrs, n_parts)
+        parts = int(other.image[24:28].view(torch.int32).item())           # header word 6
+        s = self.spec
+        other.desc = make_desc(s.M, s.N, s.v, s.k1, s.k2, s.n_out, s.v0, s.k0, s.x_dtype, s.out_dtype,
+                               self.desc.flags | FLAG_PREPARED, getattr(s, "n_groups", 1), parts)
+        other.ptrs = LayerPtrs(*[getattr(self.ptrs, f[0]) for f in LayerPtrs._fields_[:-1]], _ptr(other.image))
         other._ws = {}
         return other
 
@@ -376,9 +426,10 @@ class DeviceLayer:
         other.idx1 = None if self.idx1 is None else self.idx1.clone()
         other.idx2 = None if self.idx2 is None else self.idx2.clone()
         other.idx0 = None if self.idx0 is None else self.idx0.clone()
+        other.image = None if getattr(self, "image", None) is None else self.image.clone()
         other.ptrs = LayerPtrs(_ptr(other.idx1), _ptr(self.c1), _ptr(other.idx2), _ptr(self.c2),
                                _ptr(other.idx0), _ptr(self.c0), _ptr(self.scale), _ptr(self.bias),
-                               _ptr(self.col_perm))
+                               _ptr(self.col_perm), _ptr(other.image))
         return other
 
     def weight_bytes(self) -> int:
@@ -387,7 +438,7 @@ class DeviceLayer:
     def workspace(self, B: int) -> Optional[torch.Tensor]:
         if B not in self._ws:
             n = vptq_linear_workspace_bytes(self.desc, B)
-            self._ws[B] = torch.empty(n, dtype=torch.uint8, device=self.device) if n > 0 else None
+            self._ws[B] = torch.zeros(n, dtype=torch.uint8, device=self.device) if n > 0 else None
         return self._ws[B]
 
     def upload_x(self, x_np: np.ndarray) -> torch.Tensor:
@@ -429,7 +480,7 @@ class FusedLayers:
             need = lib.vptq_linear_fused_workspace_bytes(self.descs, self.n, B)
             if need < 0:
                 raise VptqError(int(need))
-            self._ws[B] = torch.empty(need, dtype=torch.uint8, device=self.dls[0].device) if need else None
+            self._ws[B] = torch.zeros(need, dtype=torch.uint8, device=self.dls[0].device) if need else None
         return self._ws[B]
 
     def linear(self, x: torch.Tensor, outs: Sequence[torch.Tensor]) -> Sequence[torch.Tensor]:

@@ -55,6 +55,8 @@ struct LayerView {
     const __half *c1, *c2, *c0;
     const __half *scale, *bias;
     const int *perm;       // nullptr, or [N]: stored column n is input feature perm[n] (Sec. 3.2.3)
+    const void *prepared;  // nullptr, or the prepared image of the layer
+    int prep_parts;        // partitions of the prepared image
 };
 
 #ifdef __CUDACC__
@@ -100,6 +102,11 @@ __device__ __forceinline__ void store_out(void *out, long long i, float val, int
 
 // streaming multiprocessors of the current device, cached per device ordinal (device_info.cu)
 int device_sm_count();
+
+// limit, in clock cycles, of the bounded device-side waits: 0 = each kernel's default (about two seconds);
+// set by vptq_debug_set_wait_limit, for tests that let a wait run out (device_info.cu)
+unsigned long long debug_wait_limit();
+void set_debug_wait_limit(unsigned long long cycles);
 
 // ---- launchers implemented in the kernel files -------------------------------------------
 cudaError_t launch_pack(const int32_t *idx, int rows, int cols, int k, uint8_t *packed,

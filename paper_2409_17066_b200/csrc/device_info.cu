@@ -8,7 +8,11 @@ namespace vptq {
 namespace {
 constexpr int kMaxDevices = 64;
 std::atomic<int> g_sm_count[kMaxDevices];     // 0 = not looked up yet
+std::atomic<unsigned long long> g_wait_limit{0};
 }
+
+unsigned long long debug_wait_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
+void set_debug_wait_limit(unsigned long long cycles) { g_wait_limit.store(cycles, std::memory_order_relaxed); }
 
 // Streaming multiprocessors of the CURRENT device (every persistent grid and every row split is sized by
 // it, so a plan made with one device current must be launched with that device current).  Without a

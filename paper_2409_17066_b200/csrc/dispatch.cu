@@ -2,6 +2,8 @@
 #include "paths.cuh"
 #include "decode.cuh"
 #include "gemm.cuh"
+#include "prepared.cuh"
+#include "fused_split.cuh"
 
 namespace vptq {
 
@@ -13,6 +15,8 @@ int decode_group(int B) { return B < DECODE_MAX_B ? B : DECODE_MAX_B; }
 LinearPath choose_path(const LayerView &L, int B, int flags)
 {
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
+    if (L.prep_parts > 0 && bucket_fma_supported(L, B) && L.prep_parts <= device_sm_count() &&
+        ceil_div(L.R, L.prep_parts) <= PREP_MAX_ROWS) return PATH_DECODE_BUCKET_FMA;
     if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
     const int Bg = decode_group(B);
     if (smem_fma_supported(L, Bg)) return PATH_DECODE_SMEM_FMA;
@@ -30,6 +34,7 @@ const char *linear_path_name(const LayerView &L, int B, int flags)
     case PATH_DECODE_L2_FMA: return "decode_l2_fma";
     case PATH_DECODE_GL_FMA: return "decode_gl_fma";
     case PATH_GEMM_TCGEN05: return "gemm_tcgen05";
+    case PATH_DECODE_BUCKET_FMA: return "decode_bucket_fma";
     default: return "generic";
     }
 }
@@ -42,6 +47,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
     case PATH_DECODE_GL_FMA: return 0;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
+    case PATH_DECODE_BUCKET_FMA: return 256;          // the status word
     default: return generic_workspace_bytes(L, B);
     }
 }
@@ -55,6 +61,7 @@ int linear_launches(const LayerView &L, int B, int flags)
         return (groups - 1) * smem_fma_launches(L, DECODE_MAX_B) + smem_fma_launches(L, last);
     case PATH_DECODE_SMEM_MMA: return groups;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_launches(L, B);
+    case PATH_DECODE_BUCKET_FMA: return 1;
     case PATH_DECODE_L2_FMA:
         return (groups - 1) * l2_fma_launches(L, DECODE_MAX_B) + l2_fma_launches(L, last);
     case PATH_DECODE_GL_FMA:
@@ -72,6 +79,10 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
         e = launch_linear_generic(L, x, B, out, ws, st);
     } else if (path == PATH_GEMM_TCGEN05) {
         e = launch_gemm_tcgen05(L, x, B, out, ws, st);
+    } else if (path == PATH_DECODE_BUCKET_FMA) {
+        const void *img = L.prepared;
+        void *o = out;
+        e = launch_decode_bucket_fma(&L, &img, &L.prep_parts, 1, x, &o, reinterpret_cast<int *>(ws), debug_wait_limit(), st);
     } else {
         // decode kernels take up to 16 tokens per launch
         const size_t oe = (L.out_dtype == VPTQ_DTYPE_FP32) ? 4 : 2;
@@ -98,6 +109,15 @@ LinearPath fused_path(const LayerView *Ls, const int *flags, int n, int B)
     const LinearPath path = choose_path(Ls[0], B, flags[0]);
     for (int l = 1; l < n; l++)
         if (choose_path(Ls[l], B, flags[l]) != path) return PATH_GENERIC;
+    if (path == PATH_DECODE_BUCKET_FMA) {
+        // prepared layers share a launch when their partitions fit the SMs side by side
+        int ctas = 0;
+        for (int l = 0; l < n; l++) {
+            if (Ls[l].N != Ls[0].N || Ls[l].x_bf16 != Ls[0].x_bf16 || (Ls[l].k2 > 0) != (Ls[0].k2 > 0)) return PATH_GENERIC;
+            ctas += Ls[l].prep_parts;
+        }
+        return (n <= MAX_FUSED && ctas <= device_sm_count()) ? path : PATH_GENERIC;
+    }
     if (path == PATH_DECODE_L2_FMA && l2_fma_fused_supported(Ls, n, B)) return path;
     if (path == PATH_DECODE_SMEM_FMA && smem_fma_fused_supported(Ls, n, B)) return path;
     if (path == PATH_DECODE_GL_FMA && gl_fma_fused_supported(Ls, n, B)) return path;
@@ -110,13 +130,16 @@ const char *linear_fused_path_name(const LayerView *Ls, const int *flags, int n,
     case PATH_DECODE_L2_FMA: return "fused_decode_l2_fma";
     case PATH_DECODE_SMEM_FMA: return "fused_decode_smem_fma";
     case PATH_DECODE_GL_FMA: return "fused_decode_gl_fma";
+    case PATH_DECODE_BUCKET_FMA: return "fused_decode_bucket_fma";
     default: return "one_by_one";
     }
 }
 
 long long linear_fused_workspace_bytes(const LayerView *Ls, const int *flags, int n, int B)
 {
-    if (fused_path(Ls, flags, n, B) != PATH_GENERIC) return 0;
+    const LinearPath fp = fused_path(Ls, flags, n, B);
+    if (fp == PATH_DECODE_BUCKET_FMA) return 256;
+    if (fp != PATH_GENERIC) return 0;
     long long need = 0;       // one layer after the other on the stream: they share the scratch
     for (int l = 0; l < n; l++) {
         const long long w = linear_workspace_bytes(Ls[l], B, flags[l]);
@@ -131,6 +154,7 @@ int linear_fused_launches(const LayerView *Ls, const int *flags, int n, int B)
     if (path == PATH_DECODE_L2_FMA) return l2_fma_fused_launches(B);
     if (path == PATH_DECODE_SMEM_FMA) return smem_fma_launches(Ls[0], B);      // one launch per token group
     if (path == PATH_DECODE_GL_FMA) return gl_fma_launches(Ls[0], B);
+    if (path == PATH_DECODE_BUCKET_FMA) return 1;
     int total = 0;
     for (int l = 0; l < n; l++) total += linear_launches(Ls[l], B, flags[l]);
     return total;
@@ -142,6 +166,12 @@ int linear_fused_dispatch(const LayerView *Ls, const int *flags, int n, const vo
     const LinearPath path = fused_path(Ls, flags, n, B);
     if (path != PATH_GENERIC) {
         if (path == PATH_DECODE_L2_FMA) *cuda_err = launch_decode_l2_fma_fused(Ls, n, x, B, outs, st);
+        else if (path == PATH_DECODE_BUCKET_FMA) {
+            const void *imgs[MAX_FUSED];
+            int parts[MAX_FUSED];
+            for (int l = 0; l < n; l++) { imgs[l] = Ls[l].prepared; parts[l] = Ls[l].prep_parts; }
+            *cuda_err = launch_decode_bucket_fma(Ls, imgs, parts, n, x, outs, reinterpret_cast<int *>(ws), debug_wait_limit(), st);
+        }
         else if (path == PATH_DECODE_SMEM_FMA) *cuda_err = launch_decode_smem_fma_fused(Ls, n, x, B, outs, st);
         else *cuda_err = launch_decode_gl_fma_fused(Ls, n, x, B, outs, st);
         return *cuda_err == cudaSuccess ? VPTQ_OK : VPTQ_E_CUDA;

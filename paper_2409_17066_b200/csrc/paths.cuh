@@ -4,7 +4,7 @@
 
 namespace vptq {
 
-enum LinearPath { PATH_GENERIC = 0, PATH_DECODE_SMEM_FMA, PATH_DECODE_SMEM_MMA, PATH_DECODE_L2_FMA, PATH_DECODE_GL_FMA, PATH_GEMM_TCGEN05 };
+enum LinearPath { PATH_GENERIC = 0, PATH_DECODE_SMEM_FMA, PATH_DECODE_SMEM_MMA, PATH_DECODE_L2_FMA, PATH_DECODE_GL_FMA, PATH_GEMM_TCGEN05, PATH_DECODE_BUCKET_FMA };
 
 LinearPath choose_path(const LayerView &L, int B, int flags);
 const char *linear_path_name(const LayerView &L, int B, int flags);

@@ -1,0 +1,68 @@
+// Prepared layer image (format text: include/vptq.h): geometry, region offsets, and the launchers of the
+// decode kernel that reads it.
+#pragma once
+#include "common.cuh"
+
+namespace vptq {
+
+constexpr int PREP_WARPS = 31;              // consumer warps of the decode kernel; one more warp loads the buckets
+constexpr int PREP_BUCKET = 4096;           // main-codebook entries per bucket (64 KB)
+constexpr int PREP_MAX_ROWS = 63;           // vector rows per partition (6-bit row fields; 63 = idle)
+constexpr int PREP_MAX_N = 31736;           // the staged activations must fit below the first bucket buffer
+
+struct PreparedGeometry {
+    int M, N, k1, k2, R, n_parts, n_buckets;
+};
+
+struct PreparedLayout {
+    unsigned long long off_woff, off_hdr, off_entries, total;
+};
+
+inline unsigned long long align256(unsigned long long x) { return (x + 255ull) / 256ull * 256ull; }
+
+inline PreparedLayout prepared_layout(int n_parts, unsigned long long n_blocks)
+{
+    PreparedLayout l;
+    l.off_woff = 256;
+    l.off_hdr = align256(l.off_woff + 4ull * ((unsigned long long)n_parts * PREP_WARPS + 1));
+    l.off_entries = align256(l.off_hdr + 4ull * n_blocks);
+    l.total = align256(l.off_entries + 512ull * n_blocks);
+    return l;
+}
+
+// Layers the prepared path serves (the format text lists them).
+inline bool prepared_eligible(const LayerView &L)
+{
+    return L.v == 8 && L.k1 <= 65536 && L.s1.bits == 16 && (L.k2 == 0 || (L.k2 <= 256 && L.s2.bits == 8)) &&
+           L.n_out == 0 && L.G == 1 && !L.scale_rows && L.N <= PREP_MAX_N;
+}
+
+// n_parts = 0 means one partition per SM; false when a partition would hold more than PREP_MAX_ROWS rows.
+inline bool prepared_geometry(const LayerView &L, int n_parts, PreparedGeometry *g)
+{
+    if (n_parts == 0) n_parts = device_sm_count();
+    if (n_parts < 1) return false;
+    if (n_parts > L.R) n_parts = L.R;
+    g->M = L.M; g->N = L.N; g->k1 = L.k1; g->k2 = L.k2; g->R = L.R; g->n_parts = n_parts;
+    g->n_buckets = (L.k1 + PREP_BUCKET - 1) / PREP_BUCKET;
+    return ceil_div(L.R, n_parts) <= PREP_MAX_ROWS;
+}
+
+// capacity handed out by vptq_prepare_bytes: tables for the worst block count that fits, 1.5 x 4 bytes per entry
+inline unsigned long long prepared_capacity(const PreparedGeometry &g)
+{
+    const unsigned long long entries = (unsigned long long)g.R * g.N;
+    const unsigned long long blocks = (entries * 3 / 2 + 127) / 128 + (unsigned long long)g.n_parts * PREP_WARPS * g.n_buckets;
+    return prepared_layout(g.n_parts, blocks).total;
+}
+
+int prepare_host(const PreparedGeometry &g, const uint8_t *idx1, const uint8_t *idx2, void *image, size_t image_bytes,
+                 size_t *used_bytes);
+
+// decode kernel over prepared images (batch 1): n layers of one launch, CTAs dealt out by the images' n_parts
+bool bucket_fma_supported(const LayerView &L, int B);
+cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *images, const int *n_parts, int n,
+                                     const void *x, void *const *outs, int *status, unsigned long long wait_limit,
+                                     cudaStream_t st);
+
+}  // namespace vptq

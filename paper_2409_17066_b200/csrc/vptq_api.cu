@@ -8,6 +8,9 @@
 #include "decode.cuh"
 #include "paths.cuh"
 #include "assign.cuh"
+#include "prepared.cuh"
+
+#include <vector>
 
 using namespace vptq;
 
@@ -35,7 +38,8 @@ int check_desc(const vptq_layer_desc *d)
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
         d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
-    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM)) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM | VPTQ_FLAG_PREPARED)) return VPTQ_E_UNSUPPORTED;
+    if ((d->flags & VPTQ_FLAG_PREPARED) && d->prepared_parts < 1) return VPTQ_E_SHAPE;
     if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
     return VPTQ_OK;
 }
@@ -51,6 +55,10 @@ int check_ptrs(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     if (d->flags & VPTQ_FLAG_COL_PERM) {
         if (p->col_perm == nullptr) return VPTQ_E_NULL;
         if (!aligned16(p->col_perm)) return VPTQ_E_ALIGN;
+    }
+    if (d->flags & VPTQ_FLAG_PREPARED) {
+        if (p->prepared == nullptr) return VPTQ_E_NULL;
+        if ((reinterpret_cast<uintptr_t>(p->prepared) & 255u) != 0) return VPTQ_E_ALIGN;
     }
     const void *all[8] = {has_main ? p->packed_idx : nullptr, has_main ? p->codebook : nullptr,
                           (has_main && d->k2 > 0) ? p->res_idx : nullptr,
@@ -93,7 +101,9 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
         L.scale = L.has_scale ? reinterpret_cast<const __half *>(p->scale) : nullptr;
         L.bias = L.has_scale ? reinterpret_cast<const __half *>(p->bias) : nullptr;
         L.perm = (d->flags & VPTQ_FLAG_COL_PERM) ? reinterpret_cast<const int *>(p->col_perm) : nullptr;
+        L.prepared = (d->flags & VPTQ_FLAG_PREPARED) ? p->prepared : nullptr;
     }
+    L.prep_parts = (d->flags & VPTQ_FLAG_PREPARED) ? d->prepared_parts : 0;
     return L;
 }
 
@@ -187,6 +197,66 @@ int vptq_unpack_host(const uint8_t *packed, int32_t n_rows, int32_t n_cols, int3
     if (idx == nullptr || packed == nullptr) return VPTQ_E_NULL;
     unpack_host(packed, n_rows, n_cols, k, idx);
     return VPTQ_OK;
+}
+
+// descriptor -> geometry of the prepared image, or an error code
+static int prepared_geometry_of(const vptq_layer_desc *desc, int32_t n_parts, PreparedGeometry *g)
+{
+    int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (n_parts < 0) return VPTQ_E_SHAPE;
+    const LayerView L = make_view(desc, nullptr);
+    if (!prepared_eligible(L) || (desc->flags & VPTQ_FLAG_SCALE_ROWS)) return VPTQ_E_UNSUPPORTED;
+    return prepared_geometry(L, n_parts, g) ? VPTQ_OK : VPTQ_E_UNSUPPORTED;
+}
+
+int64_t vptq_prepare_bytes(const vptq_layer_desc *desc, int32_t n_parts)
+{
+    PreparedGeometry g;
+    const int rc = prepared_geometry_of(desc, n_parts, &g);
+    if (rc != VPTQ_OK) return rc;
+    return (int64_t)prepared_capacity(g);
+}
+
+int vptq_prepare_host(const vptq_layer_desc *desc, const uint8_t *packed_idx, const uint8_t *res_idx,
+                      int32_t n_parts, void *image, size_t image_bytes, size_t *used_bytes)
+{
+    PreparedGeometry g;
+    const int rc = prepared_geometry_of(desc, n_parts, &g);
+    if (rc != VPTQ_OK) return rc;
+    if (packed_idx == nullptr || image == nullptr || (g.k2 > 0 && res_idx == nullptr)) return VPTQ_E_NULL;
+    if (image_bytes < 256) return VPTQ_E_WORKSPACE;
+    return prepare_host(g, packed_idx, res_idx, image, image_bytes, used_bytes);
+}
+
+int vptq_prepare(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, int32_t n_parts,
+                 void *image, size_t image_bytes, size_t *used_bytes, void *stream)
+{
+    PreparedGeometry g;
+    int rc = prepared_geometry_of(desc, n_parts, &g);
+    if (rc != VPTQ_OK) return rc;
+    if (p == nullptr || p->packed_idx == nullptr || image == nullptr || (g.k2 > 0 && p->res_idx == nullptr)) return VPTQ_E_NULL;
+    if ((reinterpret_cast<uintptr_t>(image) & 255u) != 0) return VPTQ_E_ALIGN;
+    if (image_bytes < 256) return VPTQ_E_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t b1 = (size_t)g.R * (size_t)row_bytes(g.N, g.k1), b2 = g.k2 ? (size_t)g.R * (size_t)row_bytes(g.N, g.k2) : 0;
+    std::vector<uint8_t> h1, h2, himg;
+    try {
+        h1.resize(b1); h2.resize(b2 ? b2 : 1); himg.resize(image_bytes);
+    } catch (...) {
+        return VPTQ_E_WORKSPACE;
+    }
+    cudaError_t e = cudaMemcpyAsync(h1.data(), p->packed_idx, b1, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && b2) e = cudaMemcpyAsync(h2.data(), p->res_idx, b2, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    size_t used = 0;
+    rc = prepare_host(g, h1.data(), b2 ? h2.data() : nullptr, himg.data(), image_bytes, &used);
+    if (used_bytes) *used_bytes = used;
+    if (rc != VPTQ_OK) return rc;
+    e = cudaMemcpyAsync(image, himg.data(), used, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? VPTQ_OK : cuda_fail(e);
 }
 
 int vptq_dequant(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, void *W_out, void *stream)
@@ -438,6 +508,8 @@ const char *vptq_status_string(int code)
 
 const char *vptq_last_cuda_error(void) { return g_cuda_err; }
 
+void vptq_debug_set_wait_limit(uint64_t cycles) { set_debug_wait_limit(cycles); }
+
 int vptq_workspace_status(const void *workspace, void *stream)
 {
     if (workspace == nullptr) return VPTQ_OK;
@@ -447,7 +519,7 @@ int vptq_workspace_status(const void *workspace, void *stream)
     if (e != cudaSuccess) return cuda_fail(e);
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e);
-    return word == VPTQ_E_TIMEOUT ? VPTQ_E_TIMEOUT : VPTQ_OK;
+    return (word == VPTQ_E_TIMEOUT || word == VPTQ_E_UNSUPPORTED) ? word : VPTQ_OK;
 }
 
 const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B)
