@@ -78,6 +78,13 @@ __device__ __forceinline__ int load_index(const uint8_t *row, int c, int bits)
 
 __device__ __forceinline__ int clamp_index(int i, int k) { return i < k ? i : k - 1; }
 
+// Programmatic dependent launch (the decode kernels of consecutive calls on a stream): a kernel lets the next
+// one start as soon as SMs free up, and waits for the previous one only where it first touches data that the
+// previous one may have written (the activations).  What comes before the wait must read weights only and
+// write nothing outside the CTA.  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Input feature of stored column n.  A list entry outside [0, N) is clamped, as indices are.
 __device__ __forceinline__ int in_col(const LayerView &L, int n)
 {
@@ -107,6 +114,25 @@ int device_sm_count();
 // set by vptq_debug_set_wait_limit, for tests that let a wait run out (device_info.cu)
 unsigned long long debug_wait_limit();
 void set_debug_wait_limit(unsigned long long cycles);
+
+#ifdef __CUDACC__
+// Launch `kernel` as a programmatic dependent of the stream's previous kernel (see pdl_wait above).
+template <typename Params>
+inline cudaError_t launch_dependent(void (*kernel)(Params), int grid, int block, size_t smem, cudaStream_t st, const Params &P)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, P);
+}
+#endif
 
 // ---- launchers implemented in the kernel files -------------------------------------------
 cudaError_t launch_pack(const int32_t *idx, int rows, int cols, int k, uint8_t *packed,

@@ -13,7 +13,14 @@ cudaError_t launch_decode_smem_fma_fused(const LayerView *Ls, int n, const void 
 
 // codebooks in shared memory, ldmatrix gathers + mma.sync (per-output-row scale, all-outlier layers)
 bool smem_mma_supported(const LayerView &L, int B);
-cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st);
+long long smem_mma_workspace_bytes(const LayerView &L, int B);
+cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
+
+// the same family for the common kind of layer (main columns, per-column scale): persistent row-owner grid,
+// activations staged in shared memory in mma A-fragment order, 32 warps (decode_smem_tc.cu)
+bool smem_tc_supported(const LayerView &L, int B);
+long long smem_tc_workspace_bytes(const LayerView &L, int B);
+cudaError_t launch_decode_smem_tc(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
 
 // main codebook in global memory (L2), residual codebook in shared memory, FP32 FMAs
 bool l2_fma_supported(const LayerView &L, int B);

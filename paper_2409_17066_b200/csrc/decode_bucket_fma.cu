@@ -127,7 +127,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // the next kernel of the stream may start its own prologue as soon as SMs free up
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_launch_dependents();
 
     int li = 0;
     while (li + 1 < P.n_layers && (int)blockIdx.x >= P.cta_begin[li + 1]) li++;
@@ -206,7 +206,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     }
 
     // ---- a6: x*s as FP16 by stored column, bias term sum_n x*b; the activations are the previous kernel's ----
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    pdl_wait();
     {
         float bacc = 0.f;
         if ((L.N & 7) == 0 && L.perm == nullptr) {
@@ -396,18 +396,7 @@ cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *ima
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the prologue (barriers, tables, first blocks) runs under the previous kernel's tail
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(BK_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, P);
+    return launch_dependent(kern, grid, BK_THREADS, smem, st, P);
 }
 
 }  // namespace vptq

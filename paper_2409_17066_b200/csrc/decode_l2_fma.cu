@@ -94,6 +94,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
     static_assert(!FUSED || OWNER, "a fused launch hands whole vector rows to CTAs");
     constexpr int THREADS = WARPS * 32;
     extern __shared__ __align__(16) uint8_t smem[];
+    pdl_launch_dependents();
     // the layer this CTA works on, and its place among that layer's CTAs
     int li = 0;
     if (FUSED)
@@ -163,6 +164,8 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
         }
 
         // ---- stage x*s of the slab (FP16) and accumulate the bias term sum_n x*b ----------------------
+        // (the activations may be the previous kernel's output: everything above read weights only)
+        pdl_wait();
         {
             float bacc[TB];
 #pragma unroll
@@ -461,6 +464,8 @@ cudaError_t launch_one(const L2FmaParams &P, const L2Plan &pl, cudaStream_t st)
     cudaError_t e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
+    // balanced mode clears its scratch with a memset in front of the kernel, so there is no kernel to depend on
+    if (OWNER) return launch_dependent(decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED>, pl.grid, WARPS * 32, pl.smem, st, P);
     decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
     return cudaGetLastError();
 }

@@ -128,6 +128,7 @@ decode_smem_fma_kernel(const __grid_constant__ SmemFmaParams P)
 {
     constexpr int THREADS = WARPS * 32;
     extern __shared__ __align__(16) uint8_t smem[];
+    pdl_launch_dependents();
     // the layer this CTA works on, and its place among that layer's CTAs
     int li = 0;
     if (FUSED)
@@ -199,6 +200,8 @@ decode_smem_fma_kernel(const __grid_constant__ SmemFmaParams P)
         }
 
         // ---- stage x*s (FP16): outlier columns once, the slab's main columns; bias term in slab 0 -----
+        // (the activations may be the previous kernel's output: everything above read weights only)
+        pdl_wait();
         {
             float bacc[TB];
 #pragma unroll
@@ -450,8 +453,7 @@ cudaError_t launch_kernel(const SmemFmaParams &P, const SmemFmaPlan &pl, cudaStr
     cudaError_t e = cudaFuncSetAttribute(decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
-    return cudaGetLastError();
+    return launch_dependent(decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>, pl.grid, WARPS * 32, pl.smem, st, P);
 }
 
 template <int TB, int VV, int WARPS>

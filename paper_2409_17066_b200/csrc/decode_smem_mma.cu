@@ -493,8 +493,16 @@ cudaError_t launch_variant(const SmemMmaParams &P, bool perm, int grid, size_t s
 }
 }  // namespace
 
-cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, cudaStream_t st)
+long long smem_mma_workspace_bytes(const LayerView &L, int B)
 {
+    return smem_tc_supported(L, B) ? smem_tc_workspace_bytes(L, B) : 0;
+}
+
+cudaError_t launch_decode_smem_mma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
+{
+    // the common kind of layer goes to the row-owner kernel with shared-memory A fragments; per-row scale and
+    // all-outlier layers stay here
+    if (smem_tc_supported(L, B)) return launch_decode_smem_tc(L, x, B, out, ws, st);
     SmemMmaParams P;
     P.L = L; P.x = x; P.out = out; P.B = B;
     const int NT = B <= 8 ? 1 : 2;

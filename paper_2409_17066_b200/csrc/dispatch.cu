@@ -43,7 +43,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
 {
     switch (choose_path(L, B, flags)) {
     case PATH_DECODE_SMEM_FMA: return 0;
-    case PATH_DECODE_SMEM_MMA: return 0;
+    case PATH_DECODE_SMEM_MMA: return smem_mma_workspace_bytes(L, decode_group(B));
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
     case PATH_DECODE_GL_FMA: return 0;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
@@ -59,7 +59,7 @@ int linear_launches(const LayerView &L, int B, int flags)
     switch (choose_path(L, B, flags)) {
     case PATH_DECODE_SMEM_FMA:
         return (groups - 1) * smem_fma_launches(L, DECODE_MAX_B) + smem_fma_launches(L, last);
-    case PATH_DECODE_SMEM_MMA: return groups;
+    case PATH_DECODE_SMEM_MMA: return groups * (smem_tc_supported(L, decode_group(B)) ? 2 : 1);      // pre-pass + main kernel
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_launches(L, B);
     case PATH_DECODE_BUCKET_FMA: return 1;
     case PATH_DECODE_L2_FMA:
@@ -91,7 +91,7 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
             const void *xg = reinterpret_cast<const uint8_t *>(x) + (size_t)t0 * L.N * 2;
             void *og = reinterpret_cast<uint8_t *>(out) + (size_t)t0 * L.M * oe;
             if (path == PATH_DECODE_SMEM_FMA) e = launch_decode_smem_fma(L, xg, Bg, og, st);
-            else if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, st);
+            else if (path == PATH_DECODE_SMEM_MMA) e = launch_decode_smem_mma(L, xg, Bg, og, ws, st);
             else if (path == PATH_DECODE_GL_FMA) e = launch_decode_gl_fma(L, xg, Bg, og, st);
             else e = launch_decode_l2_fma(L, xg, Bg, og, ws, st);
         }

@@ -56,27 +56,56 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
         for (int b = 0; b < g.n_buckets; b++) {
             int steps = 0;
             for (int c = 0; c < 8; c++) steps = std::max(steps, count[b * 8 + c]);
-            for (int s4 = 0; s4 < steps; s4 += 4) {
-                QuarterBlock q;
-                q.row = (uint32_t)(r - r0);
-                for (int c = 0; c < 8; c++)
-                    for (int s = 0; s < 4; s++)
-                        q.e[c][s] = s4 + s < count[b * 8 + c] ? sorted[(size_t)start[b * 8 + c] + s4 + s] : pad;
-                qb[b].push_back(q);
+            // The order of a lane's entries is free.  It is chosen so that the 32 lanes of a warp step look their
+            // activations up in different shared-memory banks where possible (bank = bits 1..5 of the column):
+            // quarter blocks that will share a warp block are filled together, step by step, each lane taking
+            // an entry of its residue class whose bank no lane of the step has taken yet.
+            const int nq = (steps + 3) / 4;
+            const size_t q_first = qb[b].size();
+            qb[b].resize(q_first + (size_t)nq);
+            int left[8];
+            for (int c = 0; c < 8; c++) left[c] = count[b * 8 + c];
+            for (int lq0 = 0; lq0 < nq;) {
+                int lq1 = lq0 + 1;                                        // quarter blocks [lq0, lq1) share a warp block
+                while (lq1 < nq && (q_first + (size_t)lq1) / 4 == (q_first + (size_t)lq0) / 4) lq1++;
+                for (int lq = lq0; lq < lq1; lq++) qb[b][q_first + (size_t)lq].row = (uint32_t)(r - r0);
+                for (int s = 0; s < 4; s++) {
+                    uint32_t taken = 0;
+                    for (int lq = lq0; lq < lq1; lq++)
+                        for (int c = 0; c < 8; c++) {
+                            uint32_t *list = &sorted[(size_t)start[b * 8 + c]];
+                            uint32_t e = pad;
+                            if (left[c] > 0) {
+                                int pick = 0;
+                                for (int i = 0; i < left[c]; i++)
+                                    if (!((taken >> ((list[i] >> 18) & 31u)) & 1u)) { pick = i; break; }
+                                e = list[pick];
+                                list[pick] = list[--left[c]];
+                                taken |= 1u << ((e >> 18) & 31u);
+                            }
+                            qb[b][q_first + (size_t)lq].e[c][s] = e;
+                        }
+                }
+                lq0 = lq1;
             }
         }
     }
     // A warp block is four consecutive quarter blocks of a bucket's list (the last one filled up with idle
-    // quarters); a bucket's warp blocks are dealt out to the warps evenly, and the warps that get one block
-    // more than the others change from bucket to bucket, so that every warp ends up with about the same work.
+    // quarters).  A bucket's warp blocks go to the warps in order, floor(n / warps) each, and the remainder one
+    // each to the warps that have had the least work so far: the kernel lets a warp run one bucket ahead of
+    // the slowest, so what has to be even is the running total, not every bucket by itself.
     std::vector<std::vector<uint32_t>> w_hdr(PREP_WARPS), w_ent(PREP_WARPS);
+    long long done[PREP_WARPS] = {0};
     for (int b = 0; b < g.n_buckets; b++) {
         const long long Q = (long long)qb[b].size(), nblk = (Q + 3) / 4;
-        const int shift = (int)((7LL * b) % PREP_WARPS);
-        for (int i = 0; i < PREP_WARPS; i++) {
-            const int w = (i + shift) % PREP_WARPS;
-            const long long j0 = nblk * i / PREP_WARPS, j1 = nblk * (i + 1) / PREP_WARPS;
-            for (long long j = j0; j < j1; j++) {
+        long long share[PREP_WARPS];
+        int order[PREP_WARPS];
+        for (int w = 0; w < PREP_WARPS; w++) { share[w] = nblk / PREP_WARPS; order[w] = w; }
+        std::stable_sort(order, order + PREP_WARPS, [&](int a, int c) { return done[a] < done[c]; });
+        for (int i = 0; i < (int)(nblk % PREP_WARPS); i++) share[order[i]]++;
+        long long j = 0;
+        for (int w = 0; w < PREP_WARPS; w++) {
+            for (const long long j1 = j + share[w]; j < j1; j++) {
                 uint32_t h = (uint32_t)b << 24;
                 const size_t base = w_ent[w].size();
                 w_ent[w].resize(base + 128, pad);
@@ -89,6 +118,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
                 }
                 w_hdr[w].push_back(h);
             }
+            done[w] += share[w];
         }
     }
     for (int w = 0; w < PREP_WARPS; w++) {
