@@ -15,6 +15,7 @@ Inputs are seeded and synthetic (paper_2409_17066_b200/synth.py).  Prints ONE JS
 from __future__ import annotations
 
 import argparse
+import ctypes as C
 import json
 import os
 import statistics
@@ -245,7 +246,7 @@ def run_ours(args):
             continue
         d = synth.make_layer(spec, cfg_id, replica_layer_ordinal(li, rank), B)
         dl = vb.DeviceLayer(d)
-        if spec.name in prepared:
+        if spec.name in prepared and vb.lib.vptq_prepare_bytes(C.byref(dl.desc), 0) > 0:      # eligible layers only
             # CTAs for the layer: its share (by vector rows) of the SMs when its whole fuse group is prepared and
             # present, else all SMs
             group = next((g for g in FUSE_GROUPS if spec.name in g), None)

@@ -64,6 +64,8 @@ extern "C" {
 #define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
 #define VPTQ_FLAG_COL_PERM      8 /* the layer has a stored column order (vptq_layer_ptrs.col_perm)   */
 #define VPTQ_FLAG_PREPARED     16 /* vptq_layer_ptrs.prepared holds a prepared image (see vptq_prepare) */
+#define VPTQ_FLAG_CONCURRENT   32 /* the call may share the GPU with other work (other streams, other processes,
+                                     fewer SMs than the device reports): no CTA waits for another CTA of its grid */
 
 /* Geometry of one quantized linear layer (App. C.1 names: v1,k1,k2 / N%,v0,k0). */
 typedef struct vptq_layer_desc {
@@ -181,7 +183,14 @@ int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B);
  * B <= 16 runs the split-K decode kernels; larger B runs the tensor-core path
  * (tcgen05) when the layer qualifies (v = 8, k1 > 8192, x bf16/fp16), otherwise the
  * decode kernels over groups of 16 tokens.  Calls on one stream are ordered; calls
- * on different streams must not share a workspace. */
+ * on different streams must not share a workspace.
+ * The tensor-core path splits the input dimension of some output tiles over CTAs.  With long shares the CTA
+ * that holds a tile's last piece stores it and raises a flag, and the CTAs that hold the other pieces wait for
+ * that flag (bounded: about two seconds, then VPTQ_E_TIMEOUT in the status word) before they add theirs.  That
+ * is only live while every CTA of the grid (one per SM of the current device) is resident at once, i.e. while
+ * the call has the GPU to itself.  A call that may overlap other GPU work — another stream, another process, an
+ * SM limit — must set VPTQ_FLAG_CONCURRENT: the output is then cleared first and every piece is added, and no
+ * CTA waits for another (a few percent slower). */
 int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
                 const vptq_layer_ptrs *p, void *out,
                 void *workspace, size_t workspace_bytes, void *stream);
@@ -390,6 +399,10 @@ int vptq_workspace_status(const void *workspace, void *stream);
  * not already satisfied, reports VPTQ_E_TIMEOUT in its status word, leaves no copy in flight and returns;
  * the context stays usable.  Honoured by the path "decode_bucket_fma".  Process-wide; not for production. */
 void vptq_debug_set_wait_limit(uint64_t cycles);
+/* 1 when the kernels of vptq_linear for (desc, B) let one CTA wait for a flag that another CTA of the same grid
+ * raises, 0 when no CTA waits for another, negative VPTQ_E_* on bad arguments.  Only the batched path does this
+ * (see vptq_linear), and VPTQ_FLAG_CONCURRENT switches it off. */
+int vptq_linear_waits_between_ctas(const vptq_layer_desc *desc, int32_t B);
 /* Name of the kernel family vptq_linear picks for (desc, B): "generic", "decode_smem_fma",
  * "decode_smem_mma", "decode_l2_fma", "decode_gl_fma", "gemm_tcgen05", "decode_bucket_fma".  For tests and
  * benchmark logs. */

@@ -30,6 +30,7 @@ E_SCRATCH_LIMIT = -9
 NOALLOC_SCRATCH_BYTES = 1 << 20
 DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
 FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC, FLAG_COL_PERM, FLAG_PREPARED = 1, 2, 4, 8, 16
+FLAG_CONCURRENT = 32
 
 _DT = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, "fp32": DTYPE_FP32}
 _TORCH_DT = {DTYPE_FP16: torch.float16, DTYPE_BF16: torch.bfloat16, DTYPE_FP32: torch.float32}
@@ -93,6 +94,7 @@ EXPORTS = {
     "vptq_last_cuda_error": (C.c_char_p, []),
     "vptq_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "vptq_debug_set_wait_limit": (None, [C.c_uint64]),
+    "vptq_linear_waits_between_ctas": (C.c_int, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear_path": (C.c_char_p, [C.POINTER(LayerDesc), C.c_int32]),
     "vptq_linear_launches": (C.c_int, [C.POINTER(LayerDesc), C.c_int32]),
 }

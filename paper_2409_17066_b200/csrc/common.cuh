@@ -57,6 +57,7 @@ struct LayerView {
     const int *perm;       // nullptr, or [N]: stored column n is input feature perm[n] (Sec. 3.2.3)
     const void *prepared;  // nullptr, or the prepared image of the layer
     int prep_parts;        // partitions of the prepared image
+    int concurrent;        // the call may share the GPU: no waits between CTAs of a grid
 };
 
 #ifdef __CUDACC__
@@ -77,6 +78,20 @@ __device__ __forceinline__ int load_index(const uint8_t *row, int c, int bits)
 }
 
 __device__ __forceinline__ int clamp_index(int i, int k) { return i < k ? i : k - 1; }
+
+// a0 += x * lo(w), a1 += x * hi(w) with x and the two halves of w in FP16: the mixed-precision fma of sm_100
+// (f16 factors, f32 addend and result; the product of two f16 values is exact in f32, so this is the same
+// arithmetic as converting both factors and using an f32 fma, in a third of the instructions).
+// `hi_x` selects the upper half of xw as x.
+__device__ __forceinline__ void fma_f16x2(float &a0, float &a1, uint32_t xw, bool hi_x, uint32_t w)
+{
+    if (hi_x)
+        asm("{\n\t.reg .b16 xl, xh, lo, hi;\n\tmov.b32 {xl, xh}, %2;\n\tmov.b32 {lo, hi}, %3;\n\t"
+            "fma.rn.f32.f16 %0, xh, lo, %0;\n\tfma.rn.f32.f16 %1, xh, hi, %1;\n\t}" : "+f"(a0), "+f"(a1) : "r"(xw), "r"(w));
+    else
+        asm("{\n\t.reg .b16 xl, xh, lo, hi;\n\tmov.b32 {xl, xh}, %2;\n\tmov.b32 {lo, hi}, %3;\n\t"
+            "fma.rn.f32.f16 %0, xl, lo, %0;\n\tfma.rn.f32.f16 %1, xl, hi, %1;\n\t}" : "+f"(a0), "+f"(a1) : "r"(xw), "r"(w));
+}
 
 // Programmatic dependent launch (the decode kernels of consecutive calls on a stream): a kernel lets the next
 // one start as soon as SMs free up, and waits for the previous one only where it first touches data that the
@@ -115,10 +130,15 @@ int device_sm_count();
 unsigned long long debug_wait_limit();
 void set_debug_wait_limit(unsigned long long cycles);
 
+// true unless the environment variable VPTQ_NO_PDL names this kernel family (or "all"): then the kernel is
+// launched the ordinary way, after the stream's previous kernel has finished (device_info.cu)
+bool pdl_enabled(const char *family);
+
 #ifdef __CUDACC__
 // Launch `kernel` as a programmatic dependent of the stream's previous kernel (see pdl_wait above).
 template <typename Params>
-inline cudaError_t launch_dependent(void (*kernel)(Params), int grid, int block, size_t smem, cudaStream_t st, const Params &P)
+inline cudaError_t launch_dependent(const char *family, void (*kernel)(Params), int grid, int block, size_t smem,
+                                    cudaStream_t st, const Params &P)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -129,7 +149,7 @@ inline cudaError_t launch_dependent(void (*kernel)(Params), int grid, int block,
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled(family) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, P);
 }
 #endif

@@ -396,7 +396,7 @@ cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *ima
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the prologue (barriers, tables, first blocks) runs under the previous kernel's tail
-    return launch_dependent(kern, grid, BK_THREADS, smem, st, P);
+    return launch_dependent("bucket", kern, grid, BK_THREADS, smem, st, P);
 }
 
 }  // namespace vptq

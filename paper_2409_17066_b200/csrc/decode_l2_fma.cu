@@ -54,11 +54,6 @@ struct L2FmaParams {
     unsigned *counters;    // balanced: [ceil(R / RB_ROWS)] scratch, zero on entry
 };
 
-__device__ __forceinline__ float2 h2f(uint32_t w)
-{
-    return __half22float2(*reinterpret_cast<__half2 *>(&w));
-}
-
 // streaming 128-/64-bit loads of the packed index rows: read once, keep them out of L1
 __device__ __forceinline__ uint4 ld_stream16(const void *p)
 {
@@ -290,16 +285,13 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
                         w.x = *reinterpret_cast<uint32_t *>(&a0); w.y = *reinterpret_cast<uint32_t *>(&a1);
                         w.z = *reinterpret_cast<uint32_t *>(&a2); w.w = *reinterpret_cast<uint32_t *>(&a3);
                     }
-                    const float2 c01 = h2f(w.x), c23 = h2f(w.y), c45 = h2f(w.z), c67 = h2f(w.w);
 #pragma unroll
                     for (int t = 0; t < TB; t++) {
                         const uint32_t xw = (s >> 1) == 0 ? xv4[t].x : (s >> 1) == 1 ? xv4[t].y : (s >> 1) == 2 ? xv4[t].z : xv4[t].w;
-                        const float2 xp = h2f(xw);
-                        const float xv = (s & 1) ? xp.y : xp.x;
-                        acc[t][0] += xv * c01.x; acc[t][1] += xv * c01.y;
-                        acc[t][2] += xv * c23.x; acc[t][3] += xv * c23.y;
-                        acc[t][4] += xv * c45.x; acc[t][5] += xv * c45.y;
-                        acc[t][6] += xv * c67.x; acc[t][7] += xv * c67.y;
+                        fma_f16x2(acc[t][0], acc[t][1], xw, (s & 1) != 0, w.x);
+                        fma_f16x2(acc[t][2], acc[t][3], xw, (s & 1) != 0, w.y);
+                        fma_f16x2(acc[t][4], acc[t][5], xw, (s & 1) != 0, w.z);
+                        fma_f16x2(acc[t][6], acc[t][7], xw, (s & 1) != 0, w.w);
                     }
                 }
             }
@@ -464,8 +456,9 @@ cudaError_t launch_one(const L2FmaParams &P, const L2Plan &pl, cudaStream_t st)
     cudaError_t e = cudaFuncSetAttribute(decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    // balanced mode clears its scratch with a memset in front of the kernel, so there is no kernel to depend on
-    if (OWNER) return launch_dependent(decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED>, pl.grid, WARPS * 32, pl.smem, st, P);
+    // Launched the ordinary way: as a programmatic dependent this kernel measured slower back to back (the
+    // 70B-shaped layer 377 us per pass instead of 295 us), although its prologue is short.  It still lets the
+    // kernel after it start early (pdl_launch_dependents above), which is where the gain is.
     decode_l2_fma_kernel<TB, RES, OWNER, WARPS, FUSED><<<pl.grid, WARPS * 32, pl.smem, st>>>(P);
     return cudaGetLastError();
 }

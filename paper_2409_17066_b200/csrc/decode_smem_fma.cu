@@ -340,18 +340,13 @@ decode_smem_fma_kernel(const __grid_constant__ SmemFmaParams P)
                             w.w = *reinterpret_cast<uint32_t *>(&a3);
                         }
                     }
-                    float cj[8];
-                    { const float2 p = h2f(w.x); cj[0] = p.x; cj[1] = p.y; }
-                    { const float2 p = h2f(w.y); cj[2] = p.x; cj[3] = p.y; }
-                    if (VV > 4) { const float2 p = h2f(w.z); cj[4] = p.x; cj[5] = p.y; }
-                    if (VV > 6) { const float2 p = h2f(w.w); cj[6] = p.x; cj[7] = p.y; }
 #pragma unroll
                     for (int t = 0; t < TB; t++) {
                         const uint32_t xw = (s >> 1) == 0 ? xv4[t].x : (s >> 1) == 1 ? xv4[t].y : (s >> 1) == 2 ? xv4[t].z : xv4[t].w;
-                        const float2 xp = h2f(xw);
-                        const float xv = (s & 1) ? xp.y : xp.x;
-#pragma unroll
-                        for (int j = 0; j < VV; j++) acc[t][j] += xv * cj[j];
+                        fma_f16x2(acc[t][0], acc[t][1], xw, (s & 1) != 0, w.x);
+                        fma_f16x2(acc[t][2], acc[t][3], xw, (s & 1) != 0, w.y);
+                        if (VV > 4) fma_f16x2(acc[t][4], acc[t][VV > 4 ? 5 : 0], xw, (s & 1) != 0, w.z);
+                        if (VV > 6) fma_f16x2(acc[t][VV > 6 ? 6 : 0], acc[t][VV > 6 ? 7 : 0], xw, (s & 1) != 0, w.w);
                     }
                 }
             }
@@ -453,7 +448,7 @@ cudaError_t launch_kernel(const SmemFmaParams &P, const SmemFmaPlan &pl, cudaStr
     cudaError_t e = cudaFuncSetAttribute(decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>, pl.grid, WARPS * 32, pl.smem, st, P);
+    return launch_dependent("smem_fma", decode_smem_fma_kernel<TB, VV, RES, WARPS, FUSED>, pl.grid, WARPS * 32, pl.smem, st, P);
 }
 
 template <int TB, int VV, int WARPS>

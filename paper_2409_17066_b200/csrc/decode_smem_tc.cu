@@ -472,12 +472,12 @@ cudaError_t launch_decode_smem_tc(const LayerView &L, const void *x, int B, void
         auto kern = res ? decode_smem_tc_kernel<2, true> : decode_smem_tc_kernel<2, false>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
         if (e != cudaSuccess) return e;
-        return launch_dependent(kern, pl.grid, TC_THREADS, pl.smem, st, P);
+        return launch_dependent("smem_tc", kern, pl.grid, TC_THREADS, pl.smem, st, P);
     }
     auto kern = res ? decode_smem_tc_kernel<1, true> : decode_smem_tc_kernel<1, false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
     if (e != cudaSuccess) return e;
-    return launch_dependent(kern, pl.grid, TC_THREADS, pl.smem, st, P);
+    return launch_dependent("smem_tc", kern, pl.grid, TC_THREADS, pl.smem, st, P);
 }
 
 }  // namespace vptq

@@ -2,6 +2,8 @@
 #include "common.cuh"
 
 #include <atomic>
+#include <stdlib.h>
+#include <string.h>
 
 namespace vptq {
 
@@ -29,6 +31,13 @@ int device_sm_count()
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
     if (dev < kMaxDevices) g_sm_count[dev].store(v, std::memory_order_relaxed);
     return v;
+}
+
+bool pdl_enabled(const char *family)
+{
+    static const char *off = getenv("VPTQ_NO_PDL");          // read once
+    if (off == nullptr || off[0] == 0) return true;
+    return strstr(off, "all") == nullptr && strstr(off, family) == nullptr;
 }
 
 }  // namespace vptq

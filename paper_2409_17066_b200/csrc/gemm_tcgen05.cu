@@ -697,7 +697,8 @@ GemmPlan plan_gemm(const LayerView &L, int B)
     p.any_split = 0;
     for (int c = 1; c < workers; c++)
         if ((groups * c / workers * p.unit_gran) % p.kb_total != 0) p.any_split = 1;
-    p.flag_order = (p.any_split && p.units / workers >= FLAG_ORDER_MIN_SHARE) ? 1 : 0;
+    // flag order makes CTAs wait for one another: only for a call that has the GPU to itself
+    p.flag_order = (p.any_split && p.units / workers >= FLAG_ORDER_MIN_SHARE && !L.concurrent) ? 1 : 0;
     p.smem = gemm_smem_bytes(p.cb2_bytes);
     p.off_flags = WS_STATUS_BYTES;
     p.off_bterm = p.off_flags + ((long long)p.tiles_m * p.tiles_t * 4 + 255) / 256 * 256;
@@ -723,6 +724,8 @@ bool gemm_tcgen05_supported(const LayerView &L, int B)
 long long gemm_tcgen05_workspace_bytes(const LayerView &L, int B) { return plan_gemm(L, B).ws_bytes; }
 
 int gemm_tcgen05_launches(const LayerView &, int) { return 2; }   // pre-pass + GEMM
+
+bool gemm_tcgen05_waits_between_ctas(const LayerView &L, int B) { return plan_gemm(L, B).flag_order != 0; }
 
 cudaError_t launch_gemm_tcgen05(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st)
 {

@@ -9,6 +9,7 @@
 #include "paths.cuh"
 #include "assign.cuh"
 #include "prepared.cuh"
+#include "gemm.cuh"
 
 #include <vector>
 
@@ -38,7 +39,7 @@ int check_desc(const vptq_layer_desc *d)
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
         d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
-    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM | VPTQ_FLAG_PREPARED)) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM | VPTQ_FLAG_PREPARED | VPTQ_FLAG_CONCURRENT)) return VPTQ_E_UNSUPPORTED;
     if ((d->flags & VPTQ_FLAG_PREPARED) && d->prepared_parts < 1) return VPTQ_E_SHAPE;
     if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
     return VPTQ_OK;
@@ -104,6 +105,7 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
         L.prepared = (d->flags & VPTQ_FLAG_PREPARED) ? p->prepared : nullptr;
     }
     L.prep_parts = (d->flags & VPTQ_FLAG_PREPARED) ? d->prepared_parts : 0;
+    L.concurrent = (d->flags & VPTQ_FLAG_CONCURRENT) ? 1 : 0;
     return L;
 }
 
@@ -527,6 +529,15 @@ const char *vptq_linear_path(const vptq_layer_desc *desc, int32_t B)
     if (check_desc(desc) != VPTQ_OK || B <= 0) return "invalid";
     LayerView L = make_view(desc, nullptr);
     return linear_path_name(L, B, desc->flags);
+}
+
+int vptq_linear_waits_between_ctas(const vptq_layer_desc *desc, int32_t B)
+{
+    const int rc = check_desc(desc);
+    if (rc != VPTQ_OK) return rc;
+    if (B <= 0) return VPTQ_E_SHAPE;
+    LayerView L = make_view(desc, nullptr);
+    return choose_path(L, B, desc->flags) == PATH_GEMM_TCGEN05 && gemm_tcgen05_waits_between_ctas(L, B) ? 1 : 0;
 }
 
 int vptq_linear_launches(const vptq_layer_desc *desc, int32_t B)

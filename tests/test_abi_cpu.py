@@ -169,3 +169,25 @@ def test_host_pack_argument_errors(binding):
     assert b.lib.vptq_pack_host(None, 0, 4, 5, None) == b.OK
     assert b.lib.vptq_unpack_host(out.ctypes.data, 2, 4, 70000, idx.ctypes.data) == b.E_SHAPE
     assert b.lib.vptq_unpack_host(None, 2, 4, 5, idx.ctypes.data) == b.E_NULL
+
+
+def test_calls_that_share_the_gpu_never_wait_between_ctas(binding):
+    # the batched path lets CTAs wait for a flag of another CTA only with long shares of k blocks, and never when
+    # the caller says that the call may overlap other GPU work
+    b = binding
+    down = b.make_desc(4096, 14336, 8, 65536, 256, x_dtype="bf16", out_dtype="fp32")
+    assert b.vptq_linear_path(down, 512) == "gemm_tcgen05"
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(down), 512) == 1
+    shared = b.make_desc(4096, 14336, 8, 65536, 256, x_dtype="bf16", out_dtype="fp32",
+                         flags=b.FLAG_SCALE_BIAS | b.FLAG_CONCURRENT)
+    assert b.vptq_linear_path(shared, 512) == "gemm_tcgen05"
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(shared), 512) == 0
+    # two layers prepared for two streams: both descriptors carry the flag, neither plan waits
+    for d in (shared, b.make_desc(14336, 4096, 8, 65536, 256, x_dtype="bf16", out_dtype="fp32",
+                                  flags=b.FLAG_SCALE_BIAS | b.FLAG_CONCURRENT)):
+        assert b.lib.vptq_linear_waits_between_ctas(C.byref(d), 512) == 0
+    # decode paths and whole-tile outputs never wait
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(down), 1) == 0
+    half = b.make_desc(4096, 14336, 8, 65536, 256, x_dtype="bf16", out_dtype="fp16")
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(half), 512) == 0
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(down), 0) == b.E_SHAPE

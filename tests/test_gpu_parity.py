@@ -192,6 +192,24 @@ def test_linear_batched_tcgen05(b, M, N, k2, B, out_dtype):
     assert rel_err(y.float().cpu().numpy(), yg.astype(np.float64)) <= TOL
 
 
+def test_linear_batched_tcgen05_without_waits_between_ctas(b):
+    # VPTQ_FLAG_CONCURRENT: the long-share shape whose split tiles otherwise meet by flag order; cleared output,
+    # every piece added, no CTA waits for another
+    spec = synth.LayerSpec("gc", 1100, 13000, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32")
+    B = 24
+    d = synth.make_layer(spec, 76, 3, B)
+    dl = b.DeviceLayer(d)
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(dl.desc), B) == 1
+    sh = dl.with_flags(dl.desc.flags | b.FLAG_CONCURRENT)
+    assert b.vptq_linear_path(sh.desc, B) == "gemm_tcgen05" and b.lib.vptq_linear_waits_between_ctas(C.byref(sh.desc), B) == 0
+    y_ref = oracle.Layer.from_synth(d).linear(d["x"])
+    x = dl.upload_x(d["x"])
+    for _ in range(2):
+        y = sh.linear(x)
+        assert b.vptq_workspace_status(sh.workspace(B)) == b.OK
+        assert rel_err(y.float().cpu().numpy(), y_ref) <= TOL
+
+
 def test_linear_batched_tcgen05_with_a_stored_column_order(b):
     # Sec. 3.2.3: stored column j is input feature col_perm[j]; the pre-pass gathers the activations
     spec = synth.LayerSpec("gp", 264, 1032, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32", permuted=True)
