@@ -64,6 +64,7 @@ extern "C" {
 #define VPTQ_FLAG_FORCE_GENERIC 4 /* use the plain fallback kernels (for testing them)               */
 #define VPTQ_FLAG_COL_PERM      8 /* the layer has a stored column order (vptq_layer_ptrs.col_perm)   */
 #define VPTQ_FLAG_PREPARED     16 /* vptq_layer_ptrs.prepared holds a prepared image (see vptq_prepare) */
+#define VPTQ_FLAG_DETERMINISTIC 64 /* two calls with the same inputs give bit-identical outputs (see vptq_linear)  */
 #define VPTQ_FLAG_CONCURRENT   32 /* the call may share the GPU with other work (other streams, other processes,
                                      fewer SMs than the device reports): no CTA waits for another CTA of its grid */
 
@@ -190,7 +191,13 @@ int64_t vptq_linear_workspace_bytes(const vptq_layer_desc *desc, int32_t B);
  * is only live while every CTA of the grid (one per SM of the current device) is resident at once, i.e. while
  * the call has the GPU to itself.  A call that may overlap other GPU work — another stream, another process, an
  * SM limit — must set VPTQ_FLAG_CONCURRENT: the output is then cleared first and every piece is added, and no
- * CTA waits for another (a few percent slower). */
+ * CTA waits for another (a few percent slower).
+ * Run-to-run differences: the fast kernels combine partial sums with atomic additions, whose order is not
+ * fixed, so two calls with the same inputs may differ in the last bits (well inside the tolerance).  With
+ * VPTQ_FLAG_DETERMINISTIC every sum is formed in a fixed order: layers on the path "decode_l2_fma" keep their
+ * kernel (row-owner mode, warp partial sums kept apart and added in warp order), the batched path gives every
+ * CTA whole output tiles (no split of the input dimension), prepared images are not used, and every other
+ * layer takes the plain fallback kernel (one warp per output row), which is several times slower. */
 int vptq_linear(const vptq_layer_desc *desc, const void *x, int32_t B,
                 const vptq_layer_ptrs *p, void *out,
                 void *workspace, size_t workspace_bytes, void *stream);

@@ -31,6 +31,7 @@ NOALLOC_SCRATCH_BYTES = 1 << 20
 DTYPE_FP16, DTYPE_BF16, DTYPE_FP32 = 0, 1, 2
 FLAG_SCALE_BIAS, FLAG_SCALE_ROWS, FLAG_FORCE_GENERIC, FLAG_COL_PERM, FLAG_PREPARED = 1, 2, 4, 8, 16
 FLAG_CONCURRENT = 32
+FLAG_DETERMINISTIC = 64
 
 _DT = {"fp16": DTYPE_FP16, "bf16": DTYPE_BF16, "fp32": DTYPE_FP32}
 _TORCH_DT = {DTYPE_FP16: torch.float16, DTYPE_BF16: torch.bfloat16, DTYPE_FP32: torch.float32}

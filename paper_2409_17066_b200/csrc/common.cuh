@@ -58,6 +58,7 @@ struct LayerView {
     const void *prepared;  // nullptr, or the prepared image of the layer
     int prep_parts;        // partitions of the prepared image
     int concurrent;        // the call may share the GPU: no waits between CTAs of a grid
+    int deterministic;     // every sum in a fixed order
 };
 
 #ifdef __CUDACC__

@@ -26,6 +26,8 @@ cudaError_t launch_decode_smem_tc(const LayerView &L, const void *x, int B, void
 bool l2_fma_supported(const LayerView &L, int B);
 long long l2_fma_workspace_bytes(const LayerView &L, int B);
 int l2_fma_launches(const LayerView &L, int B);
+// row-owner mode with its ordered partial sums fits shared memory for this layer (deterministic mode)
+bool l2_fma_deterministic_ok(const LayerView &L, int B);
 cudaError_t launch_decode_l2_fma(const LayerView &L, const void *x, int B, void *out, void *ws, cudaStream_t st);
 // ... several layers that read the same activations in one launch per token group (no scratch)
 bool l2_fma_fused_supported(const LayerView *Ls, int n, int B);

@@ -50,6 +50,8 @@ struct L2FmaParams {
     int chunks_total;      // 256-column chunks of a whole row
     int cb2_replicated;    // 1: [k2][8 replicas][16 B], 0: [k2][16 B]
     int part_floats;       // OWNER: floats of the per-row partial sums
+    int det;               // OWNER: warp partial sums are kept apart and added in warp order (no atomics)
+    int rows_cta;          // OWNER: most vector rows a CTA owns
     float *yacc;           // balanced: [B][M] scratch, zero on entry
     unsigned *counters;    // balanced: [ceil(R / RB_ROWS)] scratch, zero on entry
 };
@@ -105,6 +107,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
     float *red = bterm + 4;                                                          // [WARPS][4]
     uint4 *cb2 = reinterpret_cast<uint4 *>(red + WARPS * 4);
     float *part = reinterpret_cast<float *>(cb2 + (RES ? (size_t)L.k2 * (P.cb2_replicated ? 8 : 1) : 0));
+    float *slots = part + P.part_floats;         // det: [rows_cta + WARPS][TB * 8], slot (row - r0) + warp
 
     // rows of this CTA (OWNER) / rank among the CTAs of its slab (balanced)
     const int r0 = OWNER ? (int)((long long)L.R * bid / gdim) : 0;
@@ -334,7 +337,11 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
             const bool holder = (lane & (dup - 1)) == 0;
             const int t = vi >> 3, j = vi & 7;
             if (OWNER) {
-                if (holder) atomicAdd(part + ((cur_r - r0) * TB + t) * 8 + j, v[0]);
+                if (P.det) {
+                    // a warp meets a row once per slab, and warps meet rows in ascending order: (row, warp) pairs
+                    // have slots of their own at row + warp
+                    if (holder) slots[((cur_r - r0) + warp) * (TB * 8) + t * 8 + j] = v[0];
+                } else if (holder) atomicAdd(part + ((cur_r - r0) * TB + t) * 8 + j, v[0]);
             } else {
                 const int m = cur_r * 8 + j;
                 if (holder && t < P.B && m < L.M) atomicAdd(P.yacc + (long long)t * L.M + m, v[0]);
@@ -365,6 +372,21 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
             done_in_row = 0;
         }
         if (OWNER) __syncthreads();      // the slab's xs is dead; part[] complete after the last slab
+        if (OWNER && P.det) {
+            // one thread per sum adds the slab's warp partial sums in warp order: the warps whose task range
+            // [n_tasks*w/WARPS, n_tasks*(w+1)/WARPS) meets the row's tasks [rho*chunks, (rho+1)*chunks)
+            for (int i = threadIdx.x; i < (r1 - r0) * TB * 8; i += THREADS) {
+                const int rho = i / (TB * 8), e = i % (TB * 8);
+                const long long lo = (long long)rho * chunks, hi = lo + chunks;
+                float a = part[i];
+                for (int w = 0; w < WARPS; w++) {
+                    const long long qa = n_tasks * w / WARPS, qb = n_tasks * (w + 1) / WARPS;
+                    if (qa < hi && qb > lo) a += slots[(rho + w) * (TB * 8) + e];
+                }
+                part[i] = a;
+            }
+            __syncthreads();
+        }
     }
 
     // ---- OWNER: bias term, conversion, store -----------------------------------------------------------
@@ -381,7 +403,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
 }
 
 struct L2Plan {
-    int slab_cols, n_slabs, chunks_total, cb2_rep, grid, owner, part_floats, warps;
+    int slab_cols, n_slabs, chunks_total, cb2_rep, grid, owner, part_floats, warps, det, rows_cta;
     size_t smem;
     long long ws_bytes, off_counters;
     int cta_begin[MAX_FUSED + 1];   // fused launches only
@@ -405,11 +427,14 @@ L2Plan plan_l2(const LayerView &L, int TB)
     const long long t_cta = (long long)rows_cta * (slab / 256);
     const double eff_warp = (double)t_cta / ((double)p.warps * (double)((t_cta + p.warps - 1) / p.warps));
     p.part_floats = rows_cta * TB * 8;
-    p.owner = (eff_cta * eff_warp >= 0.80 && (long long)p.part_floats * 4 <= PART_BUDGET) ? 1 : 0;
+    p.rows_cta = rows_cta;
+    p.det = L.deterministic ? 1 : 0;
+    // a deterministic call takes row-owner mode whatever the balance (the other mode adds by global atomics)
+    p.owner = ((eff_cta * eff_warp >= 0.80 || p.det) && (long long)p.part_floats * 4 <= PART_BUDGET) ? 1 : 0;
     if (!p.owner) p.part_floats = 0;
     p.grid = p.owner ? (L.R < G ? L.R : G) : (G < p.n_slabs ? p.n_slabs : G);
     p.smem = (size_t)TB * slab * 2 + 4 * 4 + (size_t)p.warps * 4 * 4 + (size_t)L.k2 * 16 * (p.cb2_rep ? 8 : 1) +
-             (size_t)p.part_floats * 4;
+             (size_t)p.part_floats * 4 + (p.det && p.owner ? (size_t)(rows_cta + p.warps) * TB * 8 * 4 : 0);
     p.ws_bytes = 0;
     p.off_counters = 0;
     if (!p.owner) {
@@ -473,6 +498,7 @@ cudaError_t launch_group(const LayerView &L, const L2Plan &pl, const void *x, in
     P.x = x; P.B = Bg;
     P.slab_cols = pl.slab_cols; P.n_slabs = pl.n_slabs; P.chunks_total = pl.chunks_total;
     P.cb2_replicated = pl.cb2_rep; P.part_floats = pl.part_floats;
+    P.det = pl.det && pl.owner; P.rows_cta = pl.rows_cta;
     P.yacc = nullptr; P.counters = nullptr;
     if (!pl.owner) {
         P.yacc = reinterpret_cast<float *>(ws);
@@ -511,6 +537,12 @@ bool l2_fma_supported(const LayerView &L, int B)
     if (L.s1.bits != 16) return false;
     if (L.k2 && (L.s2.bits != 8 || L.k2 > 2048)) return false;
     return true;
+}
+
+bool l2_fma_deterministic_ok(const LayerView &L, int B)
+{
+    const L2Plan pl = plan_l2(L, token_group(B));
+    return pl.owner != 0 && pl.smem <= 200 * 1024;
 }
 
 long long l2_fma_workspace_bytes(const LayerView &L, int B)

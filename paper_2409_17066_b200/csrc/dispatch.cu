@@ -15,6 +15,13 @@ int decode_group(int B) { return B < DECODE_MAX_B ? B : DECODE_MAX_B; }
 LinearPath choose_path(const LayerView &L, int B, int flags)
 {
     if (flags & VPTQ_FLAG_FORCE_GENERIC) return PATH_GENERIC;
+    if (L.deterministic) {
+        // fixed summation order: the batched path with whole tiles, the L2 decode kernel in row-owner mode with
+        // ordered warp partial sums, else the plain kernel (one warp per output row)
+        if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
+        if (l2_fma_supported(L, decode_group(B)) && l2_fma_deterministic_ok(L, decode_group(B))) return PATH_DECODE_L2_FMA;
+        return PATH_GENERIC;
+    }
     if (L.prep_parts > 0 && bucket_fma_supported(L, B) && L.prep_parts <= device_sm_count() &&
         ceil_div(L.R, L.prep_parts) <= PREP_MAX_ROWS) return PATH_DECODE_BUCKET_FMA;
     if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
@@ -106,6 +113,8 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
 LinearPath fused_path(const LayerView *Ls, const int *flags, int n, int B)
 {
     if (n < 2 || B > DECODE_MAX_B) return PATH_GENERIC;
+    for (int l = 0; l < n; l++)
+        if (Ls[l].deterministic) return PATH_GENERIC;          // one layer after the other
     const LinearPath path = choose_path(Ls[0], B, flags[0]);
     for (int l = 1; l < n; l++)
         if (choose_path(Ls[l], B, flags[l]) != path) return PATH_GENERIC;

@@ -690,7 +690,8 @@ GemmPlan plan_gemm(const LayerView &L, int B)
     p.kb_total = ceil_div(L.N, TILE_K);
     p.units = (long long)p.tiles_m * p.tiles_t * p.kb_total;
     // the pieces of a split tile meet in an FP32 output by red.add; other output types get whole tiles
-    p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32) ? 1 : p.kb_total;
+    // (and so does a deterministic call: reduce-adds of several pieces arrive in no fixed order)
+    p.unit_gran = (L.out_dtype == VPTQ_DTYPE_FP32 && !L.deterministic) ? 1 : p.kb_total;
     const long long groups = p.units / p.unit_gran;
     if (groups < workers) workers = (int)groups;
     p.grid = workers;

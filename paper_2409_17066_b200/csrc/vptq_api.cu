@@ -39,7 +39,7 @@ int check_desc(const vptq_layer_desc *d)
     if (d->x_dtype != VPTQ_DTYPE_FP16 && d->x_dtype != VPTQ_DTYPE_BF16) return VPTQ_E_UNSUPPORTED;
     if (d->out_dtype != VPTQ_DTYPE_FP16 && d->out_dtype != VPTQ_DTYPE_BF16 &&
         d->out_dtype != VPTQ_DTYPE_FP32) return VPTQ_E_UNSUPPORTED;
-    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM | VPTQ_FLAG_PREPARED | VPTQ_FLAG_CONCURRENT)) return VPTQ_E_UNSUPPORTED;
+    if (d->flags & ~(VPTQ_FLAG_SCALE_BIAS | VPTQ_FLAG_SCALE_ROWS | VPTQ_FLAG_FORCE_GENERIC | VPTQ_FLAG_COL_PERM | VPTQ_FLAG_PREPARED | VPTQ_FLAG_CONCURRENT | VPTQ_FLAG_DETERMINISTIC)) return VPTQ_E_UNSUPPORTED;
     if ((d->flags & VPTQ_FLAG_PREPARED) && d->prepared_parts < 1) return VPTQ_E_SHAPE;
     if ((d->flags & VPTQ_FLAG_SCALE_ROWS) && !(d->flags & VPTQ_FLAG_SCALE_BIAS)) return VPTQ_E_UNSUPPORTED;
     return VPTQ_OK;
@@ -106,6 +106,7 @@ LayerView make_view(const vptq_layer_desc *d, const vptq_layer_ptrs *p)
     }
     L.prep_parts = (d->flags & VPTQ_FLAG_PREPARED) ? d->prepared_parts : 0;
     L.concurrent = (d->flags & VPTQ_FLAG_CONCURRENT) ? 1 : 0;
+    L.deterministic = (d->flags & VPTQ_FLAG_DETERMINISTIC) ? 1 : 0;
     return L;
 }
 

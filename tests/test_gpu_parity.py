@@ -141,6 +141,49 @@ def test_linear_is_repeatable_and_leaves_inputs_alone(b):
     assert rel_err(y2.float().cpu().numpy(), y1.double().cpu().numpy()) <= 1e-3
 
 
+DET_CASES = [
+    # (path a deterministic call takes, spec, batch)
+    ("decode_l2_fma", synth.LayerSpec("d_l2", 1030, 2100, v=8, k1=65536, k2=256), 1),
+    ("decode_l2_fma", synth.LayerSpec("d_l2b", 1200, 4360, v=8, k1=65536, k2=256), 7),      # rows that divide badly over the SMs
+    ("generic", synth.LayerSpec("d_smem", 520, 700, v=6, k1=4096, k2=256, n_out=7, v0=4, k0=4096), 1),
+    ("generic", synth.LayerSpec("d_mma", 520, 700, v=6, k1=4096, k2=256, n_out=7, v0=4, k0=4096), 12),
+    ("generic", synth.LayerSpec("d_gl", 600, 134, v=12, k1=4096, k2=4096, n_out=2, v0=4, k0=8192, n_groups=4), 2),
+    ("gemm_tcgen05", synth.LayerSpec("d_gemm", 264, 4100, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="fp32"), 40),
+]
+
+
+@pytest.mark.parametrize("path,spec,B", DET_CASES, ids=[c[1].name for c in DET_CASES])
+def test_deterministic_calls_repeat_bit_for_bit(b, path, spec, B):
+    # VPTQ_FLAG_DETERMINISTIC: every sum in a fixed order; two calls give identical bits, and the right ones
+    d = synth.make_layer(spec, 83, 1, B)
+    dl = b.DeviceLayer(d)
+    det = dl.with_flags(dl.desc.flags | b.FLAG_DETERMINISTIC)
+    assert b.vptq_linear_path(det.desc, B) == path
+    assert b.lib.vptq_linear_waits_between_ctas(C.byref(det.desc), B) == 0
+    x = dl.upload_x(d["x"])
+    ys = [det.linear(x).clone() for _ in range(4)]
+    for y in ys[1:]:
+        assert torch.equal(y, ys[0])
+    assert rel_err(ys[0].float().cpu().numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+    # and agrees with the fast path to summation order
+    assert rel_err(dl.linear(x).float().cpu().numpy(), ys[0].double().cpu().numpy()) <= TOL
+
+
+def test_deterministic_calls_ignore_prepared_images_and_fused_launches(b):
+    spec = synth.LayerSpec("d_prep", 520, 1030, v=8, k1=65536, k2=256)
+    d = synth.make_layer(spec, 84, 0, 1)
+    dl = b.DeviceLayer(d)
+    pl = dl.prepared(7)
+    det = pl.with_flags(pl.desc.flags | b.FLAG_DETERMINISTIC)
+    det.desc.prepared_parts = pl.desc.prepared_parts
+    assert b.vptq_linear_path(det.desc, 1) == "decode_l2_fma"
+    x = dl.upload_x(d["x"])
+    y1, y2 = det.linear(x).clone(), det.linear(x).clone()
+    assert torch.equal(y1, y2)
+    assert rel_err(y1.float().cpu().numpy(), oracle.Layer.from_synth(d).linear(d["x"])) <= TOL
+    assert b.vptq_linear_fused_path([det.desc, det.desc], 1) == "one_by_one"
+
+
 def test_linear_argument_errors(b):
     spec = synth.small_specs()[0]
     d = synth.make_layer(spec, 75, 0, 1)
