@@ -27,6 +27,7 @@
 // a prologue and a ragged tail each.
 #include "common.cuh"
 #include "decode.cuh"
+#include "index_words.cuh"
 #include "fused_split.cuh"
 
 namespace vptq {
@@ -308,30 +309,7 @@ decode_l2_fma_kernel(const __grid_constant__ L2FmaParams P)
             for (int t = 0; t < TB; t++)
 #pragma unroll
                 for (int j = 0; j < 8; j++) { v[t * 8 + j] = acc[t][j]; acc[t][j] = 0.f; }
-            int vi = 0;            // index of the value this lane ends up holding
-            {
-                int n = NV, o = 16;
-#pragma unroll
-                for (int step = 0; step < 5; step++) {
-                    if (n > 1) {
-                        const bool up = (lane & o) != 0;
-                        const int h = n / 2;
-#pragma unroll
-                        for (int k = 0; k < NV / 2; k++) {
-                            if (k < h) {
-                                float send = up ? v[k] : v[k + h];
-                                float keep = up ? v[k + h] : v[k];
-                                v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                            }
-                        }
-                        vi += up ? h : 0;
-                        n = h;
-                    } else {
-                        v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
-                    }
-                    o >>= 1;
-                }
-            }
+            const int vi = halving_butterfly<NV>(v, lane);     // index of the value this lane ends up holding
             // lanes that hold a distinct value: NV = 8: (lane & 3) == 0, NV = 16: (lane & 1) == 0, NV = 32: all
             constexpr int dup = 32 / NV;
             const bool holder = (lane & (dup - 1)) == 0;

@@ -19,6 +19,7 @@
 // sums meet in shared memory; the epilogue adds the bias term and converts (a7).  No scratch.
 #include "common.cuh"
 #include "decode.cuh"
+#include "index_words.cuh"
 #include "fused_split.cuh"
 
 namespace vptq {
@@ -46,80 +47,6 @@ struct SmemFmaParams {
 __device__ __forceinline__ float2 h2f(uint32_t w)
 {
     return __half22float2(*reinterpret_cast<__half2 *>(&w));
-}
-
-__device__ __forceinline__ uint32_t ld_stream4(const void *p)
-{
-    uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-
-// Raw packed bits of the 8 indices of lane group g (columns 8g..8g+7) of one packed row.
-// Never reads beyond the row: words past row_bytes read as zero.
-__device__ __forceinline__ uint4 load_raw8(const uint8_t *__restrict__ row, long long row_bytes, int g, int cols, int bits)
-{
-    uint4 q = make_uint4(0, 0, 0, 0);
-    if (8 * g >= cols) return q;
-    if (bits == 16) {
-        q = __ldg(reinterpret_cast<const uint4 *>(row) + g);
-    } else if (bits == 8) {
-        const uint2 h = __ldg(reinterpret_cast<const uint2 *>(row) + g);
-        q.x = h.x; q.y = h.y;
-    } else if (bits == 12) {
-        const uint8_t *w = row + 12LL * g;
-        const long long off = 12LL * g;
-        q.x = ld_stream4(w);
-        q.y = (off + 8 <= row_bytes) ? ld_stream4(w + 4) : 0u;
-        q.z = (off + 12 <= row_bytes) ? ld_stream4(w + 8) : 0u;
-    } else {
-        // any other width: decode here, store as eight 16-bit values
-        uint32_t v[8];
-#pragma unroll
-        for (int s = 0; s < 8; s++) v[s] = (8 * g + s < cols) ? (uint32_t)load_index(row, 8 * g + s, bits) : 0u;
-        q.x = v[0] | (v[1] << 16); q.y = v[2] | (v[3] << 16);
-        q.z = v[4] | (v[5] << 16); q.w = v[6] | (v[7] << 16);
-    }
-    return q;
-}
-
-// Raw bits -> eight indices as 16-bit pairs in 4 words, clamped to k-1.
-__device__ __forceinline__ void decode8(uint4 q, int bits, int k, uint32_t (&w)[4])
-{
-    if (bits == 8) {
-        w[0] = __byte_perm(q.x, 0, 0x4140); w[1] = __byte_perm(q.x, 0, 0x4342);
-        w[2] = __byte_perm(q.y, 0, 0x4140); w[3] = __byte_perm(q.y, 0, 0x4342);
-    } else if (bits == 12) {
-        const uint32_t a = q.x, b = q.y, c = q.z;
-        const uint32_t i0 = a & 0xFFFu, i1 = (a >> 12) & 0xFFFu, i2 = __funnelshift_r(a, b, 24) & 0xFFFu;
-        const uint32_t i3 = (b >> 4) & 0xFFFu, i4 = (b >> 16) & 0xFFFu, i5 = __funnelshift_r(b, c, 28) & 0xFFFu;
-        const uint32_t i6 = (c >> 8) & 0xFFFu, i7 = c >> 20;
-        w[0] = i0 | (i1 << 16); w[1] = i2 | (i3 << 16); w[2] = i4 | (i5 << 16); w[3] = i6 | (i7 << 16);
-    } else {
-        w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
-    }
-    const uint32_t lim = (uint32_t)(k - 1) * 0x10001u;
-#pragma unroll
-    for (int i = 0; i < 4; i++) w[i] = __vminu2(w[i], lim);
-}
-
-// One centroid [v] fp16 (dense table, entry e) as a zero-padded 16-byte row.
-__device__ __forceinline__ uint4 load_centroid_row(const __half *__restrict__ tab, int e, int v)
-{
-    if (v == 8) return __ldg(reinterpret_cast<const uint4 *>(tab) + e);
-    uint32_t w[4] = {0, 0, 0, 0};
-    if ((v & 1) == 0) {
-        const uint32_t *p = reinterpret_cast<const uint32_t *>(tab) + (long long)e * (v >> 1);   // tables are 16-byte aligned
-#pragma unroll
-        for (int i = 0; i < 4; i++)
-            if (i < (v >> 1)) w[i] = __ldg(p + i);
-    } else {
-        const uint16_t *p = reinterpret_cast<const uint16_t *>(tab) + (long long)e * v;
-#pragma unroll
-        for (int i = 0; i < 8; i++)
-            if (i < v) w[i >> 1] |= (uint32_t)__ldg(p + i) << (16 * (i & 1));
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 template <int TB, int VV, bool RES, int WARPS, bool FUSED>
@@ -362,31 +289,7 @@ decode_smem_fma_kernel(const __grid_constant__ SmemFmaParams P)
                     v[t * 8 + j] = j < VV ? acc[t][j < VV ? j : 0] : 0.f;
                     if (j < VV) acc[t][j] = 0.f;
                 }
-            int vi = 0;            // index of the first value this lane ends up holding
-            int n = NV;
-            {
-                int o = 16;
-#pragma unroll
-                for (int step = 0; step < 5; step++) {
-                    if (n > 1) {
-                        const bool up = (lane & o) != 0;
-                        const int h = n / 2;
-#pragma unroll
-                        for (int k = 0; k < NV / 2; k++) {
-                            if (k < h) {
-                                const float send = up ? v[k] : v[k + h];
-                                const float keep = up ? v[k + h] : v[k];
-                                v[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                            }
-                        }
-                        vi += up ? h : 0;
-                        n = h;
-                    } else {
-                        v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
-                    }
-                    o >>= 1;
-                }
-            }
+            const int vi = halving_butterfly<NV>(v, lane);     // index of the first value this lane ends up holding
             // NV >= 32: every lane holds NV/32 distinct values; NV < 32: lanes with the low bits clear
             constexpr int KEEP = NV >= 32 ? NV / 32 : 1;
             constexpr int dup = NV >= 32 ? 1 : 32 / NV;

@@ -21,6 +21,7 @@
 // term and converts.
 #include "common.cuh"
 #include "decode.cuh"
+#include "index_words.cuh"
 
 namespace vptq {
 
@@ -59,25 +60,6 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// One centroid [v] fp16 (dense table, entry e) as a zero-padded 16-byte row.
-__device__ __forceinline__ uint4 padded_centroid_row(const __half *__restrict__ tab, int e, int v)
-{
-    if (v == 8) return __ldg(reinterpret_cast<const uint4 *>(tab) + e);
-    uint32_t w[4] = {0, 0, 0, 0};
-    if ((v & 1) == 0) {
-        const uint32_t *p = reinterpret_cast<const uint32_t *>(tab) + (long long)e * (v >> 1);   // tables are 16-byte aligned
-#pragma unroll
-        for (int i = 0; i < 4; i++)
-            if (i < (v >> 1)) w[i] = __ldg(p + i);
-    } else {
-        const uint16_t *p = reinterpret_cast<const uint16_t *>(tab) + (long long)e * v;
-#pragma unroll
-        for (int i = 0; i < 8; i++)
-            if (i < v) w[i >> 1] |= (uint32_t)__ldg(p + i) << (16 * (i & 1));
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-}
-
 // Stage a codebook [k][v] fp16 (dense) into shared memory as [k][8] fp16, zero padded.  The loads of
 // 4 entries are issued before the first store: one L2 round trip per 4 entries, not per entry.
 __device__ void stage_codebook(const __half *__restrict__ src, int k, int v, __half *dst)
@@ -87,7 +69,7 @@ __device__ void stage_codebook(const __half *__restrict__ src, int k, int v, __h
         uint4 row[4];
 #pragma unroll
         for (int u = 0; u < 4; u++)
-            if (e0 + u * THREADS < k) row[u] = padded_centroid_row(src, e0 + u * THREADS, v);
+            if (e0 + u * THREADS < k) row[u] = load_centroid_row(src, e0 + u * THREADS, v);
 #pragma unroll
         for (int u = 0; u < 4; u++)
             if (e0 + u * THREADS < k) d4[e0 + u * THREADS] = row[u];
@@ -174,54 +156,6 @@ __device__ __forceinline__ void load_xs16(const SmemMmaParams &P, int t, int n0,
         }
         hw[i] = *reinterpret_cast<uint32_t *>(&xv);
     }
-}
-
-// Raw packed bits of the 8 indices of lane group g (columns 8g..8g+7) of one packed row.
-__device__ __forceinline__ uint4 load_raw8(const uint8_t *__restrict__ row, long long row_bytes, int g, int cols,
-                                           int bits)
-{
-    uint4 q = make_uint4(0, 0, 0, 0);
-    if (8 * g >= cols) return q;
-    if (bits == 16) {
-        q = __ldg(reinterpret_cast<const uint4 *>(row) + g);
-    } else if (bits == 8) {
-        uint2 h = __ldg(reinterpret_cast<const uint2 *>(row) + g);
-        q.x = h.x; q.y = h.y;
-    } else if (bits == 12) {
-        const uint32_t *w = reinterpret_cast<const uint32_t *>(row) + 3 * g;
-        long long off = 12LL * g;
-        q.x = __ldg(w);
-        q.y = (off + 8 <= row_bytes) ? __ldg(w + 1) : 0u;
-        q.z = (off + 12 <= row_bytes) ? __ldg(w + 2) : 0u;
-    } else {
-        // any other width: decode here, store as eight 16-bit values
-        uint32_t v[8];
-#pragma unroll
-        for (int s = 0; s < 8; s++) v[s] = (8 * g + s < cols) ? (uint32_t)load_index(row, 8 * g + s, bits) : 0u;
-        q.x = v[0] | (v[1] << 16); q.y = v[2] | (v[3] << 16);
-        q.z = v[4] | (v[5] << 16); q.w = v[6] | (v[7] << 16);
-    }
-    return q;
-}
-
-// Raw bits -> eight indices as 16-bit pairs in 4 words, clamped to k-1.
-__device__ __forceinline__ void decode8(uint4 q, int bits, int k, uint32_t (&w)[4])
-{
-    if (bits == 8) {
-        w[0] = __byte_perm(q.x, 0, 0x4140); w[1] = __byte_perm(q.x, 0, 0x4342);
-        w[2] = __byte_perm(q.y, 0, 0x4140); w[3] = __byte_perm(q.y, 0, 0x4342);
-    } else if (bits == 12) {
-        uint32_t a = q.x, b = q.y, c = q.z;
-        uint32_t i0 = a & 0xFFFu, i1 = (a >> 12) & 0xFFFu, i2 = __funnelshift_r(a, b, 24) & 0xFFFu;
-        uint32_t i3 = (b >> 4) & 0xFFFu, i4 = (b >> 16) & 0xFFFu, i5 = __funnelshift_r(b, c, 28) & 0xFFFu;
-        uint32_t i6 = (c >> 8) & 0xFFFu, i7 = c >> 20;
-        w[0] = i0 | (i1 << 16); w[1] = i2 | (i3 << 16); w[2] = i4 | (i5 << 16); w[3] = i6 | (i7 << 16);
-    } else {
-        w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
-    }
-    const uint32_t lim = (uint32_t)(k - 1) * 0x10001u;
-#pragma unroll
-    for (int i = 0; i < 4; i++) w[i] = __vminu2(w[i], lim);
 }
 
 template <int NT, bool PERM>   // NT = 1: up to 8 tokens, NT = 2: up to 16 tokens

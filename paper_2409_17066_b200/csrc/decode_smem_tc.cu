@@ -21,6 +21,7 @@
 // The legacy mma.sync form is deliberate: the B operand is a per-lane gather, not a tile TMA could fetch.
 #include "common.cuh"
 #include "decode.cuh"
+#include "index_words.cuh"
 
 namespace vptq {
 
@@ -60,79 +61,6 @@ __device__ __forceinline__ uint32_t tc_hadd2(uint32_t a, uint32_t b)
     const __half2 r = __hadd2(*reinterpret_cast<const __half2 *>(&a), *reinterpret_cast<const __half2 *>(&b));
     return *reinterpret_cast<const uint32_t *>(&r);
 }
-__device__ __forceinline__ uint32_t tc_ld_stream4(const void *p)
-{
-    uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-
-// One centroid [v] fp16 (dense table, entry e) as a zero-padded 16-byte row.
-__device__ __forceinline__ uint4 tc_centroid_row(const __half *__restrict__ tab, int e, int v)
-{
-    if (v == 8) return __ldg(reinterpret_cast<const uint4 *>(tab) + e);
-    uint32_t w[4] = {0, 0, 0, 0};
-    if ((v & 1) == 0) {
-        const uint32_t *p = reinterpret_cast<const uint32_t *>(tab) + (long long)e * (v >> 1);
-#pragma unroll
-        for (int i = 0; i < 4; i++)
-            if (i < (v >> 1)) w[i] = __ldg(p + i);
-    } else {
-        const uint16_t *p = reinterpret_cast<const uint16_t *>(tab) + (long long)e * v;
-#pragma unroll
-        for (int i = 0; i < 8; i++)
-            if (i < v) w[i >> 1] |= (uint32_t)__ldg(p + i) << (16 * (i & 1));
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-}
-
-// Raw packed bits of the 8 indices of lane group g (columns 8g..8g+7) of one packed row (a1); never reads
-// beyond the row.  Widths other than 8, 12 and 16 bits are decoded here into eight 16-bit values.
-__device__ __forceinline__ uint4 tc_load_raw8(const uint8_t *__restrict__ row, long long row_bytes, int g, int cols, int bits)
-{
-    uint4 q = make_uint4(0, 0, 0, 0);
-    if (8 * g >= cols) return q;
-    if (bits == 16) {
-        q = __ldg(reinterpret_cast<const uint4 *>(row) + g);
-    } else if (bits == 8) {
-        const uint2 h = __ldg(reinterpret_cast<const uint2 *>(row) + g);
-        q.x = h.x; q.y = h.y;
-    } else if (bits == 12) {
-        const uint8_t *w = row + 12LL * g;
-        const long long off = 12LL * g;
-        q.x = tc_ld_stream4(w);
-        q.y = (off + 8 <= row_bytes) ? tc_ld_stream4(w + 4) : 0u;
-        q.z = (off + 12 <= row_bytes) ? tc_ld_stream4(w + 8) : 0u;
-    } else {
-        uint32_t v[8];
-#pragma unroll
-        for (int s = 0; s < 8; s++) v[s] = (8 * g + s < cols) ? (uint32_t)load_index(row, 8 * g + s, bits) : 0u;
-        q.x = v[0] | (v[1] << 16); q.y = v[2] | (v[3] << 16);
-        q.z = v[4] | (v[5] << 16); q.w = v[6] | (v[7] << 16);
-    }
-    return q;
-}
-
-// Raw bits -> eight indices as 16-bit pairs in 4 words, clamped to k-1.
-__device__ __forceinline__ void tc_decode8(uint4 q, int bits, int k, uint32_t (&w)[4])
-{
-    if (bits == 8) {
-        w[0] = __byte_perm(q.x, 0, 0x4140); w[1] = __byte_perm(q.x, 0, 0x4342);
-        w[2] = __byte_perm(q.y, 0, 0x4140); w[3] = __byte_perm(q.y, 0, 0x4342);
-    } else if (bits == 12) {
-        const uint32_t a = q.x, b = q.y, c = q.z;
-        const uint32_t i0 = a & 0xFFFu, i1 = (a >> 12) & 0xFFFu, i2 = __funnelshift_r(a, b, 24) & 0xFFFu;
-        const uint32_t i3 = (b >> 4) & 0xFFFu, i4 = (b >> 16) & 0xFFFu, i5 = __funnelshift_r(b, c, 28) & 0xFFFu;
-        const uint32_t i6 = (c >> 8) & 0xFFFu, i7 = c >> 20;
-        w[0] = i0 | (i1 << 16); w[1] = i2 | (i3 << 16); w[2] = i4 | (i5 << 16); w[3] = i6 | (i7 << 16);
-    } else {
-        w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
-    }
-    const uint32_t lim = (uint32_t)(k - 1) * 0x10001u;
-#pragma unroll
-    for (int i = 0; i < 4; i++) w[i] = __vminu2(w[i], lim);
-}
-
 // Pre-pass (one small launch per call): x*s of all tokens as FP16, written once in the order in which the main
 // kernel's mma instructions want their A fragments, so that every CTA fetches its slab with plain 16-byte
 // copies instead of re-deriving it; the outlier columns' activations and the bias term sum_n x*b ride along.
@@ -205,14 +133,14 @@ decode_smem_tc_kernel(const __grid_constant__ SmemTcParams P)
         uint4 row[4];
 #pragma unroll
         for (int u = 0; u < 4; u++)
-            if (e0 + u * TC_THREADS < L.k1) row[u] = tc_centroid_row(L.c1, e0 + u * TC_THREADS, L.v);
+            if (e0 + u * TC_THREADS < L.k1) row[u] = load_centroid_row(L.c1, e0 + u * TC_THREADS, L.v);
 #pragma unroll
         for (int u = 0; u < 4; u++)
             if (e0 + u * TC_THREADS < L.k1) cb1[e0 + u * TC_THREADS] = row[u];
     }
     if (RES) {
         const int n2 = P.cb2_replicated ? L.k2 * 8 : L.k2, sh = P.cb2_replicated ? 3 : 0;
-        for (int i = threadIdx.x; i < n2; i += TC_THREADS) cb2[i] = tc_centroid_row(L.c2, i >> sh, L.v);
+        for (int i = threadIdx.x; i < n2; i += TC_THREADS) cb2[i] = load_centroid_row(L.c2, i >> sh, L.v);
     }
     for (int i = threadIdx.x; i < P.rows_cta * TP * 8; i += TC_THREADS) part[i] = 0.f;
     if (threadIdx.x < TP) tok[threadIdx.x] = 0.f;
@@ -246,8 +174,8 @@ decode_smem_tc_kernel(const __grid_constant__ SmemTcParams P)
             raw1[d] = make_uint4(0, 0, 0, 0); raw2[d] = make_uint4(0, 0, 0, 0);
             if (tq + d < tq_end) {
                 const int grp = (c_begin >> 3) + ch_nxt * 32 + lane;
-                raw1[d] = tc_load_raw8(L.s1.ptr + (long long)r_nxt * L.s1.stride, L.s1.stride, grp, c_end, L.s1.bits);
-                if (RES) raw2[d] = tc_load_raw8(L.s2.ptr + (long long)r_nxt * L.s2.stride, L.s2.stride, grp, c_end, L.s2.bits);
+                raw1[d] = load_raw8(L.s1.ptr + (long long)r_nxt * L.s1.stride, L.s1.stride, grp, c_end, L.s1.bits);
+                if (RES) raw2[d] = load_raw8(L.s2.ptr + (long long)r_nxt * L.s2.stride, L.s2.stride, grp, c_end, L.s2.bits);
                 if (++ch_nxt == chunks) { ch_nxt = 0; r_nxt++; }
             }
         }
@@ -286,7 +214,7 @@ decode_smem_tc_kernel(const __grid_constant__ SmemTcParams P)
                 for (int nb = 0; nb < L.n_out; nb += 32) {
                     uint4 cw = make_uint4(0, 0, 0, 0);
                     if (nb + lane < L.n_out)
-                        cw = tc_centroid_row(L.c0, clamp_index(load_index(row0, nb + lane, L.s0.bits), L.k0), L.v0);
+                        cw = load_centroid_row(L.c0, clamp_index(load_index(row0, nb + lane, L.s0.bits), L.k0), L.v0);
                     const int cols = min(32, L.n_out - nb);
                     for (int c = 0; c < cols; c++) {
                         // component oj sits in word oj / 2 (half oj % 2), component oj + 4 two words further
@@ -340,14 +268,14 @@ decode_smem_tc_kernel(const __grid_constant__ SmemTcParams P)
             for (int dd = 0; dd < 2; dd++) {
                 if (tq < tq_end) {
                     uint32_t w1[4], w2[4] = {0, 0, 0, 0};
-                    tc_decode8(raw1[dd], L.s1.bits, L.k1, w1);
-                    if (RES) tc_decode8(raw2[dd], L.s2.bits, L.k2, w2);
+                    decode8(raw1[dd], L.s1.bits, L.k1, w1);
+                    if (RES) decode8(raw2[dd], L.s2.bits, L.k2, w2);
                     const int r = r_cur, ch = ch_cur;
                     if (++ch_cur == chunks) { ch_cur = 0; r_cur++; }
                     if (tq + 2 < tq_end) {
                         const int grp = (c_begin >> 3) + ch_nxt * 32 + lane;
-                        raw1[dd] = tc_load_raw8(L.s1.ptr + (long long)r_nxt * L.s1.stride, L.s1.stride, grp, c_end, L.s1.bits);
-                        if (RES) raw2[dd] = tc_load_raw8(L.s2.ptr + (long long)r_nxt * L.s2.stride, L.s2.stride, grp, c_end, L.s2.bits);
+                        raw1[dd] = load_raw8(L.s1.ptr + (long long)r_nxt * L.s1.stride, L.s1.stride, grp, c_end, L.s1.bits);
+                        if (RES) raw2[dd] = load_raw8(L.s2.ptr + (long long)r_nxt * L.s2.stride, L.s2.stride, grp, c_end, L.s2.bits);
                         if (++ch_nxt == chunks) { ch_nxt = 0; r_nxt++; }
                     }
                     if (r != cur_r) { flush(); cur_r = r; }
