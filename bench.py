@@ -47,17 +47,19 @@ def read_peaks():
 # in proportion to the packed index streams, so it is scaled by the bytes a launch processes).
 # An entry is removed (-> null in the output) when its kernel changes after the capture.
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
+    # kernel: (ratio, source file of the kernel, first 12 hex digits of its SHA-1 when the capture was taken)
     # profiles/decode_l2_fma_kernel_config3_gate_up_fused_B1.md: (178.44 + 3.68) MB DRAM / 178.33 MB algorithmic
-    "decode_l2_fma_kernel": 1.021,
-    # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.95 MB
-    "decode_smem_fma_kernel": 1.003,
+    # (taken before the mixed-precision fma and the ordered partial sums went into the file: null until re-captured)
+    "decode_l2_fma_kernel": (1.021, "decode_l2_fma.cu", "captured-before-later-edits"),
+    # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.95 MB (same remark)
+    "decode_smem_fma_kernel": (1.003, "decode_smem_fma.cu", "captured-before-later-edits"),
     # profiles/decode_smem_tc_kernel_config2_gate_proj_B8.md: 21.46 MB / 19.0 MB (the 0.5 MB fragment image and the
     # pre-pass's traffic included)
-    "decode_smem_tc_kernel": 1.13,
+    "decode_smem_tc_kernel": (1.13, "decode_smem_tc.cu", "ccf102769587"),
     # profiles/decode_bucket_fma_kernel_config3_gate_up_fused_B1.md: (287.97 + 4.20) MB DRAM / 178.33 MB canonical
     # compressed bytes: the kernel reads the prepared image (4 bytes per slot, 21 % padding at N = 8192; the
     # N = 28672 image of down_proj is 1.47 x its canonical bytes, so this overstates that launch by a tenth)
-    "decode_bucket_fma_kernel": 1.638,
+    "decode_bucket_fma_kernel": (1.638, "decode_bucket_fma.cu", "c889edeb5e87"),
 }
 
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_tc_kernel",
@@ -74,9 +76,20 @@ FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
 
 
 def read_traffic(kernel: str, algorithmic_bytes_per_launch: float):
-    """Per-launch DRAM traffic scaled from the committed ncu summary, if one exists."""
-    r = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(kernel)
-    return None if r is None else r * algorithmic_bytes_per_launch
+    """Per-launch DRAM traffic scaled from the committed ncu summary, if one exists AND the kernel's source file is
+    still the one the counters were taken on (else None: a stale figure is worse than none)."""
+    import hashlib
+    entry = NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE.get(kernel)
+    if entry is None:
+        return None
+    ratio, source, digest = entry
+    path = os.path.join(ROOT, "paper_2409_17066_b200", "csrc", source)
+    try:
+        with open(path, "rb") as fh:
+            now = hashlib.sha1(fh.read()).hexdigest()[:12]
+    except OSError:
+        return None
+    return ratio * algorithmic_bytes_per_launch if now == digest else None
 
 
 class ClockSampler:

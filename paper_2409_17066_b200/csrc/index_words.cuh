@@ -30,9 +30,11 @@ __device__ __forceinline__ uint4 load_raw8(const uint8_t *__restrict__ row, long
     } else if (bits == 12) {
         const uint8_t *w = row + 12LL * g;
         const long long off = 12LL * g;
-        q.x = ld_stream4(w);
-        q.y = (off + 8 <= row_bytes) ? ld_stream4(w + 4) : 0u;
-        q.z = (off + 12 <= row_bytes) ? ld_stream4(w + 8) : 0u;
+        // three word loads at a 12-byte lane stride: each touches the same 12 sectors of the warp's 384-byte span,
+        // so they go through L1 (issued back to back, the second and third merge with the first's misses)
+        q.x = __ldg(reinterpret_cast<const uint32_t *>(w));
+        q.y = (off + 8 <= row_bytes) ? __ldg(reinterpret_cast<const uint32_t *>(w + 4)) : 0u;
+        q.z = (off + 12 <= row_bytes) ? __ldg(reinterpret_cast<const uint32_t *>(w + 8)) : 0u;
     } else {
         uint32_t v[8];
 #pragma unroll

@@ -66,3 +66,28 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5, 1, "cpu") == 3.5
     assert bench.whole_job_gbps(2e9, 1, 1.0) == 2000.0
+
+
+def test_bench_traffic_figures_expire_with_the_kernel_source():
+    """bench.py scales DRAM traffic from an ncu capture only while the kernel's source file is byte for byte the
+    one the capture was taken on; any other digest gives None (reported as null)."""
+    import importlib
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if root not in sys.path:
+        sys.path.insert(0, root)
+    bench = importlib.import_module("bench")
+    table = bench.NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE
+    assert bench.read_traffic("no_such_kernel", 1.0) is None
+    for kernel, (ratio, source, digest) in table.items():
+        assert os.path.exists(os.path.join(root, "paper_2409_17066_b200", "csrc", source)), source
+        got = bench.read_traffic(kernel, 1000.0)
+        assert got is None or got == ratio * 1000.0
+    saved = dict(table)
+    try:
+        k = next(iter(table))
+        table[k] = (table[k][0], table[k][1], "000000000000")
+        assert bench.read_traffic(k, 1.0) is None
+    finally:
+        table.clear()
+        table.update(saved)
