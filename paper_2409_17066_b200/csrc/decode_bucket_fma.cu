@@ -26,7 +26,7 @@ namespace vptq {
 namespace {
 
 constexpr int BK_WARPS = PREP_WARPS + 1, BK_THREADS = BK_WARPS * 32;
-constexpr int BK_DEPTH = 3;                                  // blocks in flight per warp
+constexpr int BK_DEPTH = 2;                                  // blocks in flight per warp
 // absolute shared-memory addresses (the window starts with 1 KB the system keeps and the static variables)
 constexpr uint32_t XS_ABS = 2048, TAB_ABS = 65536, CB2_ABS = 196608, PART_ABS = CB2_ABS + 32768,
                    RED_ABS = PART_ABS + 64 * 8 * 4, END_ABS = RED_ABS + BK_WARPS * 4;
