@@ -70,7 +70,7 @@ ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "
 # layers of the headline workload that get a prepared image (vptq_prepare): the large projections, where the
 # decode over bucket-ordered entries beats the decode over the canonical streams; partitions of fused groups
 # add up to the SM count
-PREPARED_DEFAULT = "gate_proj,up_proj,down_proj"
+PREPARED_DEFAULT = "q_proj,k_proj,v_proj,o_proj,gate_proj,up_proj,down_proj"
 # projections of a decoder layer that read the same activations
 FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
 
@@ -271,9 +271,7 @@ def run_ours(args):
             parts = 0
             if group is not None and not args.no_fuse and all(n in prepared and n in kept for n in group):
                 rows = {sp.name: sp.R for sp in cfg["layers"] if sp.name in group}
-                share = [max(1, n_sm * rows[n] // sum(rows.values())) for n in group]
-                share[0] += n_sm - sum(share)
-                parts = share[group.index(spec.name)]
+                parts = vb.prepared_shares([rows[n] for n in group], n_sm)[group.index(spec.name)]
             dl = dl.prepared(parts)
         layers.append([dl])
         xs_np.append(d["x"])

@@ -258,17 +258,25 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  * indices), no outlier columns,
  * one codebook group, per-input-column scale/bias or none, N <= 31736.
  *
- * Format (version 1; all fields little-endian; the image is 256-byte aligned):
- *   bytes 0..255  header, uint32 words: [0] 0x42515056 ("VPQB")  [1] version = 1  [2] M  [3] N  [4] k1  [5] k2
+ * Format (version 2; all fields little-endian; the image is 256-byte aligned):
+ *   bytes 0..255  header, uint32 words: [0] 0x42515056 ("VPQB")  [1] version = 2  [2] M  [3] N  [4] k1  [5] k2
  *                 [6] n_parts  [7] n_warps = 31  [8] n_buckets = ceil(k1 / 4096)  [9] n_blocks
  *                 [10] byte offset of woff  [11] byte offset of hdr  [12] byte offset of entries (each a
- *                 multiple of 256)  [13] total bytes  [14] number of real entries = ceil(M/8) * N; rest zero
+ *                 multiple of 256)  [13] total bytes  [14] number of real entries = ceil(M/8) * N
+ *                 [15] n_split; rest zero
+ *   partitions    a partition is the work of one CTA.  The R = ceil(M/8) vector rows are cut into
+ *            n_parts / n_split row groups, group g = rows [R*g/groups, R*(g+1)/groups), at most 63 rows; the
+ *            n_split partitions of a group (p = g*n_split + h) each hold the group's entries of one range of
+ *            buckets, [n_buckets*h/n_split, n_buckets*(h+1)/n_split).  n_split is the largest of 8, 4, 2, 1
+ *            that divides n_parts, does not exceed n_buckets and keeps a group within 63 rows: a CTA then
+ *            brings in only its range of the main codebook, and has more rows' work per bucket to hide that
+ *            transfer behind.  The CTAs of a group add their partial sums up through the workspace.
  *   woff     uint32 [n_parts * n_warps + 1]: warp w of partition p owns blocks [woff[p*n_warps + w],
- *            woff[p*n_warps + w + 1]); partition p covers the vector rows [R*p/n_parts, R*(p+1)/n_parts),
- *            R = ceil(M/8), and must not hold more than 63 of them
+ *            woff[p*n_warps + w + 1])
  *   hdr      uint32 [n_blocks]: bits 24..31 = bucket of the block; bits 6q..6q+5 (q = 0..3) = vector row,
  *            relative to the partition's first row, that the lanes 8q..8q+7 work on in this block, or 63
- *            when those lanes have nothing to do in it.  Buckets ascend within a warp's range.
+ *            when those lanes have nothing to do in it.  Buckets ascend within a warp's range and stay
+ *            within the partition's range.
  *   entries  uint32 [n_blocks][32][4]: a block is four steps of a warp; the four entries of lane L in block
  *            b are the words 4*(32*b + L) .. + 3.  An entry:
  *              bits 0..8    (main index mod 4096) >> 3; the three low bits of the main index are L mod 8
@@ -281,7 +289,8 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *
  * vptq_prepare_bytes: capacity to allocate for the image of this layer split into n_parts partitions
  *   (0 = one per SM of the current device): the header and tables plus 4 bytes x 1.5 x the number of
- *   entries.  VPTQ_E_UNSUPPORTED for a layer that is not eligible, or n_parts too small for the 63-row limit.
+ *   entries.  VPTQ_E_UNSUPPORTED for a layer that is not eligible, or n_parts too small for the 63-row limit
+ *   (with the n_split the rule above gives).
  * vptq_prepare_host: packed_idx / res_idx are HOST copies of the canonical streams, `image` is host memory
  *   of `image_bytes` bytes; plain host code, no CUDA call.  *used_bytes (may be null) receives the size of
  *   the image.  VPTQ_E_WORKSPACE when the image does not fit image_bytes: with index histograms far from
@@ -295,13 +304,19 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  * n_parts does not exceed the SM count (other batch sizes use the canonical streams, which must still be
  * valid), and vptq_linear_fused serves prepared layers of one format (N, activation type, residual stage)
  * whose n_parts sum to at most the SM count with one launch ("fused_decode_bucket_fma"); layers meant to
- * share a launch are therefore prepared with n_parts that add up to the SM count.  The path asks for a
- * 256-byte workspace whose first int32 is a status word (vptq_workspace_status): the kernel compares the
- * image header with the descriptor and writes VPTQ_E_UNSUPPORTED there when they disagree (the outputs are
- * then not written), or VPTQ_E_TIMEOUT when a bounded wait gave up.  The word is only ever WRITTEN on an
- * error, never cleared, so that consecutive calls need nothing between their kernels: clear it once when
- * the workspace is allocated and after reading an error.  An image that vptq_prepare did not write is
- * outside the contract (its header's sizes are trusted). */
+ * share a launch are therefore prepared with n_parts that add up to the SM count (multiples of 4 or 8 where
+ * the rows allow, so that n_split can exceed 1).  The path asks for a workspace (vptq_linear_workspace_bytes:
+ * 256 bytes, plus 4 bytes and a 2 KB block of partial sums per CTA when an image has n_split > 1) whose
+ * first int32 is a status word (vptq_workspace_status): the kernel compares the image header with the
+ * descriptor and writes VPTQ_E_UNSUPPORTED there when they disagree (the outputs are then not written), or
+ * VPTQ_E_TIMEOUT when a bounded wait gave up.  Unlike the other paths this one needs the WHOLE workspace
+ * zero when it is first used: the status word is only ever written on an error and never cleared, and the
+ * arrival counters behind it (one per row group; the last CTA to count itself in adds the group's partial
+ * sums up in partition order and stores, so no CTA waits for another and the result does not depend on
+ * which one was last) are left at zero by every launch that ends without an error.  Consecutive calls
+ * therefore need nothing between their kernels: clear the workspace once when it is allocated and after
+ * reading an error.  An image that vptq_prepare did not write is outside the contract (its header's sizes
+ * are trusted). */
 #define VPTQ_PREPARED_MAGIC 0x42515056u
 int64_t vptq_prepare_bytes(const vptq_layer_desc *desc, int32_t n_parts);
 int vptq_prepare_host(const vptq_layer_desc *desc, const uint8_t *packed_idx, const uint8_t *res_idx,

@@ -442,15 +442,15 @@ double oracle_distortion(const uint16_t *W, int32_t M, int32_t N, int32_t v, con
 /* ------------------------------------------------------------------ */
 
 /* The library can re-order a layer's (main, residual) index pairs into a "prepared image" for its decode
- * kernel.  The image is derived data whose format is stated in the library's header (version 1); this is a
+ * kernel.  The image is derived data whose format is stated in the library's header (version 2); this is a
  * decoder written from that statement, used to check that an image says exactly what the canonical streams
  * say.  The paper has no counterpart (it does not describe an inference data layout).
  *
  * Walks every warp's block range of every partition, checks each rule of the format and writes the index
  * pairs back to idx1 / idx2 [ceil(M/8)][N] (int32).  Returns 0, or a positive code naming the first rule
  * that is broken:
- *   1 header magic/version  2 header geometry differs from the arguments  3 region offsets or sizes
- *   4 block ranges not ascending or not ending at n_blocks  5 bucket out of range or descending within a warp
+ *   1 header magic/version  2 header geometry differs from the arguments, or a split that does not divide the partitions  3 region offsets or sizes
+ *   4 block ranges not ascending or not ending at n_blocks  5 bucket outside the partition's range or descending within a warp
  *   6 an entry in a quarter that names no row / a row outside the partition  7 column out of range
  *   8 main or residual index out of range  9 a (row, column) pair occurs twice  10 a pair is missing
  *   11 a partition holds more than 63 vector rows  12 number of real entries differs from the header's */
@@ -460,11 +460,15 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
     if (image_bytes < 256) return 3;
     uint32_t head[16];
     memcpy(head, image, sizeof(head));
-    if (head[0] != 0x42515056u || head[1] != 1u) return 1;
+    if (head[0] != 0x42515056u || head[1] != 2u) return 1;
     const int64_t R = (M + 7) / 8;
     const uint32_t n_parts = head[6], n_warps = head[7], n_buckets = head[8], n_blocks = head[9];
     if (head[2] != (uint32_t)M || head[3] != (uint32_t)N || head[4] != (uint32_t)k1 || head[5] != (uint32_t)k2) return 2;
     if (n_warps != 31u || n_buckets != (uint32_t)((k1 + 4095) / 4096) || n_parts < 1u || (int64_t)n_parts > R) return 2;
+    /* word 15: partitions per row group; each of them holds one range of buckets */
+    const uint32_t n_split = head[15];
+    if (n_split < 1u || n_parts % n_split != 0u || n_split > n_buckets) return 2;
+    const uint32_t n_groups = n_parts / n_split;
     const uint64_t off_woff = head[10], off_hdr = head[11], off_ent = head[12], total = head[13];
     if (off_woff % 256 || off_hdr % 256 || off_ent % 256 || off_woff < 256) return 3;
     if (off_woff + 4ull * ((uint64_t)n_parts * n_warps + 1) > off_hdr) return 3;
@@ -475,7 +479,9 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
     uint64_t real = 0;
     uint32_t prev_end = 0;
     for (uint32_t p = 0; p < n_parts; p++) {
-        const int64_t r0 = R * p / n_parts, r1 = R * (p + 1) / n_parts;
+        const uint32_t grp = p / n_split, piece = p % n_split;
+        const int64_t r0 = R * grp / n_groups, r1 = R * (grp + 1) / n_groups;
+        const uint32_t bucket_lo = n_buckets * piece / n_split, bucket_hi = n_buckets * (piece + 1) / n_split;
         if (r1 - r0 > 63) return 11;
         for (uint32_t w = 0; w < n_warps; w++) {
             uint32_t lo, hi;
@@ -488,7 +494,7 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
                 uint32_t h;
                 memcpy(&h, hdr_b + 4ull * b, 4);
                 const uint32_t bucket = h >> 24;
-                if (bucket >= n_buckets || bucket < last_bucket) return 5;
+                if (bucket < bucket_lo || bucket >= bucket_hi || bucket < last_bucket) return 5;
                 last_bucket = bucket;
                 for (int lane = 0; lane < 32; lane++) {
                     const uint32_t rowf = (h >> (6 * (lane / 8))) & 63u;

@@ -217,6 +217,25 @@ def vptq_prepare(desc: LayerDesc, ptrs: LayerPtrs, n_parts: int = 0) -> torch.Te
     return image[:used.value]
 
 
+def prepared_shares(vector_rows, n_sm: int):
+    """CTAs for each of several prepared layers that are to share one launch on n_sm SMs (their n_parts): in
+    proportion to the layers' vector rows, and in multiples of 8, 4 or 2 where that lets every image split
+    its buckets over that many CTAs per row group (at most 63 rows in a group)."""
+    rows = [int(r) for r in vector_rows]
+    for q in (8, 4, 2, 1):
+        if q * len(rows) > n_sm:
+            continue
+        share = [q] * len(rows)
+        while sum(share) + q <= n_sm:
+            i = max(range(len(rows)), key=lambda j: rows[j] / share[j])
+            if share[i] + q > rows[i]:                       # never more partitions than rows
+                break
+            share[i] += q
+        if q == 1 or all(-(-r // (s // q)) <= 63 for r, s in zip(rows, share)):
+            return share
+    return [max(1, n_sm // len(rows))] * len(rows)
+
+
 def vptq_dequant(desc: LayerDesc, ptrs: LayerPtrs, W_out: torch.Tensor) -> torch.Tensor:
     assert W_out.is_cuda and W_out.dtype == torch.float16 and W_out.is_contiguous()
     assert tuple(W_out.shape) == (desc.M, desc.N)

@@ -38,9 +38,12 @@ struct BucketParams {
     const uint8_t *image[MAX_FUSED];
     void *out[MAX_FUSED];
     int cta_begin[MAX_FUSED + 1];
+    int n_split[MAX_FUSED];            // CTAs that share a group of vector rows, each with a range of buckets
     int n_layers;
     const void *x;
     int *status;                       // may be null; only ever written on an error (the caller clears it)
+    int *arrived;                      // [grid] one arrival counter per row group (at its first CTA), zero between launches
+    float *slots;                      // [grid][64 * 8] partial sums of a CTA whose row group is split
     unsigned long long wait_limit;     // cycles a device-side wait may take
 };
 
@@ -141,12 +144,16 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     uint32_t dyn;
     asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
     const uint32_t *head = reinterpret_cast<const uint32_t *>(img);
-    const int n_buckets = (L.k1 + PREP_BUCKET - 1) / PREP_BUCKET;
+    const int all_buckets = (L.k1 + PREP_BUCKET - 1) / PREP_BUCKET;
+    const int n_split = P.n_split[li];           // the host derived it from R, k1 and n_parts by the format's rule
     const bool bad = base > XS_ABS || base + dyn < END_ABS ||
-                     __ldg(head + 0) != VPTQ_PREPARED_MAGIC || __ldg(head + 1) != 1u || __ldg(head + 2) != (uint32_t)L.M ||
+                     __ldg(head + 0) != VPTQ_PREPARED_MAGIC || __ldg(head + 1) != 2u || __ldg(head + 2) != (uint32_t)L.M ||
                      __ldg(head + 3) != (uint32_t)L.N || __ldg(head + 4) != (uint32_t)L.k1 || __ldg(head + 5) != (uint32_t)L.k2 ||
                      __ldg(head + 6) != (uint32_t)n_parts || __ldg(head + 7) != (uint32_t)PREP_WARPS ||
-                     __ldg(head + 8) != (uint32_t)n_buckets || (L.R + n_parts - 1) / n_parts > PREP_MAX_ROWS;
+                     __ldg(head + 8) != (uint32_t)all_buckets || __ldg(head + 15) != (uint32_t)n_split ||
+                     n_split < 1 || n_parts % n_split != 0 || n_split > all_buckets ||
+                     (L.R + n_parts / n_split - 1) / (n_parts / n_split) > PREP_MAX_ROWS ||
+                     (n_split > 1 && (P.arrived == nullptr || P.slots == nullptr));
     if (bad) {
         if (threadIdx.x == 0 && P.status) atomicExch(P.status, VPTQ_E_UNSUPPORTED);
         return;
@@ -161,7 +168,9 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     uint4 *cb2 = reinterpret_cast<uint4 *>(abs0 + CB2_ABS);               // [256][8 replicas]
     float *part = reinterpret_cast<float *>(abs0 + PART_ABS);             // [64][8]
     float *red = reinterpret_cast<float *>(abs0 + RED_ABS);               // [BK_WARPS]
-    const int r0 = (int)((long long)L.R * part_id / n_parts), r1 = (int)((long long)L.R * (part_id + 1) / n_parts);
+    const PreparedPart pp = prepared_part(L.R, all_buckets, n_parts, n_split, part_id);
+    const int r0 = pp.r0, r1 = pp.r1;
+    const int b_first = pp.b0, n_buckets = pp.b1 - pp.b0;     // buckets are counted from the partition's first from here on
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; i++) {
@@ -175,12 +184,12 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     // the first two buckets are on their way while the rest of the prologue runs
     if (warp == PREP_WARPS && lane == 0) {
         for (int b = 0; b < 2 && b < n_buckets; b++) {
-            const uint32_t rows = (uint32_t)min(PREP_BUCKET, L.k1 - b * PREP_BUCKET);
+            const uint32_t rows = (uint32_t)min(PREP_BUCKET, L.k1 - (b_first + b) * PREP_BUCKET);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(&full[b])), "r"(rows * 16u) : "memory");
             for (uint32_t q = 0; q < rows; q += 1024)
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                              ::"r"(TAB_ABS + (uint32_t)b * 65536u + q * 16u),
-                               "l"(reinterpret_cast<const uint4 *>(L.c1) + (size_t)b * PREP_BUCKET + q),
+                               "l"(reinterpret_cast<const uint4 *>(L.c1) + (size_t)(b_first + b) * PREP_BUCKET + q),
                                "r"(min(rows - q, 1024u) * 16u), "r"(saddr(&full[b])) : "memory");
         }
     }
@@ -189,7 +198,13 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
         for (int i = threadIdx.x; i < L.k2 * 8; i += BK_THREADS) cb2[i] = __ldg(reinterpret_cast<const uint4 *>(L.c2) + (i >> 3));
     for (int i = threadIdx.x; i < 64 * 8; i += BK_THREADS) part[i] = 0.f;
 
-    // consumer warps: the first blocks of the run are in flight before the activations are touched
+    // consumer warps: the first blocks of the run are in flight before the activations are touched.  A header
+    // word is kept with its bucket counted from the partition's first (one below the range stays at 0).
+    const uint32_t first24 = (uint32_t)b_first << 24;
+    auto load_hdr = [&](const uint32_t *p) {
+        const uint32_t h = __ldg(p);
+        return h >= first24 ? h - first24 : h & 0xFFFFFFu;
+    };
     int q = 0, qe = 0;
     uint4 eb[BK_DEPTH];
     uint32_t hb[BK_DEPTH];
@@ -201,7 +216,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
 #pragma unroll
         for (int d = 0; d < BK_DEPTH; d++) {
             eb[d] = make_uint4(0, 0, 0, 0); hb[d] = 0xFFFFFFu;
-            if (q + d < qe) { eb[d] = ld_stream16(entries + (size_t)(q + d) * 32 + lane); hb[d] = __ldg(hdr + q + d); }
+            if (q + d < qe) { eb[d] = ld_stream16(entries + (size_t)(q + d) * 32 + lane); hb[d] = load_hdr(hdr + q + d); }
         }
     }
 
@@ -260,12 +275,12 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                 ok = mbar_wait(saddr(&empty[b & 1]), ((b >> 1) - 1) & 1, &abort_flag, P.status, P.wait_limit);
                 if (!ok) break;
                 b_stop = b + 1;
-                const uint32_t rows = (uint32_t)min(PREP_BUCKET, L.k1 - b * PREP_BUCKET);
+                const uint32_t rows = (uint32_t)min(PREP_BUCKET, L.k1 - (b_first + b) * PREP_BUCKET);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(&full[b & 1])), "r"(rows * 16u) : "memory");
                 for (uint32_t qq = 0; qq < rows; qq += 1024)
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                                  ::"r"(TAB_ABS + (uint32_t)(b & 1) * 65536u + qq * 16u),
-                                   "l"(reinterpret_cast<const uint4 *>(L.c1) + (size_t)b * PREP_BUCKET + qq),
+                                   "l"(reinterpret_cast<const uint4 *>(L.c1) + (size_t)(b_first + b) * PREP_BUCKET + qq),
                                    "r"(min(rows - qq, 1024u) * 16u), "r"(saddr(&full[b & 1])) : "memory");
             }
             // whatever was issued has landed before the CTA ends (bounded): the latest phase of both barriers
@@ -326,7 +341,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                     const uint32_t h = hb[d];
                     if (q + d + BK_DEPTH < qe) {
                         eb[d] = ld_stream16(entries + (size_t)(q + d + BK_DEPTH) * 32 + lane);
-                        hb[d] = __ldg(hdr + q + d + BK_DEPTH);
+                        hb[d] = load_hdr(hdr + q + d + BK_DEPTH);
                     }
                     const int b = min((int)(h >> 24), n_buckets - 1);
                     if (b > cur_b) { __syncwarp(); enter(b); }
@@ -357,8 +372,33 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     float bterm = 0.f;
     for (int w = 0; w < BK_WARPS; w++) bterm += red[w];
     const int m_lo = r0 * 8, n_m = min(L.M, r1 * 8) - m_lo;
-    for (int i = threadIdx.x; i < n_m; i += BK_THREADS)
-        store_out(P.out[li], (long long)m_lo + i, part[i] + bterm, L.out_dtype);
+    if (n_split == 1) {
+        for (int i = threadIdx.x; i < n_m; i += BK_THREADS)
+            store_out(P.out[li], (long long)m_lo + i, part[i] + bterm, L.out_dtype);
+        return;
+    }
+    // The row group's other CTAs hold the sums over their buckets.  Every CTA leaves its sums in its slot and
+    // counts itself in; the one that finds all others counted adds the slots up, in slot order whoever it is,
+    // and stores.  Nobody waits for anybody, and the counter is back at zero for the next launch.
+    const int first_cta = (int)blockIdx.x - part_id % n_split;             // the row group's first CTA
+    float *mine = P.slots + (size_t)blockIdx.x * (64 * 8);
+    for (int i = threadIdx.x; i < n_m; i += BK_THREADS) mine[i] = part[i];
+    __threadfence();
+    __syncthreads();
+    __shared__ int is_last;
+    if (threadIdx.x == 0) {
+        const int before = atomicAdd(P.arrived + first_cta, 1);
+        is_last = before == n_split - 1;
+        if (is_last) atomicExch(P.arrived + first_cta, 0);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int i = threadIdx.x; i < n_m; i += BK_THREADS) {
+        float y = 0.f;
+        for (int h = 0; h < n_split; h++) y += __ldcg(P.slots + (size_t)(first_cta + h) * (64 * 8) + i);
+        store_out(P.out[li], (long long)m_lo + i, y + bterm, L.out_dtype);
+    }
 }
 
 size_t bucket_smem_bytes() { return END_ABS - 1024 - 128; }      // dynamic part: the window starts with 1 KB + the static variables
@@ -370,8 +410,20 @@ bool bucket_fma_supported(const LayerView &L, int B)
     return B == 1 && prepared_eligible(L);
 }
 
+size_t bucket_fma_workspace_bytes(const LayerView *Ls, const int *n_parts, int n)
+{
+    int grid = 0;
+    bool split = false;
+    for (int l = 0; l < n; l++) {
+        grid += n_parts[l];
+        split = split || prepared_split(Ls[l].R, ceil_div(Ls[l].k1, PREP_BUCKET), n_parts[l]) > 1;
+    }
+    if (!split) return 256;
+    return 256 + (size_t)align256(4ull * (unsigned long long)grid) + (size_t)grid * 64 * 8 * 4;
+}
+
 cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *images, const int *n_parts, int n,
-                                     const void *x, void *const *outs, int *status, unsigned long long wait_limit,
+                                     const void *x, void *const *outs, void *workspace, unsigned long long wait_limit,
                                      cudaStream_t st)
 {
     if (n < 1 || n > MAX_FUSED) return cudaErrorInvalidValue;
@@ -383,12 +435,17 @@ cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *ima
         P.image[l] = reinterpret_cast<const uint8_t *>(images[l]);
         P.out[l] = outs[l];
         P.cta_begin[l] = grid;
+        P.n_split[l] = prepared_split(Ls[l].R, ceil_div(Ls[l].k1, PREP_BUCKET), n_parts[l]);
         grid += n_parts[l];
     }
     P.cta_begin[n] = grid;
     P.n_layers = n;
     P.x = x;
-    P.status = status;
+    P.status = reinterpret_cast<int *>(workspace);
+    if (workspace && bucket_fma_workspace_bytes(Ls, n_parts, n) > 256) {
+        P.arrived = reinterpret_cast<int *>(reinterpret_cast<uint8_t *>(workspace) + 256);
+        P.slots = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(workspace) + 256 + align256(4ull * (unsigned long long)grid));
+    }
     P.wait_limit = wait_limit ? wait_limit : WAIT_LIMIT_CYCLES;
     const bool res = Ls[0].k2 > 0;
     const size_t smem = bucket_smem_bytes();

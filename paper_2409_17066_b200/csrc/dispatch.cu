@@ -23,7 +23,8 @@ LinearPath choose_path(const LayerView &L, int B, int flags)
         return PATH_GENERIC;
     }
     if (L.prep_parts > 0 && bucket_fma_supported(L, B) && L.prep_parts <= device_sm_count() &&
-        ceil_div(L.R, L.prep_parts) <= PREP_MAX_ROWS) return PATH_DECODE_BUCKET_FMA;
+        ceil_div(L.R, L.prep_parts / prepared_split(L.R, ceil_div(L.k1, PREP_BUCKET), L.prep_parts)) <= PREP_MAX_ROWS)
+        return PATH_DECODE_BUCKET_FMA;
     if (B > DECODE_MAX_B && gemm_tcgen05_supported(L, B)) return PATH_GEMM_TCGEN05;
     const int Bg = decode_group(B);
     if (smem_fma_supported(L, Bg)) return PATH_DECODE_SMEM_FMA;
@@ -54,7 +55,7 @@ long long linear_workspace_bytes(const LayerView &L, int B, int flags)
     case PATH_DECODE_L2_FMA: return l2_fma_workspace_bytes(L, decode_group(B));
     case PATH_DECODE_GL_FMA: return 0;
     case PATH_GEMM_TCGEN05: return gemm_tcgen05_workspace_bytes(L, B);
-    case PATH_DECODE_BUCKET_FMA: return 256;          // the status word
+    case PATH_DECODE_BUCKET_FMA: return (long long)bucket_fma_workspace_bytes(&L, &L.prep_parts, 1);
     default: return generic_workspace_bytes(L, B);
     }
 }
@@ -89,7 +90,7 @@ int linear_dispatch(const LayerView &L, int flags, const void *x, int B, void *o
     } else if (path == PATH_DECODE_BUCKET_FMA) {
         const void *img = L.prepared;
         void *o = out;
-        e = launch_decode_bucket_fma(&L, &img, &L.prep_parts, 1, x, &o, reinterpret_cast<int *>(ws), debug_wait_limit(), st);
+        e = launch_decode_bucket_fma(&L, &img, &L.prep_parts, 1, x, &o, ws, debug_wait_limit(), st);
     } else {
         // decode kernels take up to 16 tokens per launch
         const size_t oe = (L.out_dtype == VPTQ_DTYPE_FP32) ? 4 : 2;
@@ -147,7 +148,11 @@ const char *linear_fused_path_name(const LayerView *Ls, const int *flags, int n,
 long long linear_fused_workspace_bytes(const LayerView *Ls, const int *flags, int n, int B)
 {
     const LinearPath fp = fused_path(Ls, flags, n, B);
-    if (fp == PATH_DECODE_BUCKET_FMA) return 256;
+    if (fp == PATH_DECODE_BUCKET_FMA) {
+        int parts[MAX_FUSED];
+        for (int l = 0; l < n; l++) parts[l] = Ls[l].prep_parts;
+        return (long long)bucket_fma_workspace_bytes(Ls, parts, n);
+    }
     if (fp != PATH_GENERIC) return 0;
     long long need = 0;       // one layer after the other on the stream: they share the scratch
     for (int l = 0; l < n; l++) {
@@ -179,7 +184,7 @@ int linear_fused_dispatch(const LayerView *Ls, const int *flags, int n, const vo
             const void *imgs[MAX_FUSED];
             int parts[MAX_FUSED];
             for (int l = 0; l < n; l++) { imgs[l] = Ls[l].prepared; parts[l] = Ls[l].prep_parts; }
-            *cuda_err = launch_decode_bucket_fma(Ls, imgs, parts, n, x, outs, reinterpret_cast<int *>(ws), debug_wait_limit(), st);
+            *cuda_err = launch_decode_bucket_fma(Ls, imgs, parts, n, x, outs, ws, debug_wait_limit(), st);
         }
         else if (path == PATH_DECODE_SMEM_FMA) *cuda_err = launch_decode_smem_fma_fused(Ls, n, x, B, outs, st);
         else *cuda_err = launch_decode_gl_fma_fused(Ls, n, x, B, outs, st);

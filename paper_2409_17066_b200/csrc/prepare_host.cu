@@ -29,7 +29,8 @@ struct QuarterBlock {
 void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long stride1, const uint8_t *idx2,
                      long long stride2, int part, PartImage *out)
 {
-    const int r0 = (int)((long long)g.R * part / g.n_parts), r1 = (int)((long long)g.R * (part + 1) / g.n_parts);
+    const PreparedPart pp = prepared_part(g.R, g.n_buckets, g.n_parts, g.n_split, part);
+    const int r0 = pp.r0, r1 = pp.r1;          // the partition's rows, and of their entries those of the buckets [b0, b1)
     const uint32_t pad = (uint32_t)g.N << 17;
     std::vector<std::vector<QuarterBlock>> qb(g.n_buckets);
     std::vector<uint32_t> sorted((size_t)g.N);                  // the row's entries, by (bucket, residue)
@@ -53,7 +54,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
             if (g.k2 > 0 && id2 >= (uint32_t)g.k2) id2 = (uint32_t)g.k2 - 1;
             sorted[(size_t)fill[(id >> 12) * 8 + (id & 7)]++] = ((id & 0xFFFu) >> 3) | (id2 << 9) | ((uint32_t)n << 17);
         }
-        for (int b = 0; b < g.n_buckets; b++) {
+        for (int b = pp.b0; b < pp.b1; b++) {
             int steps = 0;
             for (int c = 0; c < 8; c++) steps = std::max(steps, count[b * 8 + c]);
             // The order of a lane's entries is free.  It is chosen so that the 32 lanes of a warp step look their
@@ -96,7 +97,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
     // the slowest, so what has to be even is the running total, not every bucket by itself.
     std::vector<std::vector<uint32_t>> w_hdr(PREP_WARPS), w_ent(PREP_WARPS);
     long long done[PREP_WARPS] = {0};
-    for (int b = 0; b < g.n_buckets; b++) {
+    for (int b = pp.b0; b < pp.b1; b++) {
         const long long Q = (long long)qb[b].size(), nblk = (Q + 3) / 4;
         long long share[PREP_WARPS];
         int order[PREP_WARPS];
@@ -156,11 +157,12 @@ int prepare_host(const PreparedGeometry &g, const uint8_t *idx1, const uint8_t *
     uint8_t *img = reinterpret_cast<uint8_t *>(image);
     memset(img, 0, 256);
     uint32_t *head = reinterpret_cast<uint32_t *>(img);
-    head[0] = VPTQ_PREPARED_MAGIC; head[1] = 1; head[2] = (uint32_t)g.M; head[3] = (uint32_t)g.N;
+    head[0] = VPTQ_PREPARED_MAGIC; head[1] = 2; head[2] = (uint32_t)g.M; head[3] = (uint32_t)g.N;
     head[4] = (uint32_t)g.k1; head[5] = (uint32_t)g.k2; head[6] = (uint32_t)g.n_parts; head[7] = PREP_WARPS;
     head[8] = (uint32_t)g.n_buckets; head[9] = (uint32_t)n_blocks;
     head[10] = (uint32_t)lay.off_woff; head[11] = (uint32_t)lay.off_hdr; head[12] = (uint32_t)lay.off_entries;
     head[13] = (uint32_t)lay.total; head[14] = (uint32_t)((unsigned long long)g.R * g.N);
+    head[15] = (uint32_t)g.n_split;
     uint32_t *woff = reinterpret_cast<uint32_t *>(img + lay.off_woff);
     uint32_t *hdr = reinterpret_cast<uint32_t *>(img + lay.off_hdr);
     uint32_t *ent = reinterpret_cast<uint32_t *>(img + lay.off_entries);

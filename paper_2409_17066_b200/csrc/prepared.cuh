@@ -12,7 +12,34 @@ constexpr int PREP_MAX_N = 31736;           // the staged activations must fit b
 
 struct PreparedGeometry {
     int M, N, k1, k2, R, n_parts, n_buckets;
+    int n_split;                            // partitions that share a group of vector rows, each with a range of buckets
 };
+
+// Partition p of an image: row group p / n_split (the groups split the R vector rows evenly) and the
+// h-th of n_split bucket ranges, h = p % n_split.
+struct PreparedPart {
+    int r0, r1, b0, b1;
+};
+__host__ __device__ inline PreparedPart prepared_part(int R, int n_buckets, int n_parts, int n_split, int p)
+{
+    const int groups = n_parts / n_split, g = p / n_split, h = p - g * n_split;
+    PreparedPart q;
+    q.r0 = (int)((long long)R * g / groups);
+    q.r1 = (int)((long long)R * (g + 1) / groups);
+    q.b0 = n_buckets * h / n_split;
+    q.b1 = n_buckets * (h + 1) / n_split;
+    return q;
+}
+
+// The split an image of n_parts partitions gets: the largest of 8, 4, 2, 1 that divides n_parts, leaves every
+// partition a bucket, and keeps a row group within PREP_MAX_ROWS rows.  Fewer buckets per CTA mean fewer
+// codebook slices to bring in, and more rows per bucket to hide their latency behind.
+inline int prepared_split(int R, int n_buckets, int n_parts)
+{
+    for (int s = 8; s > 1; s >>= 1)
+        if (n_parts % s == 0 && s <= n_buckets && ceil_div(R, n_parts / s) <= PREP_MAX_ROWS) return s;
+    return 1;
+}
 
 struct PreparedLayout {
     unsigned long long off_woff, off_hdr, off_entries, total;
@@ -45,7 +72,8 @@ inline bool prepared_geometry(const LayerView &L, int n_parts, PreparedGeometry 
     if (n_parts > L.R) n_parts = L.R;
     g->M = L.M; g->N = L.N; g->k1 = L.k1; g->k2 = L.k2; g->R = L.R; g->n_parts = n_parts;
     g->n_buckets = (L.k1 + PREP_BUCKET - 1) / PREP_BUCKET;
-    return ceil_div(L.R, n_parts) <= PREP_MAX_ROWS;
+    g->n_split = prepared_split(L.R, g->n_buckets, n_parts);
+    return ceil_div(L.R, n_parts / g->n_split) <= PREP_MAX_ROWS;
 }
 
 // capacity handed out by vptq_prepare_bytes: tables for the worst block count that fits, 1.5 x 4 bytes per entry
@@ -61,8 +89,11 @@ int prepare_host(const PreparedGeometry &g, const uint8_t *idx1, const uint8_t *
 
 // decode kernel over prepared images (batch 1): n layers of one launch, CTAs dealt out by the images' n_parts
 bool bucket_fma_supported(const LayerView &L, int B);
+// Workspace of a launch over these layers: 256 bytes (status word) and, when an image splits its buckets over
+// several CTAs, one arrival counter and one block of partial sums per CTA.
+size_t bucket_fma_workspace_bytes(const LayerView *Ls, const int *n_parts, int n);
 cudaError_t launch_decode_bucket_fma(const LayerView *Ls, const void *const *images, const int *n_parts, int n,
-                                     const void *x, void *const *outs, int *status, unsigned long long wait_limit,
+                                     const void *x, void *const *outs, void *workspace, unsigned long long wait_limit,
                                      cudaStream_t st);
 
 }  // namespace vptq

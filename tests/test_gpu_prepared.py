@@ -35,6 +35,9 @@ SMALL = [
     (synth.LayerSpec("p_bf16out", 136, 523, v=8, k1=65536, k2=256, out_dtype="bf16"), 2),  # N not a multiple of 8
     (synth.LayerSpec("p_perm", 264, 1032, v=8, k1=65536, k2=256, permuted=True), 9),
     (synth.LayerSpec("p_148", 2048, 640, v=8, k1=65536, k2=256), 0),                       # one partition per SM
+    (synth.LayerSpec("p_split2", 1024, 300, v=8, k1=65536), 6),                            # 3 row groups x 2 bucket ranges
+    (synth.LayerSpec("p_split8", 400, 520, v=8, k1=40000, k2=200), 8),                     # 1 row group x 8 bucket ranges
+    (synth.LayerSpec("p_split4_bf16", 520, 1030, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="bf16"), 8),
 ]
 
 

@@ -25,15 +25,18 @@ def _layer(b, M, N, k1, k2, seed, flags=None):
     return desc, idx1, idx2
 
 
-@pytest.mark.parametrize("M,N,k1,k2,n_parts", [
-    (520, 300, 65536, 256, 7),       # ragged last vector row, several partitions
-    (264, 1030, 65536, 256, 33),     # one vector row per partition
-    (1024, 256, 65536, 0, 3),        # no residual stage; 43 rows in a partition
-    (400, 200, 40000, 200, 5),       # 10 buckets, the last one short; a residual table of 200 entries
-    (64, 64, 33000, 256, 1),         # nine buckets, the last one short; a single partition
-    (2048, 128, 65536, 256, 148),    # more partitions than ... one or two rows each
+@pytest.mark.parametrize("M,N,k1,k2,n_parts,n_split", [
+    (520, 300, 65536, 256, 7, 1),       # ragged last vector row, several partitions
+    (264, 1030, 65536, 256, 33, 1),     # one vector row per partition
+    (1024, 256, 65536, 0, 3, 1),        # no residual stage; 43 rows in a partition
+    (400, 200, 40000, 200, 5, 1),       # 10 buckets, the last one short; a residual table of 200 entries
+    (64, 64, 33000, 256, 1, 1),         # nine buckets, the last one short; a single partition
+    (2048, 128, 65536, 256, 148, 4),    # 37 row groups of 6 or 7 rows, four bucket ranges each
+    (520, 300, 65536, 256, 8, 4),       # 65 rows: one group of 8 partitions would exceed 63 rows, two groups of 4
+    (400, 200, 40000, 200, 8, 8),       # one row group; 10 buckets over 8 partitions (one or two each)
+    (1024, 96, 65536, 0, 6, 2),         # three row groups, two bucket ranges each
 ])
-def test_image_decodes_back_to_the_index_matrices(b, M, N, k1, k2, n_parts):
+def test_image_decodes_back_to_the_index_matrices(b, M, N, k1, k2, n_parts, n_split):
     desc, idx1, idx2 = _layer(b, M, N, k1, k2, seed=M + N)
     p1 = oracle.pack(idx1, k1)
     p2 = oracle.pack(idx2, k2) if k2 else None
@@ -44,7 +47,7 @@ def test_image_decodes_back_to_the_index_matrices(b, M, N, k1, k2, n_parts):
     assert np.array_equal(got1, idx1)
     assert np.array_equal(got2, idx2 if k2 else np.zeros_like(idx1))
     head = image[:64].view(np.uint32)
-    assert head[6] == min(n_parts, -(-M // 8)) and head[14] == idx1.size
+    assert head[6] == min(n_parts, -(-M // 8)) and head[14] == idx1.size and head[15] == n_split
     # padding stays moderate with uniform indices (bank rule: a quarter warp's 8 lanes take 8 residues mod 8)
     slots = int(head[9]) * 128
     assert slots >= idx1.size
@@ -89,6 +92,11 @@ def test_decoder_names_the_broken_rule(b):
     q = (e0 % 128) // 4 // 8
     assert broken(lambda im: set_hdr(im, blk, int(hdr[blk]) | (63 << (6 * q)))) == 6
     assert broken(lambda im: set_hdr(im, blk, (int(hdr[blk]) & 0xFFFFFF) | (200 << 24))) == 5
+    # the image has one row group and four bucket ranges: a bucket of another partition's range is refused too
+    assert head[15] == 4
+    elsewhere = ((int(hdr[blk]) >> 24) + 8) % 16
+    assert broken(lambda im: set_hdr(im, blk, (int(hdr[blk]) & 0xFFFFFF) | (elsewhere << 24))) == 5
+    assert broken(lambda im: im[60:64].view(np.uint32).__setitem__(0, 3)) == 2             # a split that does not divide 4
     # a residual index beyond the table
     assert oracle.decode_prepared(image, M, N, k1, 256)[0] == 0
     d2, i1, i2 = _layer(b, M, N, k1, 200, seed=6)
@@ -148,7 +156,10 @@ def test_eligibility_and_argument_errors(b):
     prep = b.make_desc(4096, 4096, 8, 65536, 256, flags=b.FLAG_SCALE_BIAS | b.FLAG_PREPARED, prepared_parts=148)
     assert b.vptq_linear_path(prep, 1) == "decode_bucket_fma"
     assert b.vptq_linear_path(prep, 2) == "decode_l2_fma"                    # other batch sizes read the canonical streams
-    assert b.vptq_linear_workspace_bytes(prep, 1) == 256
+    # 512 vector rows over 148 CTAs: 37 row groups of four bucket ranges; a counter and 2 KB of sums per CTA
+    assert b.vptq_linear_workspace_bytes(prep, 1) == 256 + 768 + 148 * 2048
+    odd = b.make_desc(4096, 4096, 8, 65536, 256, flags=b.FLAG_SCALE_BIAS | b.FLAG_PREPARED, prepared_parts=147)
+    assert b.vptq_linear_workspace_bytes(odd, 1) == 256                      # no split: the status word only
     noparts = b.make_desc(4096, 4096, 8, 65536, 256, flags=b.FLAG_SCALE_BIAS | b.FLAG_PREPARED)
     assert b.lib.vptq_linear_workspace_bytes(C.byref(noparts), 1) == b.E_SHAPE
     p = b.LayerPtrs(0x1000, 0x1000, 0x1000, 0x1000, None, None, 0x1000, 0x1000, None, None)
