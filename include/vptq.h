@@ -256,7 +256,7 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *
  * Eligible layers: v = 8, 32768 < k1 <= 65536 (16-bit main indices), k2 = 0 or 128 < k2 <= 256 (8-bit residual
  * indices), no outlier columns,
- * one codebook group, per-input-column scale/bias or none, N <= 31736.
+ * one codebook group, per-input-column scale/bias or none, N <= 31680.
  *
  * Format (version 2; all fields little-endian; the image is 256-byte aligned):
  *   bytes 0..255  header, uint32 words: [0] 0x42515056 ("VPQB")  [1] version = 2  [2] M  [3] N  [4] k1  [5] k2
@@ -283,7 +283,10 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *                           (so the eight lanes of a quarter warp always read eight different 16-byte banks)
  *                           and its high bits are the block's bucket
  *              bits 9..16   residual index (0 when k2 = 0)
- *              bits 17..31  stored column n of the weight, or N for "no entry" (padding)
+ *              bits 17..31  stored column n of the weight, or one of N .. N+63 for "no entry" (padding; the
+ *                           kernel keeps a zero activation for each of these, one per shared-memory bank
+ *                           and half word, and the builder names the one whose bank the step's other
+ *                           lanes leave free)
  * Every (vector row, column) pair of the layer occurs exactly once among the entries that are not padding,
  * in a quarter whose header field names that row.
  *

@@ -502,8 +502,8 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
                         uint32_t e;
                         memcpy(&e, ent_b + 4ull * (4ull * (32ull * b + (uint64_t)lane) + (uint64_t)s), 4);
                         const uint32_t col = e >> 17;
-                        if (col == (uint32_t)N) continue;                 /* padding */
-                        if (col > (uint32_t)N) return 7;
+                        if (col >= (uint32_t)N && col < (uint32_t)N + 64u) continue;   /* "no entry": columns N .. N+63 */
+                        if (col >= (uint32_t)N + 64u) return 7;
                         if (rowf == 63u || (int64_t)rowf >= r1 - r0) return 6;
                         const int64_t main_idx = (int64_t)bucket * 4096 + (int64_t)((e & 0x1FFu) << 3) + (lane % 8);
                         const int64_t res_idx = (e >> 9) & 0xFFu;

@@ -30,7 +30,7 @@ constexpr int BK_DEPTH = 2;                                  // blocks in flight
 // absolute shared-memory addresses (the window starts with 1 KB the system keeps and the static variables)
 constexpr uint32_t XS_ABS = 2048, TAB_ABS = 65536, CB2_ABS = 196608, PART_ABS = CB2_ABS + 32768,
                    RED_ABS = PART_ABS + 64 * 8 * 4, END_ABS = RED_ABS + BK_WARPS * 4;
-static_assert(XS_ABS + 2 * (PREP_MAX_N + 8) <= TAB_ABS, "activations must end below the first bucket buffer");
+static_assert(XS_ABS + 2 * (PREP_MAX_N + PREP_PAD_COLS) <= TAB_ABS, "activations must end below the first bucket buffer");
 constexpr unsigned long long WAIT_LIMIT_CYCLES = 4000000000ull;      // about two seconds
 
 struct BucketParams {
@@ -116,7 +116,7 @@ __device__ __forceinline__ void slot(uint32_t e, uint32_t pad, uint32_t tab_lane
         w.x = *reinterpret_cast<uint32_t *>(&a0); w.y = *reinterpret_cast<uint32_t *>(&a1);
         w.z = *reinterpret_cast<uint32_t *>(&a2); w.w = *reinterpret_cast<uint32_t *>(&a3);
     }
-    // a padding entry names column N; it must add nothing even when its table row holds an infinity
+    // a padding entry names a column >= N; it must add nothing even when its table row holds an infinity
     fma8(acc, xh, w, e < pad);
 }
 
@@ -164,7 +164,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     const uint32_t n_blocks = __ldg(head + 9);
 
     uint8_t *const abs0 = smem - base;                                    // generic pointer of shared address 0
-    __half *xs = reinterpret_cast<__half *>(abs0 + XS_ABS);               // [N + 8]
+    __half *xs = reinterpret_cast<__half *>(abs0 + XS_ABS);               // [N + 64]
     uint4 *cb2 = reinterpret_cast<uint4 *>(abs0 + CB2_ABS);               // [256][8 replicas]
     float *part = reinterpret_cast<float *>(abs0 + PART_ABS);             // [64][8]
     float *red = reinterpret_cast<float *>(abs0 + RED_ABS);               // [BK_WARPS]
@@ -259,7 +259,9 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                 bacc += xv * bi;
             }
         }
-        if (threadIdx.x < 8) xs[L.N + threadIdx.x] = __float2half_rn(0.f);        // column N: "no entry"
+        // columns N .. N+63 mean "no entry": a zero in every bank, so that the lanes without an entry can all
+        // read one word whose bank no other lane of the step uses
+        if (threadIdx.x < PREP_PAD_COLS) xs[L.N + threadIdx.x] = __float2half_rn(0.f);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) bacc += __shfl_xor_sync(0xffffffffu, bacc, o);
         if (lane == 0) red[warp] = bacc;

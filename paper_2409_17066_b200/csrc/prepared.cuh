@@ -8,7 +8,8 @@ namespace vptq {
 constexpr int PREP_WARPS = 31;              // consumer warps of the decode kernel; one more warp loads the buckets
 constexpr int PREP_BUCKET = 4096;           // main-codebook entries per bucket (64 KB)
 constexpr int PREP_MAX_ROWS = 63;           // vector rows per partition (6-bit row fields; 63 = idle)
-constexpr int PREP_MAX_N = 31736;           // the staged activations must fit below the first bucket buffer
+constexpr int PREP_PAD_COLS = 64;           // columns N .. N+63 stand for "no entry" (one per shared-memory bank and half)
+constexpr int PREP_MAX_N = 31680;           // the staged activations (N + 64 halves) must fit below the first bucket buffer
 
 struct PreparedGeometry {
     int M, N, k1, k2, R, n_parts, n_buckets;
