@@ -56,10 +56,10 @@ NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     # profiles/decode_smem_tc_kernel_config2_gate_proj_B8.md: 21.46 MB / 19.0 MB (the 0.5 MB fragment image and the
     # pre-pass's traffic included)
     "decode_smem_tc_kernel": (1.13, "decode_smem_tc.cu", "ccf102769587"),
-    # profiles/decode_bucket_fma_kernel_config3_gate_up_fused_B1.md: (287.97 + 4.20) MB DRAM / 178.33 MB canonical
+    # profiles/decode_bucket_fma_kernel_config3_gate_up_fused_B1.md: (287.97 + 3.70) MB DRAM / 178.33 MB canonical
     # compressed bytes: the kernel reads the prepared image (4 bytes per slot, 21 % padding at N = 8192; the
     # N = 28672 image of down_proj is 1.47 x its canonical bytes, so this overstates that launch by a tenth)
-    "decode_bucket_fma_kernel": (1.638, "decode_bucket_fma.cu", "c889edeb5e87"),
+    "decode_bucket_fma_kernel": (1.636, "decode_bucket_fma.cu", "ac422d948d6a"),
 }
 
 ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "decode_smem_fma_kernel", "decode_gl_fma": "decode_gl_fma_kernel", "decode_smem_mma": "decode_smem_tc_kernel",
@@ -67,9 +67,8 @@ ROOFLINE_KERNEL = {"decode_l2_fma": "decode_l2_fma_kernel", "decode_smem_fma": "
                    "fused_decode_l2_fma": "decode_l2_fma_kernel", "fused_decode_smem_fma": "decode_smem_fma_kernel",
                    "fused_decode_gl_fma": "decode_gl_fma_kernel",
                    "decode_bucket_fma": "decode_bucket_fma_kernel", "fused_decode_bucket_fma": "decode_bucket_fma_kernel"}
-# layers of the headline workload that get a prepared image (vptq_prepare): the large projections, where the
-# decode over bucket-ordered entries beats the decode over the canonical streams; partitions of fused groups
-# add up to the SM count
+# layers of the headline workload that get a prepared image (vptq_prepare): all seven projections; the
+# partitions of a fused group add up to the SM count
 PREPARED_DEFAULT = "q_proj,k_proj,v_proj,o_proj,gate_proj,up_proj,down_proj"
 # projections of a decoder layer that read the same activations
 FUSE_GROUPS = (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj"))
