@@ -270,7 +270,7 @@ def run_ours(args):
             parts = 0
             if group is not None and not args.no_fuse and all(n in prepared and n in kept for n in group):
                 rows = {sp.name: sp.R for sp in cfg["layers"] if sp.name in group}
-                parts = vb.prepared_shares([rows[n] for n in group], n_sm)[group.index(spec.name)]
+                parts = vb.prepared_shares([rows[n] for n in group], n_sm, -(-spec.k1 // 4096))[group.index(spec.name)]
             dl = dl.prepared(parts)
         layers.append([dl])
         xs_np.append(d["x"])
@@ -617,6 +617,15 @@ def extra_configs(vb, synth, peaks):
                     r["dense_fp16_TFLOPs"] = fl / (dm * 1e-3) / 1e12
                     del W, xh
                 res[key] = r
+                # the same layer over a prepared image, where the format has one and the call does not use it yet
+                if B == 1 and vb.lib.vptq_prepare_bytes(C.byref(base.desc), 0) > 0:
+                    pbase = base.prepared(0)
+                    pvar = [pbase] + [pbase.clone_streams() for _ in range(n_copies - 1)]
+                    gms, med, mn = time_calls(lambda i: pvar[i].linear(x, out), n_copies)
+                    res[key + "_prepared"] = {"us": 1e3 * gms, "us_eager_median": 1e3 * med, "us_eager_min": 1e3 * mn,
+                                              "GBps": wb / (gms * 1e-3) / 1e9, "frac_hbm": wb / (gms * 1e-3) / 1e9 / peaks["hbm"],
+                                              "path": vb.vptq_linear_path(pbase.desc, 1), "weight_copies": n_copies}
+                    del pvar, pbase
             del variants, base, d
             torch.cuda.empty_cache()
     res.update(extra_fused(vb, synth, peaks))
@@ -689,6 +698,18 @@ def extra_fused(vb, synth, peaks):
         res[f"cfg{cfg}_fused_{label}_B{B}"] = {
             "us": 1e3 * g, "us_one_call_per_layer": 1e3 * gs, "GBps": wb / (g * 1e-3) / 1e9,
             "frac_hbm": wb / (g * 1e-3) / 1e9 / peaks["hbm"], "path": fused[0].path(B), "weight_copies": n}
+        if B == 1 and all(vb.lib.vptq_prepare_bytes(C.byref(dl.desc), 0) > 0 for dl in base):
+            # the same call over prepared images that share the SMs
+            n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+            shares = vb.prepared_shares([dl.spec.R for dl in base], n_sm, -(-base[0].spec.k1 // 4096))
+            pbase = [dl.prepared(p) for dl, p in zip(base, shares)]
+            pcopies = [[dl] + [dl.clone_streams() for _ in range(n - 1)] for dl in pbase]
+            pfused = [vb.FusedLayers([pcopies[l][c] for l in range(len(base))]) for c in range(n)]
+            g, _, _ = time_calls(lambda i: pfused[i].linear(x, outs), n)
+            res[f"cfg{cfg}_fused_{label}_B{B}_prepared"] = {
+                "us": 1e3 * g, "GBps": wb / (g * 1e-3) / 1e9, "frac_hbm": wb / (g * 1e-3) / 1e9 / peaks["hbm"],
+                "path": pfused[0].path(B), "weight_copies": n}
+            del pfused, pcopies, pbase
         del fused, copies, base, ds
         torch.cuda.empty_cache()
     return res

@@ -254,17 +254,18 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  * the canonical streams (vptq_prepare), it can be rebuilt at any time, and the canonical streams stay the
  * interchange format (vptq_dequant and the other paths keep using them).  The paper has no counterpart.
  *
- * Eligible layers: v = 8, 32768 < k1 <= 65536 (16-bit main indices), k2 = 0 or 128 < k2 <= 256 (8-bit residual
- * indices), no outlier columns,
- * one codebook group, per-input-column scale/bias or none, N <= 31680.
+ * Eligible layers: v = 8 with any k1 <= 65536, or v < 8 with k1 <= 4096 (one bucket, which the kernel widens
+ * to 16-byte rows itself); k2 = 0 or k2 <= 256; outlier columns with v0 <= 8 (they stay on their canonical
+ * stream: the image holds the main columns' entries only); one codebook group; per-input-column scale/bias
+ * or none; N <= 31680.  "Vector row" below means v consecutive output rows, R = ceil(M/v) of them.
  *
  * Format (version 2; all fields little-endian; the image is 256-byte aligned):
  *   bytes 0..255  header, uint32 words: [0] 0x42515056 ("VPQB")  [1] version = 2  [2] M  [3] N  [4] k1  [5] k2
  *                 [6] n_parts  [7] n_warps = 31  [8] n_buckets = ceil(k1 / 4096)  [9] n_blocks
  *                 [10] byte offset of woff  [11] byte offset of hdr  [12] byte offset of entries (each a
- *                 multiple of 256)  [13] total bytes  [14] number of real entries = ceil(M/8) * N
- *                 [15] n_split; rest zero
- *   partitions    a partition is the work of one CTA.  The R = ceil(M/8) vector rows are cut into
+ *                 multiple of 256)  [13] total bytes  [14] number of real entries = R * (N - n_outlier)
+ *                 [15] n_split  [16] v  [17] n_outlier; rest zero
+ *   partitions    a partition is the work of one CTA.  The R vector rows are cut into
  *            n_parts / n_split row groups, group g = rows [R*g/groups, R*(g+1)/groups), at most 63 rows; the
  *            n_split partitions of a group (p = g*n_split + h) each hold the group's entries of one range of
  *            buckets, [n_buckets*h/n_split, n_buckets*(h+1)/n_split).  n_split is the largest of 8, 4, 2, 1
@@ -283,11 +284,12 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *                           (so the eight lanes of a quarter warp always read eight different 16-byte banks)
  *                           and its high bits are the block's bucket
  *              bits 9..16   residual index (0 when k2 = 0)
- *              bits 17..31  stored column n of the weight, or one of N .. N+63 for "no entry" (padding; the
+ *              bits 17..31  stored column n of the weight (n_outlier <= n < N: main column n - n_outlier of
+ *                           the canonical streams), or one of N .. N+63 for "no entry" (padding; the
  *                           kernel keeps a zero activation for each of these, one per shared-memory bank
  *                           and half word, and the builder names the one whose bank the step's other
  *                           lanes leave free)
- * Every (vector row, column) pair of the layer occurs exactly once among the entries that are not padding,
+ * Every (vector row, main column) pair of the layer occurs exactly once among the entries that are not padding,
  * in a quarter whose header field names that row.
  *
  * vptq_prepare_bytes: capacity to allocate for the image of this layer split into n_parts partitions

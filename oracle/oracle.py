@@ -75,8 +75,8 @@ _lib.oracle_kmeans_update.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int3
 _lib.oracle_distortion.restype = C.c_double
 _lib.oracle_distortion.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.oracle_decode_prepared.restype = C.c_int
-_lib.oracle_decode_prepared.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                                        C.c_void_p, C.c_void_p]
+_lib.oracle_decode_prepared.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_int32, C.c_void_p, C.c_void_p]
 _lib.oracle_num_threads.restype = C.c_int
 _lib.oracle_set_num_threads.argtypes = [C.c_int]
 
@@ -252,14 +252,14 @@ def distortion(W16: np.ndarray, v: int, idx: np.ndarray, codebook: np.ndarray, h
                                         None if hb is None else hb.ctypes.data, Cb.ctypes.data))
 
 
-def decode_prepared(image: np.ndarray, M: int, N: int, k1: int, k2: int):
-    """Index matrices (idx1, idx2), int32 [ceil(M/8)][N], read back from a prepared layer image by the
+def decode_prepared(image: np.ndarray, M: int, N: int, k1: int, k2: int, v: int = 8, n_out: int = 0):
+    """Index matrices (idx1, idx2), int32 [ceil(M/v)][N - n_out], read back from a prepared layer image by the
     format's rules; returns (code, idx1, idx2) where code = 0 or the number of the first broken rule."""
     img = np.ascontiguousarray(image, dtype=np.uint8)
-    R = -(-M // 8)
-    idx1 = np.empty((R, N), dtype=np.int32)
-    idx2 = np.empty((R, N), dtype=np.int32)
-    code = int(_lib.oracle_decode_prepared(img.ctypes.data, img.size, M, N, k1, k2, idx1.ctypes.data, idx2.ctypes.data))
+    R = -(-M // v)
+    idx1 = np.empty((R, N - n_out), dtype=np.int32)
+    idx2 = np.empty((R, N - n_out), dtype=np.int32)
+    code = int(_lib.oracle_decode_prepared(img.ctypes.data, img.size, M, N, v, k1, k2, n_out, idx1.ctypes.data, idx2.ctypes.data))
     return code, idx1, idx2
 
 

@@ -447,23 +447,27 @@ double oracle_distortion(const uint16_t *W, int32_t M, int32_t N, int32_t v, con
  * say.  The paper has no counterpart (it does not describe an inference data layout).
  *
  * Walks every warp's block range of every partition, checks each rule of the format and writes the index
- * pairs back to idx1 / idx2 [ceil(M/8)][N] (int32).  Returns 0, or a positive code naming the first rule
+ * pairs back to idx1 / idx2 [ceil(M/v)][N - n_out] (int32; main columns only, the image holds nothing of the
+ * outlier columns).  Returns 0, or a positive code naming the first rule
  * that is broken:
  *   1 header magic/version  2 header geometry differs from the arguments, or a split that does not divide the partitions  3 region offsets or sizes
  *   4 block ranges not ascending or not ending at n_blocks  5 bucket outside the partition's range or descending within a warp
  *   6 an entry in a quarter that names no row / a row outside the partition  7 column out of range
  *   8 main or residual index out of range  9 a (row, column) pair occurs twice  10 a pair is missing
  *   11 a partition holds more than 63 vector rows  12 number of real entries differs from the header's */
-int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M, int32_t N, int32_t k1, int32_t k2,
-                           int32_t *idx1, int32_t *idx2)
+int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M, int32_t N, int32_t v, int32_t k1, int32_t k2,
+                           int32_t n_out, int32_t *idx1, int32_t *idx2)
 {
     if (image_bytes < 256) return 3;
-    uint32_t head[16];
+    uint32_t head[18];
     memcpy(head, image, sizeof(head));
     if (head[0] != 0x42515056u || head[1] != 2u) return 1;
-    const int64_t R = (M + 7) / 8;
+    if (v < 1 || v > 8 || n_out < 0 || n_out >= N) return 2;
+    const int64_t R = (M + v - 1) / v;       /* vector rows */
+    const int64_t Nc = N - n_out;            /* main columns; they are stored after the outlier columns */
     const uint32_t n_parts = head[6], n_warps = head[7], n_buckets = head[8], n_blocks = head[9];
     if (head[2] != (uint32_t)M || head[3] != (uint32_t)N || head[4] != (uint32_t)k1 || head[5] != (uint32_t)k2) return 2;
+    if (head[16] != (uint32_t)v || head[17] != (uint32_t)n_out) return 2;
     if (n_warps != 31u || n_buckets != (uint32_t)((k1 + 4095) / 4096) || n_parts < 1u || (int64_t)n_parts > R) return 2;
     /* word 15: partitions per row group; each of them holds one range of buckets */
     const uint32_t n_split = head[15];
@@ -475,7 +479,7 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
     if (off_hdr + 4ull * n_blocks > off_ent) return 3;
     if (off_ent + 512ull * n_blocks > total || total > (uint64_t)image_bytes) return 3;
     const uint8_t *woff_b = image + off_woff, *hdr_b = image + off_hdr, *ent_b = image + off_ent;
-    for (int64_t i = 0; i < R * N; i++) { idx1[i] = -1; idx2[i] = -1; }
+    for (int64_t i = 0; i < R * Nc; i++) { idx1[i] = -1; idx2[i] = -1; }
     uint64_t real = 0;
     uint32_t prev_end = 0;
     for (uint32_t p = 0; p < n_parts; p++) {
@@ -504,12 +508,13 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
                         const uint32_t col = e >> 17;
                         if (col >= (uint32_t)N && col < (uint32_t)N + 64u) continue;   /* "no entry": columns N .. N+63 */
                         if (col >= (uint32_t)N + 64u) return 7;
+                        if (col < (uint32_t)n_out) return 7;          /* outlier columns have no entries here */
                         if (rowf == 63u || (int64_t)rowf >= r1 - r0) return 6;
                         const int64_t main_idx = (int64_t)bucket * 4096 + (int64_t)((e & 0x1FFu) << 3) + (lane % 8);
                         const int64_t res_idx = (e >> 9) & 0xFFu;
                         if (main_idx >= k1) return 8;
                         if (k2 > 0 ? res_idx >= k2 : res_idx != 0) return 8;
-                        const int64_t at = (r0 + rowf) * N + col;
+                        const int64_t at = (r0 + rowf) * Nc + ((int64_t)col - n_out);
                         if (idx1[at] != -1) return 9;
                         idx1[at] = (int32_t)main_idx;
                         idx2[at] = (int32_t)res_idx;
@@ -520,7 +525,7 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
         }
     }
     if (prev_end != n_blocks) return 4;
-    for (int64_t i = 0; i < R * N; i++)
+    for (int64_t i = 0; i < R * Nc; i++)
         if (idx1[i] == -1) return 10;
     if (real != (uint64_t)head[14]) return 12;
     return 0;

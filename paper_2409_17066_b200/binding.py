@@ -217,13 +217,13 @@ def vptq_prepare(desc: LayerDesc, ptrs: LayerPtrs, n_parts: int = 0) -> torch.Te
     return image[:used.value]
 
 
-def prepared_shares(vector_rows, n_sm: int):
+def prepared_shares(vector_rows, n_sm: int, n_buckets: int = 16):
     """CTAs for each of several prepared layers that are to share one launch on n_sm SMs (their n_parts): in
     proportion to the layers' vector rows, and in multiples of 8, 4 or 2 where that lets every image split
-    its buckets over that many CTAs per row group (at most 63 rows in a group)."""
+    its n_buckets = ceil(k1 / 4096) buckets over that many CTAs per row group (at most 63 rows in a group)."""
     rows = [int(r) for r in vector_rows]
     for q in (8, 4, 2, 1):
-        if q * len(rows) > n_sm:
+        if q * len(rows) > n_sm or q > max(1, n_buckets):
             continue
         share = [q] * len(rows)
         while sum(share) + q <= n_sm:

@@ -20,6 +20,7 @@
 #include "common.cuh"
 #include "prepared.cuh"
 #include "fused_split.cuh"
+#include "index_words.cuh"
 
 namespace vptq {
 
@@ -120,6 +121,42 @@ __device__ __forceinline__ void slot(uint32_t e, uint32_t pad, uint32_t tab_lane
     fma8(acc, xh, w, e < pad);
 }
 
+// Outlier columns (Sec. 3.2.3: the first n_out stored columns, vectors of v0 rows, codebook c0) of the vector rows
+// [r0, r1): their few indices come from the canonical stream, the centroids from global memory, products in
+// FP32; every consumer warp takes the outlier rows warp, warp + 31, ...  Sums go to part[row][8].
+__device__ __noinline__ void outlier_columns(const LayerView &L, const __half *xs, float *part, int r0, int r1, int warp, int lane)
+{
+    const int m_lo = r0 * L.v, m_hi = min(L.M, r1 * L.v);
+    const int q_lo = m_lo / L.v0, q_hi = (m_hi + L.v0 - 1) / L.v0;
+    for (int qq = q_lo + warp; qq < q_hi; qq += PREP_WARPS) {
+        const uint8_t *row0 = L.s0.ptr + (long long)qq * L.s0.stride;
+        float oacc[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) oacc[j] = 0.f;
+        for (int n = lane; n < L.n_out; n += 32) {
+            const int i0 = clamp_index(load_index(row0, n, L.s0.bits), L.k0);
+            const uint4 cw = load_centroid_row(L.c0, i0, L.v0);
+            const float2 c01 = __half22float2(*reinterpret_cast<const __half2 *>(&cw.x)), c23 = __half22float2(*reinterpret_cast<const __half2 *>(&cw.y)),
+                         c45 = __half22float2(*reinterpret_cast<const __half2 *>(&cw.z)), c67 = __half22float2(*reinterpret_cast<const __half2 *>(&cw.w));
+            const float cj[8] = {c01.x, c01.y, c23.x, c23.y, c45.x, c45.y, c67.x, c67.y};
+            const float xv = __half2float(xs[n]);
+#pragma unroll
+            for (int j = 0; j < 8; j++) oacc[j] += xv * cj[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            float a = oacc[j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            const int m = qq * L.v0 + j;
+            if (lane == 0 && j < L.v0 && m >= m_lo && m < m_hi) {
+                const int rr = m / L.v, jj = m - rr * L.v;
+                atomicAdd(part + (rr - r0) * 8 + jj, a);
+            }
+        }
+    }
+}
+
 template <bool RES>
 __global__ void __launch_bounds__(BK_THREADS, 1)
 decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
@@ -151,9 +188,11 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                      __ldg(head + 3) != (uint32_t)L.N || __ldg(head + 4) != (uint32_t)L.k1 || __ldg(head + 5) != (uint32_t)L.k2 ||
                      __ldg(head + 6) != (uint32_t)n_parts || __ldg(head + 7) != (uint32_t)PREP_WARPS ||
                      __ldg(head + 8) != (uint32_t)all_buckets || __ldg(head + 15) != (uint32_t)n_split ||
+                     __ldg(head + 16) != (uint32_t)L.v || __ldg(head + 17) != (uint32_t)L.n_out ||
                      n_split < 1 || n_parts % n_split != 0 || n_split > all_buckets ||
                      (L.R + n_parts / n_split - 1) / (n_parts / n_split) > PREP_MAX_ROWS ||
-                     (n_split > 1 && (P.arrived == nullptr || P.slots == nullptr));
+                     (n_split > 1 && (P.arrived == nullptr || P.slots == nullptr)) ||
+                     (L.v != 8 && all_buckets != 1) || L.v > 8 || (L.n_out > 0 && L.v0 > 8);
     if (bad) {
         if (threadIdx.x == 0 && P.status) atomicExch(P.status, VPTQ_E_UNSUPPORTED);
         return;
@@ -181,8 +220,10 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
         abort_flag = 0;
     }
     __syncthreads();
-    // the first two buckets are on their way while the rest of the prologue runs
-    if (warp == PREP_WARPS && lane == 0) {
+    // the first two buckets are on their way while the rest of the prologue runs (16-byte rows, v = 8, go by
+    // bulk copy; shorter vectors are widened to 16-byte rows by all threads, one bucket at a time)
+    const bool bulk = L.v == 8;
+    if (bulk && warp == PREP_WARPS && lane == 0) {
         for (int b = 0; b < 2 && b < n_buckets; b++) {
             const uint32_t rows = (uint32_t)min(PREP_BUCKET, L.k1 - (b_first + b) * PREP_BUCKET);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(&full[b])), "r"(rows * 16u) : "memory");
@@ -195,7 +236,13 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     }
     // residual table, eight copies with a 16-byte skew (a4); partial sums
     if (RES)
-        for (int i = threadIdx.x; i < L.k2 * 8; i += BK_THREADS) cb2[i] = __ldg(reinterpret_cast<const uint4 *>(L.c2) + (i >> 3));
+        for (int i = threadIdx.x; i < L.k2 * 8; i += BK_THREADS) cb2[i] = load_centroid_row(L.c2, i >> 3, L.v);
+    if (!bulk) {
+        // a layer of short vectors has one bucket (k1 <= 4096), widened to 16-byte rows here
+        uint4 *tab0 = reinterpret_cast<uint4 *>(abs0 + TAB_ABS);
+        const int rows = min(PREP_BUCKET, L.k1 - b_first * PREP_BUCKET);
+        for (int i = threadIdx.x; i < rows; i += BK_THREADS) tab0[i] = load_centroid_row(L.c1, b_first * PREP_BUCKET + i, L.v);
+    }
     for (int i = threadIdx.x; i < 64 * 8; i += BK_THREADS) part[i] = 0.f;
 
     // consumer warps: the first blocks of the run are in flight before the activations are touched.  A header
@@ -271,6 +318,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     if (warp == PREP_WARPS) {
         // ---- producer: bucket b into buffer b & 1 once every consumer warp has left bucket b - 2 ----
         if (lane == 0) {
+            if (!bulk) mbar_arrive(saddr(&full[0]));          // the one bucket was written by all threads above
             bool ok = true;
             int b_stop = min(2, n_buckets);          // buckets issued so far
             for (int b = 2; b < n_buckets && ok; b++) {
@@ -294,6 +342,8 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
             }
         }
     } else {
+        // the row group's outlier columns, once (the partition of its first bucket range)
+        if (L.n_out > 0 && part_id % n_split == 0) outlier_columns(L, xs, part, r0, r1, warp, lane);
         const uint32_t rep16 = (uint32_t)(lane & 7) * 16u;
         const uint32_t cb2_lane = CB2_ABS | rep16;
         uint32_t tab_lane = TAB_ABS | rep16;
@@ -373,10 +423,11 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     // ---- bias term, conversion, store (a7 epilogue) ----
     float bterm = 0.f;
     for (int w = 0; w < BK_WARPS; w++) bterm += red[w];
-    const int m_lo = r0 * 8, n_m = min(L.M, r1 * 8) - m_lo;
+    const int m_lo = r0 * L.v, n_m = min(L.M, r1 * L.v) - m_lo;
+    const int vv = L.v;
     if (n_split == 1) {
         for (int i = threadIdx.x; i < n_m; i += BK_THREADS)
-            store_out(P.out[li], (long long)m_lo + i, part[i] + bterm, L.out_dtype);
+            store_out(P.out[li], (long long)m_lo + i, part[(i / vv) * 8 + i % vv] + bterm, L.out_dtype);
         return;
     }
     // The row group's other CTAs hold the sums over their buckets.  Every CTA leaves its sums in its slot and
@@ -384,7 +435,8 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     // and stores.  Nobody waits for anybody, and the counter is back at zero for the next launch.
     const int first_cta = (int)blockIdx.x - part_id % n_split;             // the row group's first CTA
     float *mine = P.slots + (size_t)blockIdx.x * (64 * 8);
-    for (int i = threadIdx.x; i < n_m; i += BK_THREADS) mine[i] = part[i];
+    const int n_part = (r1 - r0) * 8;
+    for (int i = threadIdx.x; i < n_part; i += BK_THREADS) mine[i] = part[i];
     __threadfence();
     __syncthreads();
     __shared__ int is_last;
@@ -398,7 +450,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     __threadfence();
     for (int i = threadIdx.x; i < n_m; i += BK_THREADS) {
         float y = 0.f;
-        for (int h = 0; h < n_split; h++) y += __ldcg(P.slots + (size_t)(first_cta + h) * (64 * 8) + i);
+        for (int h = 0; h < n_split; h++) y += __ldcg(P.slots + (size_t)(first_cta + h) * (64 * 8) + (i / vv) * 8 + i % vv);
         store_out(P.out[li], (long long)m_lo + i, y + bterm, L.out_dtype);
     }
 }

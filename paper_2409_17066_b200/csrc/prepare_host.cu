@@ -34,28 +34,27 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
     const int n_rows = r1 - r0, nb8 = g.n_buckets * 8;
     const uint32_t pad = (uint32_t)g.N << 17;
 
-    // every row's entries sorted by (bucket, residue of the main index mod 8)
-    std::vector<uint32_t> sorted((size_t)n_rows * g.N);
+    // every row's entries sorted by (bucket, residue of the main index mod 8); the column of an entry is the
+    // stored column (the main columns follow the outlier columns)
+    std::vector<uint32_t> sorted((size_t)n_rows * g.Nc);
     std::vector<int> count((size_t)n_rows * nb8, 0), start((size_t)n_rows * nb8);
+    std::vector<int32_t> row1((size_t)g.Nc), row2((size_t)g.Nc, 0);
     for (int r = r0; r < r1; r++) {
-        const uint16_t *row1 = reinterpret_cast<const uint16_t *>(idx1 + (long long)r * stride1);
-        const uint8_t *row2 = idx2 ? idx2 + (long long)r * stride2 : nullptr;
+        unpack_host(idx1 + (long long)r * stride1, 1, g.Nc, g.k1, row1.data());
+        if (idx2) unpack_host(idx2 + (long long)r * stride2, 1, g.Nc, g.k2, row2.data());
         int *cnt = &count[(size_t)(r - r0) * nb8], *st = &start[(size_t)(r - r0) * nb8];
-        for (int n = 0; n < g.N; n++) {
-            uint32_t id = row1[n];
-            if (id >= (uint32_t)g.k1) id = (uint32_t)g.k1 - 1;             // clamp, as every kernel does
-            cnt[(id >> 12) * 8 + (id & 7)]++;
+        for (int c = 0; c < g.Nc; c++) {
+            if (row1[c] >= g.k1) row1[c] = g.k1 - 1;                       // clamp, as every kernel does
+            if (g.k2 > 0 && row2[c] >= g.k2) row2[c] = g.k2 - 1;
+            cnt[(row1[c] >> 12) * 8 + (row1[c] & 7)]++;
         }
         int at = 0;
         for (int i = 0; i < nb8; i++) { st[i] = at; at += cnt[i]; }
         std::vector<int> fill(st, st + nb8);
-        uint32_t *dst = &sorted[(size_t)(r - r0) * g.N];
-        for (int n = 0; n < g.N; n++) {
-            uint32_t id = row1[n];
-            if (id >= (uint32_t)g.k1) id = (uint32_t)g.k1 - 1;
-            uint32_t id2 = row2 ? row2[n] : 0u;
-            if (g.k2 > 0 && id2 >= (uint32_t)g.k2) id2 = (uint32_t)g.k2 - 1;
-            dst[fill[(id >> 12) * 8 + (id & 7)]++] = ((id & 0xFFFu) >> 3) | (id2 << 9) | ((uint32_t)n << 17);
+        uint32_t *dst = &sorted[(size_t)(r - r0) * g.Nc];
+        for (int c = 0; c < g.Nc; c++) {
+            const uint32_t id = (uint32_t)row1[c], id2 = (uint32_t)row2[c];
+            dst[fill[(id >> 12) * 8 + (id & 7)]++] = ((id & 0xFFFu) >> 3) | (id2 << 9) | ((uint32_t)(g.n_out + c) << 17);
         }
     }
 
@@ -126,7 +125,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
                         steps_left[k] = 4 * sg.nq;
                         for (int c = 0; c < 8; c++) {
                             for (int q = 0; q < 32; q++) stack[k][c][q].clear();
-                            const uint32_t *list = &sorted[(size_t)r * g.N + start[(size_t)r * nb8 + b * 8 + c] + sg.first[c]];
+                            const uint32_t *list = &sorted[(size_t)r * g.Nc + start[(size_t)r * nb8 + b * 8 + c] + sg.first[c]];
                             left[k][c] = sg.n[c];
                             for (int i = 0; i < left[k][c]; i++) stack[k][c][(list[i] >> 18) & 31u].push_back(list[i]);
                         }
@@ -254,7 +253,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
 int prepare_host(const PreparedGeometry &g, const uint8_t *idx1, const uint8_t *idx2, void *image, size_t image_bytes,
                  size_t *used_bytes)
 {
-    const long long stride1 = row_bytes(g.N, g.k1), stride2 = g.k2 ? row_bytes(g.N, g.k2) : 0;
+    const long long stride1 = row_bytes(g.Nc, g.k1), stride2 = g.k2 ? row_bytes(g.Nc, g.k2) : 0;
     std::vector<PartImage> parts((size_t)g.n_parts);
     unsigned n_threads = std::thread::hardware_concurrency();
     if (n_threads < 1) n_threads = 1;
@@ -281,8 +280,8 @@ int prepare_host(const PreparedGeometry &g, const uint8_t *idx1, const uint8_t *
     head[4] = (uint32_t)g.k1; head[5] = (uint32_t)g.k2; head[6] = (uint32_t)g.n_parts; head[7] = PREP_WARPS;
     head[8] = (uint32_t)g.n_buckets; head[9] = (uint32_t)n_blocks;
     head[10] = (uint32_t)lay.off_woff; head[11] = (uint32_t)lay.off_hdr; head[12] = (uint32_t)lay.off_entries;
-    head[13] = (uint32_t)lay.total; head[14] = (uint32_t)((unsigned long long)g.R * g.N);
-    head[15] = (uint32_t)g.n_split;
+    head[13] = (uint32_t)lay.total; head[14] = (uint32_t)((unsigned long long)g.R * g.Nc);
+    head[15] = (uint32_t)g.n_split; head[16] = (uint32_t)g.v; head[17] = (uint32_t)g.n_out;
     uint32_t *woff = reinterpret_cast<uint32_t *>(img + lay.off_woff);
     uint32_t *hdr = reinterpret_cast<uint32_t *>(img + lay.off_hdr);
     uint32_t *ent = reinterpret_cast<uint32_t *>(img + lay.off_entries);

@@ -12,7 +12,7 @@ constexpr int PREP_PAD_COLS = 64;           // columns N .. N+63 stand for "no e
 constexpr int PREP_MAX_N = 31680;           // the staged activations (N + 64 halves) must fit below the first bucket buffer
 
 struct PreparedGeometry {
-    int M, N, k1, k2, R, n_parts, n_buckets;
+    int M, N, v, k1, k2, n_out, Nc, R, n_parts, n_buckets;     // Nc = N - n_out main columns; stored column = n_out + c
     int n_split;                            // partitions that share a group of vector rows, each with a range of buckets
 };
 
@@ -61,8 +61,10 @@ inline PreparedLayout prepared_layout(int n_parts, unsigned long long n_blocks)
 // Layers the prepared path serves (the format text lists them).
 inline bool prepared_eligible(const LayerView &L)
 {
-    return L.v == 8 && L.k1 <= 65536 && L.s1.bits == 16 && (L.k2 == 0 || (L.k2 <= 256 && L.s2.bits == 8)) &&
-           L.n_out == 0 && L.G == 1 && !L.scale_rows && L.N <= PREP_MAX_N;
+    // vectors of 8 (16-byte codebook rows, bulk-copied slice by slice), or shorter ones with a main codebook of
+    // one bucket (widened to 16-byte rows by the kernel's threads)
+    return (L.v == 8 || (L.v < 8 && L.k1 <= PREP_BUCKET)) && L.k1 <= 65536 && (L.k2 == 0 || L.k2 <= 256) &&
+           (L.n_out == 0 || L.v0 <= 8) && L.Nc > 0 && L.G == 1 && !L.scale_rows && L.N <= PREP_MAX_N;
 }
 
 // n_parts = 0 means one partition per SM; false when a partition would hold more than PREP_MAX_ROWS rows.
@@ -71,7 +73,8 @@ inline bool prepared_geometry(const LayerView &L, int n_parts, PreparedGeometry 
     if (n_parts == 0) n_parts = device_sm_count();
     if (n_parts < 1) return false;
     if (n_parts > L.R) n_parts = L.R;
-    g->M = L.M; g->N = L.N; g->k1 = L.k1; g->k2 = L.k2; g->R = L.R; g->n_parts = n_parts;
+    g->M = L.M; g->N = L.N; g->v = L.v; g->k1 = L.k1; g->k2 = L.k2; g->n_out = L.n_out; g->Nc = L.Nc; g->R = L.R;
+    g->n_parts = n_parts;
     g->n_buckets = (L.k1 + PREP_BUCKET - 1) / PREP_BUCKET;
     g->n_split = prepared_split(L.R, g->n_buckets, n_parts);
     return ceil_div(L.R, n_parts / g->n_split) <= PREP_MAX_ROWS;
@@ -80,7 +83,7 @@ inline bool prepared_geometry(const LayerView &L, int n_parts, PreparedGeometry 
 // capacity handed out by vptq_prepare_bytes: tables for the worst block count that fits, 1.5 x 4 bytes per entry
 inline unsigned long long prepared_capacity(const PreparedGeometry &g)
 {
-    const unsigned long long entries = (unsigned long long)g.R * g.N;
+    const unsigned long long entries = (unsigned long long)g.R * g.Nc;
     const unsigned long long blocks = (entries * 3 / 2 + 127) / 128 + (unsigned long long)g.n_parts * PREP_WARPS * g.n_buckets;
     return prepared_layout(g.n_parts, blocks).total;
 }

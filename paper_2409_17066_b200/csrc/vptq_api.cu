@@ -242,7 +242,7 @@ int vptq_prepare(const vptq_layer_desc *desc, const vptq_layer_ptrs *p, int32_t 
     if ((reinterpret_cast<uintptr_t>(image) & 255u) != 0) return VPTQ_E_ALIGN;
     if (image_bytes < 256) return VPTQ_E_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const size_t b1 = (size_t)g.R * (size_t)row_bytes(g.N, g.k1), b2 = g.k2 ? (size_t)g.R * (size_t)row_bytes(g.N, g.k2) : 0;
+    const size_t b1 = (size_t)g.R * (size_t)row_bytes(g.Nc, g.k1), b2 = g.k2 ? (size_t)g.R * (size_t)row_bytes(g.Nc, g.k2) : 0;
     std::vector<uint8_t> h1, h2, himg;
     try {
         h1.resize(b1); h2.resize(b2 ? b2 : 1); himg.resize(image_bytes);

@@ -38,6 +38,13 @@ SMALL = [
     (synth.LayerSpec("p_split2", 1024, 300, v=8, k1=65536), 6),                            # 3 row groups x 2 bucket ranges
     (synth.LayerSpec("p_split8", 400, 520, v=8, k1=40000, k2=200), 8),                     # 1 row group x 8 bucket ranges
     (synth.LayerSpec("p_split4_bf16", 520, 1030, v=8, k1=65536, k2=256, x_dtype="bf16", out_dtype="bf16"), 8),
+    # other formats: vectors of 6 with 12-bit indices and outlier columns (the 7B MLP setting in small), one
+    # bucket with v = 8, vectors of 4, 15-bit indices with a split, outliers where a permutation put them
+    (synth.LayerSpec("p_v6_out", 1100, 420, v=6, k1=4096, k2=256, n_out=5, v0=4, k0=4096), 7),
+    (synth.LayerSpec("p_v8_k4096_out", 512, 300, v=8, k1=4096, n_out=3, v0=4, k0=4096), 4),
+    (synth.LayerSpec("p_v4", 260, 200, v=4, k1=1000, k2=100), 3),
+    (synth.LayerSpec("p_15bit_out", 520, 300, v=8, k1=30000, k2=256, n_out=2, v0=4, k0=256), 8),
+    (synth.LayerSpec("p_v6_perm_out", 264, 1032, v=6, k1=4096, k2=256, n_out=10, v0=4, k0=4096, permuted=True), 9),
 ]
 
 
@@ -51,7 +58,7 @@ def test_prepared_small_layers(b, spec, n_parts):
     # the device entry point wrote the host builder's image (whose content the oracle's decoder checks)
     host = b.vptq_prepare_host(dl.desc, L._keep["idx1"], L._keep["idx2"], n_parts)
     assert np.array_equal(pl.image.cpu().numpy(), host)
-    code, i1, i2 = oracle.decode_prepared(host, spec.M, spec.N, spec.k1, spec.k2)
+    code, i1, i2 = oracle.decode_prepared(host, spec.M, spec.N, spec.k1, spec.k2, v=spec.v, n_out=spec.n_out)
     assert code == 0 and np.array_equal(i1, d["idx1"]) and (spec.k2 == 0 or np.array_equal(i2, d["idx2"]))
     x = dl.upload_x(d["x"])
     y_ref = L.linear(d["x"])
@@ -155,16 +162,17 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable(
         assert rel_err(y, y_ref) <= TOL
 
 
-@pytest.mark.parametrize("name,n_parts", [("o_proj", 0), ("down_proj", 0), ("k_proj", 0)])
-def test_prepared_config3_layers_full_size(b, name, n_parts):
-    li, spec = next((i, s) for i, s in enumerate(synth.CONFIGS[3]["layers"]) if s.name == name)
-    d = synth.make_layer(spec, 3, li, 1)
+@pytest.mark.parametrize("cfg,name,n_parts", [(3, "o_proj", 0), (3, "down_proj", 0), (3, "k_proj", 0),
+                                              (2, "gate_proj", 0), (2, "down_proj", 0)])
+def test_prepared_layers_full_size(b, cfg, name, n_parts):
+    li, spec = next((i, s) for i, s in enumerate(synth.CONFIGS[cfg]["layers"]) if s.name == name)
+    d = synth.make_layer(spec, cfg, li, 1)
     L = oracle.Layer.from_synth(d)
     dl = b.DeviceLayer(d)
     pl = dl.prepared(n_parts)
     host = b.vptq_prepare_host(dl.desc, L._keep["idx1"], L._keep["idx2"], n_parts if n_parts else torch.cuda.get_device_properties(0).multi_processor_count)
     assert np.array_equal(pl.image.cpu().numpy(), host)
-    code, i1, i2 = oracle.decode_prepared(host, spec.M, spec.N, spec.k1, spec.k2)
+    code, i1, i2 = oracle.decode_prepared(host, spec.M, spec.N, spec.k1, spec.k2, v=spec.v, n_out=spec.n_out)
     assert code == 0 and np.array_equal(i1, d["idx1"]) and np.array_equal(i2, d["idx2"])
     W64 = dl.dequant().double()
     assert np.array_equal(W64.cpu().numpy().astype(np.float16).view(np.uint16), L.dequant().view(np.uint16))
@@ -172,7 +180,7 @@ def test_prepared_config3_layers_full_size(b, name, n_parts):
     y = pl.linear(dl.upload_x(d["x"]))
     assert b.vptq_workspace_status(pl.workspace(1)) == b.OK
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
-    check_outputs(y, x64, W64, L, d["x"], cta_range_rows(spec.M, spec.v, n_sm), ("cfg3-prepared", name))
+    check_outputs(y, x64, W64, L, d["x"], cta_range_rows(spec.M, spec.v, n_sm), ("cfg%d-prepared" % cfg, name))
 
 
 def test_prepared_config3_gate_and_up_in_one_launch(b):

@@ -16,13 +16,42 @@ def b():
     return binding
 
 
-def _layer(b, M, N, k1, k2, seed, flags=None):
+def _layer(b, M, N, k1, k2, seed, flags=None, v=8, n_out=0):
     rng = np.random.default_rng(seed)
-    R = -(-M // 8)
-    idx1 = rng.integers(0, k1, (R, N), dtype=np.int32)
-    idx2 = rng.integers(0, k2, (R, N), dtype=np.int32) if k2 else None
-    desc = b.make_desc(M, N, 8, k1, k2, flags=b.FLAG_SCALE_BIAS if flags is None else flags)
+    R = -(-M // v)
+    idx1 = rng.integers(0, k1, (R, N - n_out), dtype=np.int32)
+    idx2 = rng.integers(0, k2, (R, N - n_out), dtype=np.int32) if k2 else None
+    desc = b.make_desc(M, N, v, k1, k2, n_outlier=n_out, v0=4 if n_out else 0, k0=4096 if n_out else 0,
+                       flags=b.FLAG_SCALE_BIAS if flags is None else flags)
     return desc, idx1, idx2
+
+
+@pytest.mark.parametrize("M,N,v,k1,k2,n_out,n_parts", [
+    (1100, 420, 6, 4096, 256, 0, 7),      # vectors of 6 (184 vector rows, the last one ragged), 12-bit main indices
+    (1100, 420, 6, 4096, 256, 5, 7),      # the same with 5 outlier columns stored first
+    (512, 300, 8, 4096, 0, 3, 4),         # v = 8, one bucket, outlier columns, no residual stage
+    (260, 200, 4, 1000, 100, 0, 3),       # vectors of 4, 10-bit main and 7-bit residual indices
+    (520, 300, 8, 30000, 256, 2, 8),      # 15-bit main indices, 8 buckets (the last one short), two splits
+])
+def test_other_formats_decode_back(b, M, N, v, k1, k2, n_out, n_parts):
+    desc, idx1, idx2 = _layer(b, M, N, k1, k2, seed=M + N + v, v=v, n_out=n_out)
+    image = b.vptq_prepare_host(desc, oracle.pack(idx1, k1), oracle.pack(idx2, k2) if k2 else None, n_parts)
+    code, got1, got2 = oracle.decode_prepared(image, M, N, k1, k2, v=v, n_out=n_out)
+    assert code == 0
+    assert np.array_equal(got1, idx1)
+    assert np.array_equal(got2, idx2 if k2 else np.zeros_like(idx1))
+    head = image[:72].view(np.uint32)
+    assert head[14] == idx1.size and head[16] == v and head[17] == n_out
+    # the decoder is told the layer's v and outlier count: other values are a geometry mismatch
+    assert oracle.decode_prepared(image, M, N, k1, k2, v=v, n_out=n_out + 1)[0] == 2
+    if n_out:
+        # an entry that names an outlier column is refused
+        off_ent, n_blocks = int(head[12]), int(head[9])
+        ent = image[off_ent:off_ent + 512 * n_blocks].view(np.uint32)
+        j = int(np.flatnonzero((ent >> 17) < N)[0])
+        img = image.copy()
+        img[off_ent + 4 * j:off_ent + 4 * j + 4].view(np.uint32)[0] = int(ent[j]) & 0x1FFFF
+        assert oracle.decode_prepared(img, M, N, k1, k2, v=v, n_out=n_out)[0] == 7
 
 
 @pytest.mark.parametrize("M,N,k1,k2,n_parts,n_split", [
@@ -140,11 +169,14 @@ def test_eligibility_and_argument_errors(b):
     ok = b.make_desc(4096, 4096, 8, 65536, 256)
     assert b.vptq_prepare_bytes(ok, 148) > 4 * 512 * 4096
     assert b.vptq_prepare_bytes(ok, 0) > 0                                   # one partition per SM
-    for bad in (b.make_desc(4096, 4096, 6, 65536, 256),                      # v = 6
-                b.make_desc(4096, 4096, 8, 4096, 256),                       # the table fits shared memory whole
-                b.make_desc(4096, 4096, 8, 30000, 256),                      # 15-bit main indices
+    for good in (b.make_desc(4096, 4096, 8, 4096, 256),                      # one bucket
+                 b.make_desc(4096, 4096, 8, 30000, 256),                     # 15-bit main indices
+                 b.make_desc(4096, 4096, 6, 4096, 256),                      # shorter vectors, one bucket
+                 b.make_desc(4096, 4096, 8, 65536, 256, n_outlier=41, v0=4, k0=4096)):
+        assert b.vptq_prepare_bytes(good, 148) > 0
+    for bad in (b.make_desc(4096, 4096, 6, 65536, 256),                      # v = 6 with more than one bucket
                 b.make_desc(4096, 4096, 8, 65536, 4096),                     # 12-bit residual indices
-                b.make_desc(4096, 4096, 8, 65536, 256, n_outlier=41, v0=4, k0=4096),
+                b.make_desc(4096, 4096, 8, 65536, 256, n_outlier=41, v0=12, k0=4096),
                 b.make_desc(4096, 4096, 8, 65536, 256, n_groups=4),
                 b.make_desc(4096, 40000, 8, 65536, 256)):                    # N beyond the staged activations
         assert b.lib.vptq_prepare_bytes(C.byref(bad), 148) == b.E_UNSUPPORTED
