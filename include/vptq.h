@@ -230,14 +230,18 @@ int vptq_linear_fused_launches(const vptq_layer_desc *descs, int32_t n_layers, i
  * vptq_linear, copies out_dev -> out_host, all asynchronously on `stream` (the caller
  * synchronises the stream before reading out_host).  x_host/out_host should be pinned
  * host memory; x_dev ([B][N]) and out_dev ([B][M]) are caller-owned device staging
- * buffers.  The weights (p) stay resident on the device. */
+ * buffers.  The weights (p) stay resident on the device.  On the path "decode_bucket_fma", whose
+ * kernel stores every output element exactly once, a pinned out_host is written by the kernel
+ * itself (through the device's address of that buffer) and out_dev is left untouched: the result
+ * crosses the bus once either way, without a copy queued behind the kernel. */
 int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
                         const vptq_layer_ptrs *p, void *out_host,
                         void *x_dev, void *out_dev,
                         void *workspace, size_t workspace_bytes, void *stream);
 
 /* vptq_linear_fused with HOST activations and HOST results: one copy of x_host -> x_dev, the fused
- * call, one copy outs_dev[l] -> outs_host[l] per layer, all asynchronous on `stream`. */
+ * call, one copy outs_dev[l] -> outs_host[l] per layer, all asynchronous on `stream` (on the path
+ * "fused_decode_bucket_fma" with all outs_host pinned, the kernel writes them itself, as above). */
 int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptrs *ptrs, int32_t n_layers,
                               const void *x_host, int32_t B, void *const *outs_host,
                               void *x_dev, void *const *outs_dev,

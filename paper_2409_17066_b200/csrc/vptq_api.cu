@@ -445,6 +445,16 @@ const char *vptq_linear_fused_path(const vptq_layer_desc *descs, int32_t n_layer
     return linear_fused_path_name(Ls, flags, n_layers, B);
 }
 
+// The device's address of a pinned (page-locked, mapped) host buffer, or nullptr for any other memory.  A kernel
+// that stores every output element exactly once with plain stores can write such a buffer itself, which saves
+// the copy that would otherwise follow it on the stream.
+static void *device_alias_of_pinned_host(void *host)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+}
+
 int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
                         const vptq_layer_ptrs *p, void *out_host,
                         void *x_dev, void *out_dev,
@@ -459,6 +469,11 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
     size_t ob = (size_t)B * desc->M * (desc->out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
+    // the prepared-image kernel stores each output once: into the pinned host buffer directly when it can
+    if (strcmp(vptq_linear_path(desc, B), "decode_bucket_fma") == 0) {
+        void *alias = device_alias_of_pinned_host(out_host);
+        if (alias != nullptr) return vptq_linear(desc, x_dev, B, p, alias, workspace, workspace_bytes, stream);
+    }
     rc = vptq_linear(desc, x_dev, B, p, out_dev, workspace, workspace_bytes, stream);
     if (rc != VPTQ_OK) return rc;
     e = cudaMemcpyAsync(out_host, out_dev, ob, cudaMemcpyDeviceToHost, st);
@@ -482,6 +497,12 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)B * descs[0].N * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
+    if (strcmp(vptq_linear_fused_path(descs, n_layers, B), "fused_decode_bucket_fma") == 0) {
+        void *alias[VPTQ_MAX_FUSED_LAYERS];
+        bool all = true;
+        for (int l = 0; l < n_layers; l++) all = (alias[l] = device_alias_of_pinned_host(outs_host[l])) != nullptr && all;
+        if (all) return vptq_linear_fused(descs, ptrs, n_layers, x_dev, B, alias, workspace, workspace_bytes, stream);
+    }
     const int rc = vptq_linear_fused(descs, ptrs, n_layers, x_dev, B, outs_dev, workspace, workspace_bytes, stream);
     if (rc != VPTQ_OK) return rc;
     for (int l = 0; l < n_layers; l++) {

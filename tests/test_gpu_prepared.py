@@ -202,3 +202,45 @@ def test_prepared_config3_gate_and_up_in_one_launch(b):
         W64 = dl.dequant().double()
         sp = d["spec"]
         check_outputs(y, x64, W64, L, d["x"], cta_range_rows(sp.M, sp.v, n_sm // 2), ("cfg3-prepared-fused", sp.name))
+
+
+def test_host_io_over_prepared_images_pinned_and_pageable_results(b):
+    """vptq_linear_host_io / vptq_linear_fused_host_io on the prepared path: a pinned result buffer is written by
+    the kernel itself (the device staging buffer stays as it was), a pageable one arrives through the copy; the
+    numbers are the same."""
+    spec = synth.LayerSpec("p_hio", 520, 1030, v=8, k1=65536, k2=256, out_dtype="fp32")
+    d = synth.make_layer(spec, 96, 0, 1)
+    y_ref = oracle.Layer.from_synth(d).linear(d["x"])
+    pl = b.DeviceLayer(d).prepared(8)
+    x_host = torch.from_numpy(np.ascontiguousarray(d["x"])).view(torch.float16).pin_memory()
+    x_dev = torch.empty((1, spec.N), dtype=torch.float16, device="cuda")
+    marker = 12345.0
+    results = []
+    for pinned in (True, False):
+        out_host = torch.full((1, spec.M), float("nan"), dtype=torch.float32)
+        if pinned:
+            out_host = out_host.pin_memory()
+        out_dev = torch.full((1, spec.M), marker, dtype=torch.float32, device="cuda")
+        b.vptq_linear_host_io(pl.desc, x_host, pl.ptrs, out_host, x_dev, out_dev, pl.workspace(1))
+        torch.cuda.synchronize()
+        assert b.vptq_workspace_status(pl.workspace(1)) == b.OK
+        assert rel_err(out_host.numpy(), y_ref) <= TOL
+        assert bool((out_dev == marker).all().item()) == pinned          # untouched only when the kernel wrote the host buffer
+        results.append(out_host.clone())
+    assert rel_err(results[0].numpy(), results[1].numpy().astype(np.float64)) <= 1e-5
+    # two layers in one launch, one result pinned and one not: the copies are used for both
+    specs = [synth.LayerSpec("p_hf%d" % i, M, 1030, v=8, k1=65536, k2=256) for i, M in enumerate((520, 264))]
+    ds = [synth.make_layer(sp, 97 + i, 0, 1) for i, sp in enumerate(specs)]
+    ds[1]["x"] = ds[0]["x"]
+    pls = [b.DeviceLayer(dd).prepared(p) for dd, p in zip(ds, (8, 4))]
+    fused = b.FusedLayers(pls)
+    assert fused.path(1) == "fused_decode_bucket_fma"
+    xh = torch.from_numpy(np.ascontiguousarray(ds[0]["x"])).view(torch.float16).pin_memory()
+    for pin in ((True, True), (True, False)):
+        outs_host = [torch.full((1, sp.M), float("nan"), dtype=torch.float16) for sp in specs]
+        outs_host = [o.pin_memory() if pnd else o for o, pnd in zip(outs_host, pin)]
+        outs_dev = [torch.zeros((1, sp.M), dtype=torch.float16, device="cuda") for sp in specs]
+        fused.linear_host_io(xh, outs_host, x_dev, outs_dev)
+        torch.cuda.synchronize()
+        for dd, oh in zip(ds, outs_host):
+            assert rel_err(oh.float().numpy(), oracle.Layer.from_synth(dd).linear(dd["x"])) <= TOL
