@@ -183,13 +183,20 @@ def test_prepared_layers_full_size(b, cfg, name, n_parts):
     check_outputs(y, x64, W64, L, d["x"], cta_range_rows(spec.M, spec.v, n_sm), ("cfg%d-prepared" % cfg, name))
 
 
-def test_prepared_config3_gate_and_up_in_one_launch(b):
+@pytest.mark.parametrize("which", [(4, 5), (0, 1, 2)], ids=["gate+up", "q+k+v"])
+def test_prepared_config3_fused_groups_full_size(b, which):
+    # the two fused calls of the headline step, with the CTA shares the benchmark uses (74 + 74; 116 + 16 + 16,
+    # whose images split their buckets over four CTAs per row group)
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     layers = synth.CONFIGS[3]["layers"]
-    ds = [synth.make_layer(layers[li], 3, li, 1) for li in (4, 5)]
-    ds[1]["x"] = ds[0]["x"]
+    ds = [synth.make_layer(layers[li], 3, li, 1) for li in which]
+    for d in ds[1:]:
+        d["x"] = ds[0]["x"]
     dls = [b.DeviceLayer(d) for d in ds]
-    pls = [dl.prepared(p) for dl, p in zip(dls, (n_sm // 2, n_sm - n_sm // 2))]
+    shares = b.prepared_shares([d["spec"].R for d in ds], n_sm)
+    if n_sm == 148:
+        assert shares == ([74, 74] if len(which) == 2 else [116, 16, 16])
+    pls = [dl.prepared(p) for dl, p in zip(dls, shares)]
     fused = b.FusedLayers(pls)
     assert fused.path(1) == "fused_decode_bucket_fma"
     x = dls[0].upload_x(ds[0]["x"])
@@ -197,11 +204,11 @@ def test_prepared_config3_gate_and_up_in_one_launch(b):
     fused.linear(x, outs)
     assert b.vptq_workspace_status(fused.workspace(1)) == b.OK
     x64 = torch.from_numpy(x_as_float64(ds[0]["spec"], ds[0]["x"])).cuda()
-    for d, dl, y in zip(ds, dls, outs):
+    for d, dl, y, p in zip(ds, dls, outs, shares):
         L = oracle.Layer.from_synth(d)
         W64 = dl.dequant().double()
         sp = d["spec"]
-        check_outputs(y, x64, W64, L, d["x"], cta_range_rows(sp.M, sp.v, n_sm // 2), ("cfg3-prepared-fused", sp.name))
+        check_outputs(y, x64, W64, L, d["x"], cta_range_rows(sp.M, sp.v, p), ("cfg3-prepared-fused", sp.name))
 
 
 def test_host_io_over_prepared_images_pinned_and_pageable_results(b):
