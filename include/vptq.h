@@ -270,7 +270,8 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *                 multiple of 256)  [13] total bytes  [14] number of real entries = R * (N - n_outlier)
  *                 [15] n_split  [16] v  [17] n_outlier; rest zero
  *   partitions    a partition is the work of one CTA.  The R vector rows are cut into
- *            n_parts / n_split row groups, group g = rows [R*g/groups, R*(g+1)/groups), at most 63 rows; the
+ *            groups = n_parts / n_split row groups of R / groups rows, the first R % groups of them one row
+ *            longer (group g starts at row g * (R / groups) + min(g, R % groups)), at most 63 rows; the
  *            n_split partitions of a group (p = g*n_split + h) each hold the group's entries of one range of
  *            buckets, [n_buckets*h/n_split, n_buckets*(h+1)/n_split).  n_split is the largest of 8, 4, 2, 1
  *            that divides n_parts, does not exceed n_buckets and keeps a group within 63 rows: a CTA then

@@ -484,7 +484,10 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
     uint32_t prev_end = 0;
     for (uint32_t p = 0; p < n_parts; p++) {
         const uint32_t grp = p / n_split, piece = p % n_split;
-        const int64_t r0 = R * grp / n_groups, r1 = R * (grp + 1) / n_groups;
+        /* R = n_groups * base + rem: the first rem groups hold base + 1 rows, the others base */
+        const int64_t base_rows = R / n_groups, rem_rows = R % n_groups;
+        const int64_t r0 = grp * base_rows + ((int64_t)grp < rem_rows ? (int64_t)grp : rem_rows);
+        const int64_t r1 = r0 + base_rows + ((int64_t)grp < rem_rows ? 1 : 0);
         const uint32_t bucket_lo = n_buckets * piece / n_split, bucket_hi = n_buckets * (piece + 1) / n_split;
         if (r1 - r0 > 63) return 11;
         for (uint32_t w = 0; w < n_warps; w++) {

@@ -16,7 +16,7 @@ struct PreparedGeometry {
     int n_split;                            // partitions that share a group of vector rows, each with a range of buckets
 };
 
-// Partition p of an image: row group p / n_split (the groups split the R vector rows evenly) and the
+// Partition p of an image: row group p / n_split (the groups split the R vector rows evenly, the longer ones first) and the
 // h-th of n_split bucket ranges, h = p % n_split.
 struct PreparedPart {
     int r0, r1, b0, b1;
@@ -25,8 +25,11 @@ __host__ __device__ inline PreparedPart prepared_part(int R, int n_buckets, int 
 {
     const int groups = n_parts / n_split, g = p / n_split, h = p - g * n_split;
     PreparedPart q;
-    q.r0 = (int)((long long)R * g / groups);
-    q.r1 = (int)((long long)R * (g + 1) / groups);
+    // the first R % groups groups hold one row more: CTAs start in index order, a few microseconds apart when the
+    // previous kernel's CTAs end one by one, so the longer groups go to the CTAs that start first
+    const int base = R / groups, rem = R % groups;
+    q.r0 = g * base + (g < rem ? g : rem);
+    q.r1 = q.r0 + base + (g < rem ? 1 : 0);
     q.b0 = n_buckets * h / n_split;
     q.b1 = n_buckets * (h + 1) / n_split;
     return q;
