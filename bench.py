@@ -48,11 +48,10 @@ def read_peaks():
 # An entry is removed (-> null in the output) when its kernel changes after the capture.
 NCU_DRAM_BYTES_PER_ALGORITHMIC_BYTE = {
     # kernel: (ratio, source file of the kernel, first 12 hex digits of its SHA-1 when the capture was taken)
-    # profiles/decode_l2_fma_kernel_config3_gate_up_fused_B1.md: (178.44 + 3.68) MB DRAM / 178.33 MB algorithmic
-    # (taken before the mixed-precision fma and the ordered partial sums went into the file: null until re-captured)
-    "decode_l2_fma_kernel": (1.021, "decode_l2_fma.cu", "captured-before-later-edits"),
-    # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.95 MB (same remark)
-    "decode_smem_fma_kernel": (1.003, "decode_smem_fma.cu", "captured-before-later-edits"),
+    # profiles/decode_l2_fma_kernel_config3_gate_up_fused_B1.md: (178.38 + 3.18) MB DRAM / 178.33 MB algorithmic
+    "decode_l2_fma_kernel": (1.018, "decode_l2_fma.cu", "15af2fb60845"),
+    # profiles/decode_smem_fma_kernel_config2_gate_proj_B1.md: 19.00 MB / 18.92 MB
+    "decode_smem_fma_kernel": (1.004, "decode_smem_fma.cu", "160ad3290bed"),
     # profiles/decode_smem_tc_kernel_config2_gate_proj_B8.md: 21.46 MB / 19.0 MB (the 0.5 MB fragment image and the
     # pre-pass's traffic included)
     "decode_smem_tc_kernel": (1.13, "decode_smem_tc.cu", "ccf102769587"),
