@@ -230,7 +230,9 @@ int vptq_linear_fused_launches(const vptq_layer_desc *descs, int32_t n_layers, i
  * vptq_linear, copies out_dev -> out_host, all asynchronously on `stream` (the caller
  * synchronises the stream before reading out_host).  x_host/out_host should be pinned
  * host memory; x_dev ([B][N]) and out_dev ([B][M]) are caller-owned device staging
- * buffers.  The weights (p) stay resident on the device.  On the path "decode_bucket_fma", whose
+ * buffers.  The weights (p) stay resident on the device.  Pinned activations of at most 256 KB are
+ * brought over by a small kernel that reads x_host through the device's address of that buffer (it
+ * starts sooner on the stream than a copy); larger or pageable ones by cudaMemcpyAsync.  On the path "decode_bucket_fma", whose
  * kernel stores every output element exactly once, a pinned out_host is written by the kernel
  * itself (through the device's address of that buffer) and out_dev is left untouched: the result
  * crosses the bus once either way, without a copy queued behind the kernel. */

@@ -455,6 +455,32 @@ static void *device_alias_of_pinned_host(void *host)
     return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
 }
 
+// Small activations from pinned host memory: a kernel that reads them over the bus and writes the device buffer
+// starts sooner on a stream than a copy does (no copy engine to wake), and the decode kernel behind it may begin
+// its prologue while it runs.  16-byte words; `n16` of them.
+constexpr size_t FETCH_MAX_BYTES = 256 * 1024;
+__global__ void __launch_bounds__(256) fetch_host_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int n16)
+{
+    pdl_launch_dependents();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i < n16) dst[i] = src[i];
+}
+
+// x_host -> x_dev on the stream: by that kernel when x_host is pinned, both ends are 16-byte aligned and the size
+// is a small multiple of 16 bytes, else by cudaMemcpyAsync.
+static cudaError_t activations_to_device(void *x_dev, const void *x_host, size_t bytes, cudaStream_t st)
+{
+    if (bytes <= FETCH_MAX_BYTES && bytes % 16 == 0 && (reinterpret_cast<uintptr_t>(x_dev) & 15u) == 0) {
+        void *alias = device_alias_of_pinned_host(const_cast<void *>(x_host));
+        if (alias != nullptr && (reinterpret_cast<uintptr_t>(alias) & 15u) == 0) {
+            const int n16 = (int)(bytes / 16);
+            fetch_host_kernel<<<(n16 + 255) / 256, 256, 0, st>>>(reinterpret_cast<const uint4 *>(alias), reinterpret_cast<uint4 *>(x_dev), n16);
+            return cudaGetLastError();
+        }
+    }
+    return cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, st);
+}
+
 int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t B,
                         const vptq_layer_ptrs *p, void *out_host,
                         void *x_dev, void *out_dev,
@@ -467,7 +493,7 @@ int vptq_linear_host_io(const vptq_layer_desc *desc, const void *x_host, int32_t
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     size_t xb = (size_t)B * desc->N * 2;
     size_t ob = (size_t)B * desc->M * (desc->out_dtype == VPTQ_DTYPE_FP32 ? 4 : 2);
-    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, xb, cudaMemcpyHostToDevice, st);
+    cudaError_t e = activations_to_device(x_dev, x_host, xb, st);
     if (e != cudaSuccess) return cuda_fail(e);
     // the prepared-image kernel stores each output once: into the pinned host buffer directly when it can
     if (strcmp(vptq_linear_path(desc, B), "decode_bucket_fma") == 0) {
@@ -495,7 +521,7 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
         if (outs_host[l] == nullptr || outs_dev[l] == nullptr) return VPTQ_E_NULL;
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)B * descs[0].N * 2, cudaMemcpyHostToDevice, st);
+    cudaError_t e = activations_to_device(x_dev, x_host, (size_t)B * descs[0].N * 2, st);
     if (e != cudaSuccess) return cuda_fail(e);
     if (strcmp(vptq_linear_fused_path(descs, n_layers, B), "fused_decode_bucket_fma") == 0) {
         void *alias[VPTQ_MAX_FUSED_LAYERS];
