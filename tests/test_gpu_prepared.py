@@ -228,11 +228,15 @@ def test_host_io_over_prepared_images_pinned_and_pageable_results(b):
         if pinned:
             out_host = out_host.pin_memory()
         out_dev = torch.full((1, spec.M), marker, dtype=torch.float32, device="cuda")
-        b.vptq_linear_host_io(pl.desc, x_host, pl.ptrs, out_host, x_dev, out_dev, pl.workspace(1))
+        # pageable activations go through the copy, pinned ones are fetched by a kernel
+        x_in = x_host if pinned else torch.from_numpy(np.ascontiguousarray(d["x"])).view(torch.float16)
+        x_dev.zero_()
+        b.vptq_linear_host_io(pl.desc, x_in, pl.ptrs, out_host, x_dev, out_dev, pl.workspace(1))
         torch.cuda.synchronize()
         assert b.vptq_workspace_status(pl.workspace(1)) == b.OK
         assert rel_err(out_host.numpy(), y_ref) <= TOL
         assert bool((out_dev == marker).all().item()) == pinned          # untouched only when the kernel wrote the host buffer
+        assert torch.equal(x_dev.cpu().view(torch.int16), x_host.view(torch.int16))      # the staging buffer holds the activations
         results.append(out_host.clone())
     assert rel_err(results[0].numpy(), results[1].numpy().astype(np.float64)) <= 1e-5
     # two layers in one launch, one result pinned and one not: the copies are used for both
