@@ -281,7 +281,8 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *            transfer behind.  The CTAs of a group add their partial sums up through the workspace.
  *   woff     uint32 [n_parts * n_warps + 1]: warp w of partition p owns blocks [woff[p*n_warps + w],
  *            woff[p*n_warps + w + 1])
- *   hdr      uint32 [n_blocks]: bits 24..31 = bucket of the block; bits 6q..6q+5 (q = 0..3) = vector row,
+ *   hdr      uint32 [n_blocks]: bits 24..31 = bucket of the block, counted from the first bucket of the
+ *            partition's range; bits 6q..6q+5 (q = 0..3) = vector row,
  *            relative to the partition's first row, that the lanes 8q..8q+7 work on in this block, or 63
  *            when those lanes have nothing to do in it.  Buckets ascend within a warp's range and stay
  *            within the partition's range.

@@ -500,7 +500,7 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
             for (uint32_t b = lo; b < hi; b++) {
                 uint32_t h;
                 memcpy(&h, hdr_b + 4ull * b, 4);
-                const uint32_t bucket = h >> 24;
+                const uint32_t bucket = bucket_lo + (h >> 24);      /* the field counts from the partition's first bucket */
                 if (bucket < bucket_lo || bucket >= bucket_hi || bucket < last_bucket) return 5;
                 last_bucket = bucket;
                 for (int lane = 0; lane < 32; lane++) {

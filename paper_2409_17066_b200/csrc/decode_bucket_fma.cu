@@ -245,13 +245,9 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
     }
     for (int i = threadIdx.x; i < 64 * 8; i += BK_THREADS) part[i] = 0.f;
 
-    // consumer warps: the first blocks of the run are in flight before the activations are touched.  A header
-    // word is kept with its bucket counted from the partition's first (one below the range stays at 0).
-    const uint32_t first24 = (uint32_t)b_first << 24;
-    auto load_hdr = [&](const uint32_t *p) {
-        const uint32_t h = __ldg(p);
-        return h >= first24 ? h - first24 : h & 0xFFFFFFu;
-    };
+    // consumer warps: the first blocks of the run are in flight before the activations are touched (a header
+    // word counts its bucket from the partition's first)
+    auto load_hdr = [&](const uint32_t *p) { return __ldg(p); };
     int q = 0, qe = 0;
     uint4 eb[BK_DEPTH];
     uint32_t hb[BK_DEPTH];

@@ -225,7 +225,7 @@ void build_partition(const PreparedGeometry &g, const uint8_t *idx1, long long s
         long long j = 0;
         for (int w = 0; w < PREP_WARPS; w++) {
             for (const long long j1 = j + share[w]; j < j1; j++) {
-                uint32_t h = (uint32_t)b << 24;
+                uint32_t h = (uint32_t)(b - pp.b0) << 24;            // counted from the partition's first bucket
                 const size_t base = w_ent[w].size();
                 w_ent[w].resize(base + 128, pad);
                 for (int k = 0; k < 4; k++) {
