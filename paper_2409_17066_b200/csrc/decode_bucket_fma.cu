@@ -344,17 +344,20 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
         const uint32_t cb2_lane = CB2_ABS | rep16;
         uint32_t tab_lane = TAB_ABS | rep16;
         const uint32_t pad = (uint32_t)L.N << 17;
-        const int qid = lane >> 3;
-        const uint32_t qmask = 0xFFu << (8 * qid);
+        const uint32_t qmask = 0xFFu << (lane & 24);
+        // the quarter's row field of a header word, compared in place: all six bits set = no row
+        const uint32_t row_mask = 63u << (6 * (lane >> 3));
+        uint32_t cur_field = row_mask;
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; j++) acc[j] = 0.f;
-        int cur_row = 63, cur_b = -1;        // 63: no row yet
+        int cur_b = -1;
         bool ok = true;
 
         // the quarter warp's 8 sums per lane -> one output component per lane -> partial sums of the CTA
         auto flush = [&]() {
-            if (cur_row == 63) return;
+            if (cur_field == row_mask) return;
+            const int cur_row = (int)(cur_field >> (6 * (lane >> 3)));
             float v[8];
 #pragma unroll
             for (int j = 0; j < 8; j++) { v[j] = acc[j]; acc[j] = 0.f; }
@@ -369,7 +372,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                     }
             }
             atomicAdd(part + cur_row * 8 + (lane & 7), v[0]);
-            cur_row = 63;
+            cur_field = row_mask;
         };
         // every warp visits every bucket in order: wait for it, work, hand its buffer back
         auto enter = [&](int b) {
@@ -380,11 +383,12 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                 ok = __all_sync(0xffffffffu, ok);        // one lane giving up ends the warp's work
             }
             tab_lane = (TAB_ABS + (uint32_t)(cur_b & 1) * 65536u) | rep16;
+            if (!ok) qe = 0;                              // a wait that gave up ends the warp's run
         };
-        while (q < qe && ok) {
+        while (q < qe) {
 #pragma unroll
             for (int d = 0; d < BK_DEPTH; d++) {
-                if (q + d < qe && ok) {
+                if (q + d < qe) {
                     const uint32_t e[4] = {eb[d].x, eb[d].y, eb[d].z, eb[d].w};
                     const uint32_t h = hb[d];
                     if (q + d + BK_DEPTH < qe) {
@@ -393,13 +397,14 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                     }
                     const int b = min((int)(h >> 24), n_buckets - 1);
                     if (b > cur_b) { __syncwarp(); enter(b); }
-                    if (ok) {
-                        const int row = (int)((h >> (6 * qid)) & 63u);
-                        if (row != 63 && row != cur_row) {
+                    if (q + d < qe) {
+                        const uint32_t field = h & row_mask;
+                        if (field != row_mask && field != cur_field) {
                             flush();
-                            cur_row = row < r1 - r0 ? row : 63;       // a row outside the partition is ignored
+                            // a row outside the partition is ignored
+                            cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
                         }
-                        if (cur_row != 63) {
+                        if (cur_field != row_mask) {
 #pragma unroll
                             for (int s = 0; s < 4; s++) slot<RES>(e[s], pad, tab_lane, cb2_lane, acc);
                         }
