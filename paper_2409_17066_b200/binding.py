@@ -223,7 +223,7 @@ def prepared_shares(vector_rows, n_sm: int, n_buckets: int = 16):
     its n_buckets = ceil(k1 / 4096) buckets over that many CTAs per row group (at most 63 rows in a group)."""
     rows = [int(r) for r in vector_rows]
     for q in (8, 4, 2, 1):
-        if q * len(rows) > n_sm or q > max(1, n_buckets):
+        if q * len(rows) > n_sm or q > max(1, n_buckets) or (q > 1 and min(rows) < q):
             continue
         share = [q] * len(rows)
         while sum(share) + q <= n_sm:

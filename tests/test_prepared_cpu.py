@@ -202,3 +202,19 @@ def test_eligibility_and_argument_errors(b):
     assert b.vptq_linear_fused_launches([g, g], 1) == 1 and b.vptq_linear_fused_workspace_bytes([g, g], 1) == 256
     full = b.make_desc(28672, 8192, 8, 65536, 256, flags=b.FLAG_SCALE_BIAS | b.FLAG_PREPARED, prepared_parts=148)
     assert b.vptq_linear_fused_path([full, full], 1) == "one_by_one"         # 296 partitions do not fit side by side
+
+
+def test_cta_shares_of_layers_that_share_a_launch(b):
+    # q/k/v of the 70B shape: multiples of four, so that every image splits its buckets over four CTAs per row group
+    assert b.prepared_shares([1024, 128, 128], 148) == [116, 16, 16]
+    # gate/up: 48 or 49 rows per CTA leave no room for a split; the SMs are halved
+    assert b.prepared_shares([3584, 3584], 148) == [74, 74]
+    # a one-bucket codebook cannot be split whatever the rows would allow
+    assert b.prepared_shares([1835, 1835], 148, n_buckets=1) == [74, 74]
+    for rows, n_sm, nb in (([125, 65, 33], 148, 16), ([512, 512, 512], 148, 16), ([7, 900], 132, 16), ([40, 40, 40, 40], 148, 2)):
+        shares = b.prepared_shares(rows, n_sm, nb)
+        assert len(shares) == len(rows) and sum(shares) <= n_sm and all(1 <= s <= r for s, r in zip(shares, rows))
+        # what the library makes of them: every image within the 63-row limit, i.e. vptq_prepare_bytes accepts it
+        for r, s_ in zip(rows, shares):
+            d = b.make_desc(8 * r, 256, 8, 4096 * nb, 0)
+            assert b.vptq_prepare_bytes(d, s_) > 0
