@@ -286,8 +286,9 @@ int vptq_linear_fused_host_io(const vptq_layer_desc *descs, const vptq_layer_ptr
  *            relative to the partition's first row, that the lanes 8q..8q+7 work on in this block, or 63
  *            when those lanes have nothing to do in it.  Buckets ascend within a warp's range and stay
  *            within the partition's range.
- *   entries  uint32 [n_blocks][32][4]: a block is four steps of a warp; the four entries of lane L in block
- *            b are the words 4*(32*b + L) .. + 3.  An entry:
+ *   entries  uint32 [n_blocks + 2][32][4]: a block is four steps of a warp; the four entries of lane L in block
+ *            b are the words 4*(32*b + L) .. + 3; the last two blocks are spare (zero, owned by no warp: a
+ *            reader may fetch two blocks ahead of any block without a bound check).  An entry:
  *              bits 0..8    (main index mod 4096) >> 3; the three low bits of the main index are L mod 8
  *                           (so the eight lanes of a quarter warp always read eight different 16-byte banks)
  *                           and its high bits are the block's bucket

@@ -477,7 +477,8 @@ int oracle_decode_prepared(const uint8_t *image, int64_t image_bytes, int32_t M,
     if (off_woff % 256 || off_hdr % 256 || off_ent % 256 || off_woff < 256) return 3;
     if (off_woff + 4ull * ((uint64_t)n_parts * n_warps + 1) > off_hdr) return 3;
     if (off_hdr + 4ull * n_blocks > off_ent) return 3;
-    if (off_ent + 512ull * n_blocks > total || total > (uint64_t)image_bytes) return 3;
+    /* two spare blocks follow the last one */
+    if (off_ent + 512ull * ((uint64_t)n_blocks + 2u) > total || total > (uint64_t)image_bytes) return 3;
     const uint8_t *woff_b = image + off_woff, *hdr_b = image + off_hdr, *ent_b = image + off_ent;
     for (int64_t i = 0; i < R * Nc; i++) { idx1[i] = -1; idx2[i] = -1; }
     uint64_t real = 0;

@@ -385,35 +385,39 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
             tab_lane = (TAB_ABS + (uint32_t)(cur_b & 1) * 65536u) | rep16;
             if (!ok) qe = 0;                              // a wait that gave up ends the warp's run
         };
-        while (q < qe) {
-#pragma unroll
-            for (int d = 0; d < BK_DEPTH; d++) {
-                if (q + d < qe) {
-                    const uint32_t e[4] = {eb[d].x, eb[d].y, eb[d].z, eb[d].w};
-                    const uint32_t h = hb[d];
-                    if (q + d + BK_DEPTH < qe) {
-                        eb[d] = ld_stream16(entries + (size_t)(q + d + BK_DEPTH) * 32 + lane);
-                        hb[d] = load_hdr(hdr + q + d + BK_DEPTH);
-                    }
-                    const int b = min((int)(h >> 24), n_buckets - 1);
-                    if (b > cur_b) { __syncwarp(); enter(b); }
-                    if (q + d < qe) {
-                        const uint32_t field = h & row_mask;
-                        if (field != row_mask && field != cur_field) {
-                            flush();
-                            // a row outside the partition is ignored
-                            cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
-                        }
-                        if (cur_field != row_mask) {
-#pragma unroll
-                            for (int s = 0; s < 4; s++) slot<RES>(e[s], pad, tab_lane, cb2_lane, acc);
-                        }
-                        __syncwarp();
-                    }
-                }
+        // One block: its four entries per lane and its header word are in the registers of slot d; the slot is
+        // refilled with the block two ahead at once (the image ends with two spare blocks, so that this needs no
+        // bound check: what is fetched beyond the run is never used).
+        auto block = [&](const int d) {
+            const uint32_t e[4] = {eb[d].x, eb[d].y, eb[d].z, eb[d].w};
+            const uint32_t h = hb[d];
+            eb[d] = ld_stream16(entries + (size_t)(q + d + BK_DEPTH) * 32 + lane);
+            hb[d] = load_hdr(hdr + q + d + BK_DEPTH);
+            const int b = min((int)(h >> 24), n_buckets - 1);
+            if (b > cur_b) {
+                __syncwarp();
+                enter(b);
+                if (!ok) return;
             }
-            q += BK_DEPTH;
+            const uint32_t field = h & row_mask;
+            if (field != row_mask && field != cur_field) {
+                flush();
+                // a row outside the partition is ignored
+                cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
+            }
+            if (cur_field != row_mask) {
+#pragma unroll
+                for (int s = 0; s < 4; s++) slot<RES>(e[s], pad, tab_lane, cb2_lane, acc);
+            }
+            __syncwarp();
+        };
+        static_assert(BK_DEPTH == 2, "the loop below takes the blocks in pairs");
+        while (q + 1 < qe) {
+            block(0);
+            block(1);
+            q += 2;
         }
+        if (q < qe) block(0);
         flush();
         __syncwarp();
         if (ok) enter(n_buckets - 1);                 // the buckets this warp had no blocks in

@@ -8,6 +8,7 @@ namespace vptq {
 constexpr int PREP_WARPS = 31;              // consumer warps of the decode kernel; one more warp loads the buckets
 constexpr int PREP_BUCKET = 4096;           // main-codebook entries per bucket (64 KB)
 constexpr int PREP_MAX_ROWS = 63;           // vector rows per partition (6-bit row fields; 63 = idle)
+constexpr int PREP_SPARE_BLOCKS = 2;         // zero blocks after the last one: a reader may fetch two blocks ahead unchecked
 constexpr int PREP_PAD_COLS = 64;           // columns N .. N+63 stand for "no entry" (one per shared-memory bank and half)
 constexpr int PREP_MAX_N = 31680;           // the staged activations (N + 64 halves) must fit below the first bucket buffer
 
@@ -57,7 +58,7 @@ inline PreparedLayout prepared_layout(int n_parts, unsigned long long n_blocks)
     l.off_woff = 256;
     l.off_hdr = align256(l.off_woff + 4ull * ((unsigned long long)n_parts * PREP_WARPS + 1));
     l.off_entries = align256(l.off_hdr + 4ull * n_blocks);
-    l.total = align256(l.off_entries + 512ull * n_blocks);
+    l.total = align256(l.off_entries + 512ull * (n_blocks + PREP_SPARE_BLOCKS));
     return l;
 }
 
