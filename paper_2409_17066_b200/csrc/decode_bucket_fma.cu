@@ -385,6 +385,7 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
             tab_lane = (TAB_ABS + (uint32_t)(cur_b & 1) * 65536u) | rep16;
             if (!ok) qe = 0;                              // a wait that gave up ends the warp's run
         };
+        uint32_t last_h = 0xFFFFFFFFu;       // no header word has bucket 255 and four idle quarters at once
         // One block: its four entries per lane and its header word are in the registers of slot d; the slot is
         // refilled with the block two ahead at once (the image ends with two spare blocks, so that this needs no
         // bound check: what is fetched beyond the run is never used).
@@ -393,17 +394,21 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
             const uint32_t h = hb[d];
             eb[d] = ld_stream16(entries + (size_t)(q + d + BK_DEPTH) * 32 + lane);
             hb[d] = load_hdr(hdr + q + d + BK_DEPTH);
-            const int b = min((int)(h >> 24), n_buckets - 1);
-            if (b > cur_b) {
-                __syncwarp();
-                enter(b);
-                if (!ok) return;
-            }
-            const uint32_t field = h & row_mask;
-            if (field != row_mask && field != cur_field) {
-                flush();
-                // a row outside the partition is ignored
-                cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
+            // most blocks repeat the header word of the one before (same bucket, same rows): nothing to decide then
+            if (h != last_h) {
+                last_h = h;
+                const int b = min((int)(h >> 24), n_buckets - 1);
+                if (b > cur_b) {
+                    __syncwarp();
+                    enter(b);
+                    if (!ok) return;
+                }
+                const uint32_t field = h & row_mask;
+                if (field != row_mask && field != cur_field) {
+                    flush();
+                    // a row outside the partition is ignored
+                    cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
+                }
             }
             if (cur_field != row_mask) {
 #pragma unroll
