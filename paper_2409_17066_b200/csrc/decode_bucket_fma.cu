@@ -356,7 +356,11 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
 
         // the quarter warp's 8 sums per lane -> one output component per lane -> partial sums of the CTA
         auto flush = [&]() {
-            if (cur_field == row_mask) return;
+            if (cur_field == row_mask) {             // no row, or one outside the partition: whatever was summed is dropped
+#pragma unroll
+                for (int j = 0; j < 8; j++) acc[j] = 0.f;
+                return;
+            }
             const int cur_row = (int)(cur_field >> (6 * (lane >> 3)));
             float v[8];
 #pragma unroll
@@ -410,10 +414,9 @@ decode_bucket_fma_kernel(const __grid_constant__ BucketParams P)
                     cur_field = (int)(field >> (6 * (lane >> 3))) < r1 - r0 ? field : row_mask;
                 }
             }
-            if (cur_field != row_mask) {
+            // a quarter without a row holds entries that name no column: they add nothing, so nobody branches
 #pragma unroll
-                for (int s = 0; s < 4; s++) slot<RES>(e[s], pad, tab_lane, cb2_lane, acc);
-            }
+            for (int s = 0; s < 4; s++) slot<RES>(e[s], pad, tab_lane, cb2_lane, acc);
             __syncwarp();
         };
         static_assert(BK_DEPTH == 2, "the loop below takes the blocks in pairs");
